@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the Sparbit step executor on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one whole allgather (own-block copy + all ceil(log2 P) schedule steps) over P = 256
+virtual ranks with m = 64 KiB blocks: 4 GiB of receive buffers, 2*P*(P-1)*m = 8.556 GB moved.
+Prints ONE JSON line.  The metric is effective GB/s = 2*P*(P-1)*m / time per collective.
+
+With N > 1 (launched under torch.distributed.run) every rank runs an independent replica of the
+same collective on its own GPU ("replicas only": the path has no exchange between GPUs); the
+value is the sum over ranks divided by the slowest rank's time.
+
+`--impl reference` times the CPU oracle (the plain simulator under oracle/) on the host cores, on
+a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import seeded_inputs as si  # noqa: E402
+
+P_DEFAULT, M_DEFAULT = 256, 64 * 1024
+METRIC = "sparbit_allgather_effective_GBps"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (bytes; None = not captured for this workload)
+NCU_TRAFFIC_BYTES = {}
+
+
+def effective_bytes(P: int, m: int) -> int:
+    return 2 * P * (P - 1) * m
+
+
+def algorithmic_bytes(P: int, m: int) -> int:
+    """Bytes one collective must read plus write: every delivered block once each way, plus the
+    own-block copy."""
+    return 2 * P * (P - 1) * m + 2 * P * m
+
+
+def measured_peak():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            pass
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+                for n, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------------
+def time_oracle(P: int, m: int, steps: int, warmup: int, threads: int, seed: int):
+    """Seconds per collective of the CPU oracle's execute phase (message lists already built)."""
+    import oracle
+    plan = oracle.Plan(oracle.SPARBIT, P)
+    send = si.send_blocks(P, m, seed).reshape(-1)
+    recv = si.sentinel_buffer(P * P * m)
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        plan.run(m, send, recv, None, threads=threads)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    ok = bool(np.array_equal(recv.reshape(P, P * m)[P // 2], send))
+    return times, ok
+
+
+def cpu_baseline_leg(P: int, m: int, seed: int):
+    """The oracle as it stands on this machine's cores, on a bounded sample (about 10-30 s of work)."""
+    cores = os.cpu_count() or 1
+    threads = min(cores, 16)
+    try:
+        import psutil
+        free = psutil.virtual_memory().available
+    except Exception:
+        free = 8 << 30
+    ms = m
+    while P * P * ms * 2.5 > free and ms > 1024:
+        ms //= 2
+    t1, ok1 = time_oracle(P, ms, steps=1, warmup=1, threads=1, seed=seed)
+    tn, okn = time_oracle(P, ms, steps=2, warmup=0, threads=threads, seed=seed)
+    best1, bestn = min(t1), min(tn)
+    return {
+        "value": effective_bytes(P, ms) / bestn / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+        "sample": f"whole collective P={P}, m={ms} B on host buffers, execute phase only "
+                  f"(message lists prebuilt), best of 2; box has {cores} cores",
+        "single_thread_value": effective_bytes(P, ms) / best1 / 1e9,
+        "checked": bool(ok1 and okn),
+    }
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    P, m = args.P, args.m
+    cores = os.cpu_count() or 1
+    threads = min(cores, 16)
+    # bounded sample: shrink the block until (steps + warmup) collectives fit in about two minutes
+    ms = m
+    budget = 120.0
+    while True:
+        t, _ = time_oracle(P, ms, steps=1, warmup=0, threads=threads, seed=args.seed)
+        if t[0] * (args.steps + args.warmup) <= budget or ms <= 1024:
+            break
+        ms //= 4
+    times, ok = time_oracle(P, ms, steps=args.steps, warmup=args.warmup, threads=threads, seed=args.seed)
+    per = float(np.mean(times))
+    value = effective_bytes(P, ms) / per / 1e9
+    sample = (f"each step = one whole collective P={P}, m={ms} B (block shrunk from {m} B to bound the run), "
+              f"oracle execute phase on host buffers; box has {cores} cores")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"sparbit allgather P={P} m={m}B (sampled at m={ms}B)", "P": P, "block_bytes": ms},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "checked": ok,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    P, m = args.P, args.m
+    algo = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
+            "bruck": sp.ALGO_BRUCK}[args.algo]
+    exec_mode = {"auto": sp.EXEC_AUTO, "persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH,
+                 "stream": sp.EXEC_STREAM, "cluster": sp.EXEC_CLUSTER}[args.exec]
+    copy = {"auto": sp.COPY_AUTO, "vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}[args.copy]
+
+    plan = sp.Plan(P, m, algo, exec_mode)
+    plan.set_copy_path(copy)
+    seed = args.seed + rank
+    # two input sets, alternated, so that no step finds its answer already in place
+    sends = [torch.from_numpy(si.send_blocks(P, m, seed + k).reshape(-1)).to(dev) for k in range(2)]
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    work = None
+    if algo == sp.ALGO_BRUCK:
+        work = torch.empty(P * P * m, dtype=torch.uint8, device=dev)
+        plan.set_workspace(work, P * P * m)
+    stream = torch.cuda.Stream(device=dev)
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        for it in range(args.warmup):
+            plan.allgather(sends[it & 1], recv, stream)
+        stream.synchronize()
+        assert plan.status() == sp.OK
+
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.25)
+        k0, g0 = plan.launch_counts()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        barrier()
+        t_wall0 = time.time()
+        ev[0].record(stream)
+        for it in range(args.steps):
+            plan.allgather(sends[it & 1], recv, stream)
+            ev[it + 1].record(stream)
+        stream.synchronize()
+        barrier()
+        t_wall1 = time.time()
+        k1, g1 = plan.launch_counts()
+    assert plan.status() == sp.OK
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # the last collective's result, checked against the result's definition on the device
+    last_send = sends[(args.steps - 1) & 1]
+    view = recv.view(P, P * m)
+    checked = all(bool(torch.equal(view[r], last_send)) for r in (0, P // 3, P - 1))
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if use_dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    max_total_ms = float(t.item())
+    ms_per_step = max_total_ms / args.steps
+    value = world * effective_bytes(P, m) / (ms_per_step * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point (pinned host memory; H2D + D2H inside)
+    e2e = None
+    if not args.no_e2e:
+        hs = torch.from_numpy(si.send_blocks(P, m, seed + 7).reshape(-1)).pin_memory()
+        hr = torch.empty(P * P * m, dtype=torch.uint8).pin_memory()
+        e2e_steps = max(1, min(args.steps, 3))
+        hplan = sp.Plan(P, m, algo, exec_mode)
+        hplan.set_copy_path(copy)
+        hplan.allgather_host(hs.numpy(), hr.numpy())  # warm-up: allocates device staging
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            hplan.allgather_host(hs.numpy(), hr.numpy())
+        torch.cuda.synchronize(dev)
+        dt = (time.perf_counter() - t0) / e2e_steps
+        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if use_dist:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dt = float(tt.item())
+        ok = bool(np.array_equal(hr.numpy()[(P - 1) * P * m:], hs.numpy()))
+        e2e = {"value": world * effective_bytes(P, m) / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3,
+               "h2d_bytes_per_step": P * m, "d2h_bytes_per_step": P * P * m, "steps": e2e_steps,
+               "checked": ok}
+        hplan.destroy()
+        del hs, hr
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        launches_per_step = (k1 - k0) / args.steps
+        avg_ms = float(np.mean(per_ms))
+        achieved = algorithmic_bytes(P, m) / (avg_ms * 1e-3) / 1e9
+        key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[plan.exec_mode]}:{sp.COPY_NAMES[plan.copy_path]}"
+        roofline = {
+            "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": peak_src,
+            "kernel": f"{sp.EXEC_NAMES[plan.exec_mode]} executor, {sp.COPY_NAMES[plan.copy_path]} engine "
+                      f"({launches_per_step:g} launch(es) per collective)",
+            "algorithmic_bytes_per_launch": algorithmic_bytes(P, m) / max(launches_per_step, 1),
+        }
+        cpu = None if args.no_cpu else cpu_baseline_leg(P, m, seed)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": f"{args.algo} allgather, P={P} virtual ranks, m={m} B blocks "
+                                   f"({P * P * m / 2**30:.3g} GiB of receive buffers per GPU)",
+                       "P": P, "block_bytes": m, "algo": args.algo,
+                       "exec": sp.EXEC_NAMES[plan.exec_mode], "copy": sp.COPY_NAMES[plan.copy_path],
+                       "l2": "inputs larger than L2 (no flush needed)" if P * P * m > (256 << 20)
+                             else "working set may sit in L2 (latency regime, reported as such)",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "us_per_collective": {"min": min(per_ms) * 1e3, "avg": avg_ms * 1e3, "max": max(per_ms) * 1e3},
+            "pct_of_hbm_peak": 100.0 * value / world / peak,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(k1 - k0), "graph_launches": int(g1 - g0),
+            "clocks": clocks, "checked": bool(checked),
+        }
+        print(json.dumps(line), flush=True)
+    plan.destroy()
+    if use_dist:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--P", type=int, default=P_DEFAULT)
+    ap.add_argument("--m", type=int, default=M_DEFAULT)
+    ap.add_argument("--algo", choices=["sparbit", "ring", "rd", "bruck"], default="sparbit")
+    ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "cluster"], default="auto")
+    ap.add_argument("--copy", choices=["auto", "vector", "bulk"], default="auto")
+    ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

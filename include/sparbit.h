@@ -1,0 +1,228 @@
+/*
+ * sparbit.h - C ABI of the B200 step executor for the Sparbit allgather (Stripe Parallel
+ * Binomial Trees) and its comparators.
+ *
+ * The P ranks of a communicator are P virtual ranks resident in one GPU's memory.  Rank r owns
+ * one send block of m bytes and one receive buffer of P slots of m bytes.  A collective runs the
+ * chosen algorithm's exchange schedule; each step of the schedule is one data-parallel copy pass
+ * over all ranks, a forwarded block being read from the SENDING rank's receive buffer and written
+ * into its final slot of the RECEIVING rank's receive buffer, as the algorithm prescribes.  The
+ * result is the one MPI_Allgather defines (paper, Section II): slot j of every receive buffer
+ * holds the block sent by rank j.
+ *
+ * Notation: m is the bytes of ONE block (sendcount = recvcount = m).  The paper writes m for the
+ * total a process ends up with and m/p for a block.
+ *
+ * Layout (all device pointers, caller-owned, contiguous):
+ *   sendbuf   P * m bytes        rank r's block at byte offset r * m
+ *   recvbuf   P * P * m bytes    rank r's buffer at r * P * m, slot b at + b * m
+ *   workspace P * P * m bytes    Bruck only (its rotated working buffers), same layout
+ *
+ * Phases of a collective, in execution order:
+ *   -1          local copy of the own block, sendbuf[r] -> recvbuf[r][r] (Bruck: -> workspace[r][0]).
+ *               Algorithm 1 sends displacement `rank` at j = 0 as if it were in place already;
+ *               Section II's semantics need this copy.  MPI_IN_PLACE is not supported.
+ *   0 .. K-1    the algorithm's communication steps (Sparbit: Algorithm 1's loop, K = ceil(log2 P)).
+ *   K           Bruck only: the final rotation workspace[r][i] -> recvbuf[r][(r + i) mod P]
+ *               (the "memory shifts" of Section II-B).
+ * Every phase ends with the equivalent of Algorithm 1's MPI_Waitall: no copy of the next phase
+ * starts before all copies of this one are visible.
+ *
+ * Conventions: every function is extern "C", never throws, never aborts the process.  Functions
+ * returning int return SPARBIT_OK (0) or a positive SPARBIT_ERR_* code.  Nothing here
+ * synchronises the device unless its comment says so.  All argument errors are found on the
+ * host before anything is launched.  A plan may be used by one host thread and on one stream at
+ * a time.
+ */
+#ifndef SPARBIT_H
+#define SPARBIT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    SPARBIT_OK = 0,
+    SPARBIT_ERR_ARG = 1,         /* null handle/buffer, P < 1, phase range or enum out of range */
+    SPARBIT_ERR_OVERFLOW = 2,    /* P*P*m (or an internal work count) is not representable */
+    SPARBIT_ERR_ALIAS = 3,       /* send / receive / workspace byte ranges overlap */
+    SPARBIT_ERR_UNSUPPORTED = 4, /* recursive doubling with P not a power of two; bad mode combo */
+    SPARBIT_ERR_WORKSPACE = 5,   /* Bruck without a workspace, or one that is too small */
+    SPARBIT_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sparbit_last_cuda_error() */
+    SPARBIT_ERR_TIMEOUT = 7,     /* the device-side grid barrier gave up waiting */
+    SPARBIT_ERR_NOMEM = 8        /* host allocation failed */
+};
+
+/* Algorithms (paper, Section II-A and Section III).  Only Sparbit is the product's hot path; the
+ * other three run on the same executor as comparators. */
+enum {
+    SPARBIT_ALGO_SPARBIT = 0,
+    SPARBIT_ALGO_RING = 1,
+    SPARBIT_ALGO_RECURSIVE_DOUBLING = 2, /* powers of two only, as the paper states */
+    SPARBIT_ALGO_BRUCK = 3
+};
+
+/* How the phases are put on the GPU. */
+enum {
+    SPARBIT_EXEC_AUTO = 0,       /* chosen from P and m */
+    SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per phase */
+    SPARBIT_EXEC_GRAPH = 2,      /* one kernel per phase, chained in a cached CUDA graph */
+    SPARBIT_EXEC_STREAM = 3,     /* one kernel per phase, launched one by one on the stream */
+    SPARBIT_EXEC_CLUSTER = 4     /* one thread-block cluster, hardware cluster barrier per phase;
+                                    for collectives small enough to be latency-bound */
+};
+
+/* Which copy engine a phase uses. */
+enum {
+    SPARBIT_COPY_AUTO = 0,   /* chosen from m and the alignment of the buffers */
+    SPARBIT_COPY_VECTOR = 1, /* warp-cooperative ld/st.global, 16/8/4/2/1-byte vectors */
+    SPARBIT_COPY_BULK = 2    /* cp.async.bulk global->shared->global ring (needs 16-byte
+                                alignment of buffers and m); falls back to VECTOR otherwise */
+};
+
+/* Address spaces a message endpoint can live in. */
+enum { SPARBIT_SPACE_SEND = 0, SPARBIT_SPACE_RECV = 1, SPARBIT_SPACE_WORKSPACE = 2 };
+
+typedef struct sparbit_plan_s sparbit_plan_t; /* opaque; owned by the library */
+
+/* One single-block message of a phase, as Algorithm 1 issues them (one MPI_Isend/MPI_Irecv pair
+ * per block).  Slots are displacements in blocks inside the rank's buffer of that space. */
+typedef struct {
+    int32_t phase;
+    int32_t src_rank;
+    int32_t dst_rank;
+    int32_t src_space;
+    int32_t src_slot;
+    int32_t dst_space;
+    int32_t dst_slot;
+} sparbit_msg;
+
+/*
+ * sparbit_plan - the short form: a Sparbit plan with automatic executor choice for P ranks and
+ * blocks of block_bytes.  Returns NULL on any error (use sparbit_plan_create for the code).
+ * Host-only: runs Algorithm 1's set-up (lines 1-5) and derives the per-step descriptors; makes
+ * no CUDA call.  Device resources (a few hundred bytes plus the descriptor table) are allocated
+ * by the first sparbit_allgather on the plan, which should therefore not be inside a stream
+ * capture.
+ */
+sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
+
+/*
+ * sparbit_plan_create - full form.  algo: SPARBIT_ALGO_*; exec: SPARBIT_EXEC_*.  On success
+ * *out receives a plan the caller must release with sparbit_plan_destroy.  block_bytes may be 0
+ * (the collective is then a no-op, as MPI allows count 0).  Errors: ERR_ARG (P < 1, null out,
+ * unknown enum), ERR_OVERFLOW (P*P*block_bytes does not fit in 63 bits, or P > 2^24),
+ * ERR_UNSUPPORTED (recursive doubling with P not a power of two: Section II-A defines it for
+ * powers of two only), ERR_NOMEM.  Host-only.
+ */
+int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out);
+
+/* Releases the plan and everything it owns (device table, graph).  Synchronises the device if
+ * the plan ever launched work.  NULL is allowed. */
+int sparbit_plan_destroy(sparbit_plan_t* plan);
+
+/*
+ * sparbit_allgather - the collective (paper, Section II; Sparbit: Algorithm 1).  Mirrors
+ * MPI_Allgather(sendbuf, m, MPI_BYTE, recvbuf, m, MPI_BYTE, comm) for a communicator of P ranks.
+ *   sendbuf  device, P*m bytes, read only          recvbuf  device, P*P*m bytes, fully overwritten
+ *   stream   a cudaStream_t passed as void* (NULL = the legacy default stream)
+ * Asynchronous: work is enqueued on `stream` and the call returns.  Any alignment of the
+ * pointers and any m >= 1 give the right answer; 16-byte aligned buffers with m % 16 == 0 get
+ * the fast paths.  Errors (nothing is launched): ERR_ARG (null plan; null buffer with P*m > 0),
+ * ERR_ALIAS (ranges overlap), ERR_WORKSPACE (Bruck without workspace), ERR_CUDA.
+ * A device-side barrier time-out is reported later by sparbit_plan_status.
+ */
+int sparbit_allgather(sparbit_plan_t* plan, const void* sendbuf, void* recvbuf, void* stream);
+
+/*
+ * sparbit_allgather_steps - run only phases first..last (inclusive; -1 <= first <= last <=
+ * sparbit_plan_last_phase).  For step-by-step comparison with a reference; same contract as
+ * sparbit_allgather otherwise.  Phases skipped are the caller's business: the buffers must
+ * already hold what the earlier phases would have produced.
+ */
+int sparbit_allgather_steps(sparbit_plan_t* plan, const void* sendbuf, void* recvbuf, void* stream,
+                            int first, int last);
+
+/*
+ * sparbit_allgather_host - the same collective for HOST buffers (host_send P*m bytes, host_recv
+ * P*P*m bytes; pinned memory makes the copies faster but is not required).  Copies the send
+ * blocks to device staging owned by the plan (allocated on first use), runs the collective,
+ * copies all P receive buffers back, and SYNCHRONISES before returning.  Errors as for
+ * sparbit_allgather, plus ERR_TIMEOUT if the device barrier gave up.
+ */
+int sparbit_allgather_host(sparbit_plan_t* plan, const void* host_send, void* host_recv);
+
+/* ---- introspection (host-only, no CUDA call) ------------------------------------------------ */
+
+/* K, the number of communication steps: Sparbit and Bruck ceil(log2 P), recursive doubling
+ * log2 P, ring P-1 (the latency terms of the cost formulae of Sections II-A and III-B). */
+int sparbit_plan_num_steps(const sparbit_plan_t* plan);
+
+/* Index of the last phase: K-1, or K for Bruck (rotation).  -1 when P = 1 and not Bruck. */
+int sparbit_plan_last_phase(const sparbit_plan_t* plan);
+
+/*
+ * Step variables of one communication step (0 <= step < K).  distance: ranks between sender and
+ * receiver (Algorithm 1's d).  blocks_per_rank: messages each rank sends in the step
+ * (Algorithm 1's data - ignore).  ignore: 1 if the step withholds a block (Sparbit only, else 0).
+ * Any out pointer may be NULL.
+ */
+int sparbit_plan_step_info(const sparbit_plan_t* plan, int step, int* distance, int* blocks_per_rank,
+                           int* ignore);
+
+/*
+ * Expands the compact descriptor of one phase (-1 .. last phase) into explicit single-block
+ * messages, using the same index function the kernels use.  Writes min(cap, *n) entries to out
+ * (out may be NULL when cap is 0) and always stores the full count in *n.  Order inside a phase
+ * is unspecified.
+ */
+int sparbit_plan_messages(const sparbit_plan_t* plan, int phase, sparbit_msg* out, size_t cap, size_t* n);
+
+/* Bytes of workspace the plan needs: 0, or P*P*m for Bruck. */
+size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* plan);
+
+/* Gives the plan its workspace (device memory; the caller keeps ownership and must keep it alive
+ * while the plan is used).  ERR_WORKSPACE if bytes is too small. */
+int sparbit_plan_set_workspace(sparbit_plan_t* plan, void* dev, size_t bytes);
+
+/* Forces the copy engine (SPARBIT_COPY_*).  BULK silently runs as VECTOR for a call whose
+ * buffers or m are not 16-byte aligned. */
+int sparbit_plan_set_copy_path(sparbit_plan_t* plan, int copy_path);
+
+/* What the plan resolved to: executor (SPARBIT_EXEC_*, never AUTO) and the copy engine the last
+ * launch used (SPARBIT_COPY_*; AUTO before the first launch). */
+int sparbit_plan_exec_mode(const sparbit_plan_t* plan);
+int sparbit_plan_copy_path(const sparbit_plan_t* plan);
+
+/* Kernels (and graph launches) the library has enqueued for this plan so far. */
+int sparbit_plan_launch_counts(const sparbit_plan_t* plan, uint64_t* kernel_launches, uint64_t* graph_launches);
+
+/*
+ * Synchronises the plan's last stream and reports the device status word: SPARBIT_OK, or
+ * SPARBIT_ERR_TIMEOUT if a grid barrier of the persistent executor gave up (all CTAs then left
+ * the kernel early and the receive buffers are incomplete).  Clears the condition so the plan
+ * can be used again.  *device_status (may be NULL) receives the raw word.
+ */
+int sparbit_plan_status(sparbit_plan_t* plan, int* device_status);
+
+/*
+ * Test hook for the bounded wait of the grid barrier: the next persistent launches expect
+ * `extra_arrivals` more arrivals than there are CTAs and give up after `timeout_ns`
+ * nanoseconds (0 restores the defaults: no extra arrivals, 2 s).  With extra_arrivals > 0 the
+ * barrier can never complete, so the kernel must return with the time-out status instead of
+ * hanging.
+ */
+int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint64_t timeout_ns);
+
+const char* sparbit_strerror(int code);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* sparbit_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARBIT_H */

@@ -120,6 +120,26 @@ class Plan:
         if rc:
             raise OracleError(lib.oracle_last_error().decode())
 
+    def trace(self, rank: int, slot: int):
+        """Follow the messages that fill receive slot `slot` of `rank` back to a send buffer.
+
+        Returns the list of messages on the way, first hop first.  The first hop reads the send
+        block of the rank whose data ends up in the slot, so a sampled output of a run too large
+        to simulate in full is `send[trace(...)[0]["src_rank"]]`.
+        """
+        if not hasattr(self, "_by_dst"):
+            m = self.messages
+            key = (m["dst_space"].astype(np.int64) * self.P + m["dst_rank"]) * self.P + m["dst_slot"]
+            self._by_dst = dict(zip(key.tolist(), range(len(m))))
+        path = []
+        space, r, s = SPACE_RECV, int(rank), int(slot)
+        while space != SPACE_SEND:
+            k = self._by_dst[(space * self.P + r) * self.P + s]
+            msg = self.messages[k]
+            path.append(msg)
+            space, r, s = int(msg["src_space"]), int(msg["src_rank"]), int(msg["src_slot"])
+        return path[::-1]
+
     def close(self) -> None:
         if getattr(self, "_h", None):
             _load().oracle_plan_destroy(self._h)

@@ -1,0 +1,202 @@
+"""ctypes binding of libsparbit_b200.so: argument marshalling only, same names as the C ABI.
+
+Every step of a collective runs in the library's CUDA kernels.  There is no fallback: if the
+shared library is missing or cannot be loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+
+_LIB_PATH = Path(__file__).resolve().parent / "libsparbit_b200.so"
+
+OK = 0
+ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = range(1, 9)
+ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK = range(4)
+EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_CLUSTER = range(5)
+COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
+SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
+
+ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
+              ALGO_BRUCK: "bruck"}
+EXEC_NAMES = {EXEC_AUTO: "auto", EXEC_PERSISTENT: "persistent", EXEC_GRAPH: "graph", EXEC_STREAM: "stream",
+              EXEC_CLUSTER: "cluster"}
+COPY_NAMES = {COPY_AUTO: "auto", COPY_VECTOR: "vector", COPY_BULK: "bulk"}
+
+MSG_DTYPE = np.dtype([("phase", "<i4"), ("src_rank", "<i4"), ("dst_rank", "<i4"), ("src_space", "<i4"),
+                      ("src_slot", "<i4"), ("dst_space", "<i4"), ("dst_slot", "<i4")])
+
+#: every symbol include/sparbit.h declares, with (restype, argtypes)
+_vp, _sz, _i, _u64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64
+_pi = ctypes.POINTER(ctypes.c_int)
+SYMBOLS = {
+    "sparbit_plan": (_vp, [_i, _sz]),
+    "sparbit_plan_create": (_i, [_i, _sz, _i, _i, ctypes.POINTER(_vp)]),
+    "sparbit_plan_destroy": (_i, [_vp]),
+    "sparbit_allgather": (_i, [_vp, _vp, _vp, _vp]),
+    "sparbit_allgather_steps": (_i, [_vp, _vp, _vp, _vp, _i, _i]),
+    "sparbit_allgather_host": (_i, [_vp, _vp, _vp]),
+    "sparbit_plan_num_steps": (_i, [_vp]),
+    "sparbit_plan_last_phase": (_i, [_vp]),
+    "sparbit_plan_step_info": (_i, [_vp, _i, _pi, _pi, _pi]),
+    "sparbit_plan_messages": (_i, [_vp, _i, _vp, _sz, ctypes.POINTER(_sz)]),
+    "sparbit_plan_workspace_bytes": (_sz, [_vp]),
+    "sparbit_plan_set_workspace": (_i, [_vp, _vp, _sz]),
+    "sparbit_plan_set_copy_path": (_i, [_vp, _i]),
+    "sparbit_plan_exec_mode": (_i, [_vp]),
+    "sparbit_plan_copy_path": (_i, [_vp]),
+    "sparbit_plan_launch_counts": (_i, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
+    "sparbit_plan_status": (_i, [_vp, _pi]),
+    "sparbit_plan_set_barrier_test": (_i, [_vp, _i, _u64]),
+    "sparbit_strerror": (ctypes.c_char_p, [_i]),
+    "sparbit_last_cuda_error": (ctypes.c_char_p, []),
+}
+
+if not _LIB_PATH.exists():
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2109_08751_b200.build` "
+        "(there is no fallback path)")
+lib = ctypes.CDLL(str(_LIB_PATH))
+for _name, (_res, _args) in SYMBOLS.items():
+    _fn = getattr(lib, _name)  # AttributeError here means the library does not match the header
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class SparbitError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib.sparbit_strerror(code).decode()
+        if code == ERR_CUDA:
+            msg += ": " + lib.sparbit_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} (code {code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise SparbitError(code, where)
+
+
+def _ptr(x) -> int | None:
+    """Device or host address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()  # torch.Tensor
+
+
+def _stream_handle(stream) -> int | None:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream  # torch.cuda.Stream
+
+
+class Plan:
+    """A plan of the C library (sparbit_plan_create ... sparbit_plan_destroy)."""
+
+    def __init__(self, P: int, block_bytes: int, algo: int = ALGO_SPARBIT, exec_mode: int = EXEC_AUTO):
+        h = _vp()
+        _check(lib.sparbit_plan_create(P, block_bytes, algo, exec_mode, ctypes.byref(h)), "sparbit_plan_create")
+        self._h = h
+        self.P, self.block_bytes, self.algo = P, block_bytes, algo
+        self._workspace = None
+
+    # -- the collective
+    def allgather(self, sendbuf, recvbuf, stream=None) -> None:
+        _check(lib.sparbit_allgather(self._h, _ptr(sendbuf), _ptr(recvbuf), _stream_handle(stream)),
+               "sparbit_allgather")
+
+    def allgather_steps(self, sendbuf, recvbuf, first: int, last: int, stream=None) -> None:
+        _check(lib.sparbit_allgather_steps(self._h, _ptr(sendbuf), _ptr(recvbuf), _stream_handle(stream),
+                                           first, last), "sparbit_allgather_steps")
+
+    def allgather_host(self, host_send, host_recv) -> None:
+        _check(lib.sparbit_allgather_host(self._h, _ptr(host_send), _ptr(host_recv)), "sparbit_allgather_host")
+
+    # -- introspection
+    @property
+    def num_steps(self) -> int:
+        return lib.sparbit_plan_num_steps(self._h)
+
+    @property
+    def last_phase(self) -> int:
+        return lib.sparbit_plan_last_phase(self._h)
+
+    def step_info(self, step: int):
+        d, n, ig = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        _check(lib.sparbit_plan_step_info(self._h, step, ctypes.byref(d), ctypes.byref(n), ctypes.byref(ig)),
+               "sparbit_plan_step_info")
+        return d.value, n.value, ig.value
+
+    def messages(self, phase: int) -> np.ndarray:
+        n = _sz()
+        _check(lib.sparbit_plan_messages(self._h, phase, None, 0, ctypes.byref(n)), "sparbit_plan_messages")
+        out = np.zeros(n.value, dtype=MSG_DTYPE)
+        if n.value:
+            _check(lib.sparbit_plan_messages(self._h, phase, out.ctypes.data, n.value, ctypes.byref(n)),
+                   "sparbit_plan_messages")
+        return out
+
+    @property
+    def workspace_bytes(self) -> int:
+        return lib.sparbit_plan_workspace_bytes(self._h)
+
+    def set_workspace(self, dev, nbytes: int) -> None:
+        _check(lib.sparbit_plan_set_workspace(self._h, _ptr(dev), nbytes), "sparbit_plan_set_workspace")
+        self._workspace = dev  # keep the owner alive
+
+    def set_copy_path(self, path: int) -> None:
+        _check(lib.sparbit_plan_set_copy_path(self._h, path), "sparbit_plan_set_copy_path")
+
+    @property
+    def exec_mode(self) -> int:
+        return lib.sparbit_plan_exec_mode(self._h)
+
+    @property
+    def copy_path(self) -> int:
+        return lib.sparbit_plan_copy_path(self._h)
+
+    def launch_counts(self):
+        k, g = _u64(), _u64()
+        _check(lib.sparbit_plan_launch_counts(self._h, ctypes.byref(k), ctypes.byref(g)),
+               "sparbit_plan_launch_counts")
+        return k.value, g.value
+
+    def status(self) -> int:
+        """Synchronises; returns OK or ERR_TIMEOUT (raises on CUDA errors)."""
+        raw = ctypes.c_int()
+        code = lib.sparbit_plan_status(self._h, ctypes.byref(raw))
+        if code not in (OK, ERR_TIMEOUT):
+            raise SparbitError(code, "sparbit_plan_status")
+        return code
+
+    def set_barrier_test(self, extra_arrivals: int, timeout_ns: int) -> None:
+        _check(lib.sparbit_plan_set_barrier_test(self._h, extra_arrivals, timeout_ns),
+               "sparbit_plan_set_barrier_test")
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            h, self._h = self._h, None
+            _check(lib.sparbit_plan_destroy(h), "sparbit_plan_destroy")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def sparbit_plan(P: int, block_bytes: int) -> Plan:
+    """The short form of the C ABI: a Sparbit plan with automatic executor choice."""
+    return Plan(P, block_bytes, ALGO_SPARBIT, EXEC_AUTO)
+
+
+def sparbit_allgather(plan: Plan, sendbuf, recvbuf, stream=None) -> None:
+    plan.allgather(sendbuf, recvbuf, stream)

@@ -1,0 +1,671 @@
+// C ABI of the step executor: plans, argument checks, executor selection and launches.
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/sparbit.h"
+#include "kernels.cuh"
+#include "schedule.h"
+
+using namespace spb;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+    return SPARBIT_ERR_CUDA;
+}
+#define CU(call)                                         \
+    do {                                                 \
+        cudaError_t e_ = (call);                         \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s
+constexpr int kVecBlock = 512;
+constexpr int kClusterBlock = 512;
+
+struct GraphKey {
+    const void* send = nullptr;
+    void* recv = nullptr;
+    void* work = nullptr;
+    int first = 0, last = -2;
+    int path = 0, vec = 0;
+    bool operator==(const GraphKey& o) const {
+        return send == o.send && recv == o.recv && work == o.work && first == o.first && last == o.last &&
+               path == o.path && vec == o.vec;
+    }
+};
+
+}  // namespace
+
+struct sparbit_plan_s {
+    Schedule sched;
+    int exec_req = SPARBIT_EXEC_AUTO;
+    int copy_req = SPARBIT_COPY_AUTO;
+    int copy_last = SPARBIT_COPY_AUTO;
+    void* work = nullptr;
+    size_t work_bytes = 0;
+
+    // device side, created by the first launch
+    bool dev_ready = false;
+    int device = -1;
+    int sm_count = 0;
+    int coop = 0;
+    int max_smem_optin = 0;
+    int cluster_ok = 0;
+    PhaseDesc* d_descs = nullptr;
+    unsigned* d_ctl = nullptr;  // [0] barrier counter, [1] status word
+    unsigned bar_base = 0;
+    int extra_arrivals = 0;
+    unsigned long long timeout_ns = kDefaultTimeoutNs;
+
+    // bulk engine geometry
+    uint32_t bulk_warps = 2;
+    uint32_t bulk_stage_bytes = 14336;
+
+    // cached graph
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t gexec = nullptr;
+    GraphKey gkey;
+
+    // host-buffer entry point
+    void* stage_send = nullptr;
+    void* stage_recv = nullptr;
+    void* stage_work = nullptr;
+
+    cudaStream_t last_stream = nullptr;
+    bool launched = false;
+    uint64_t kernel_launches = 0, graph_launches = 0;
+};
+
+namespace {
+
+int map_sched_err(int e) {
+    switch (e) {
+        case SCHED_OK: return SPARBIT_OK;
+        case SCHED_ARG: return SPARBIT_ERR_ARG;
+        case SCHED_OVERFLOW: return SPARBIT_ERR_OVERFLOW;
+        case SCHED_UNSUPPORTED: return SPARBIT_ERR_UNSUPPORTED;
+        default: return SPARBIT_ERR_ARG;
+    }
+}
+
+size_t bulk_smem_bytes(const sparbit_plan_s* p) {
+    return (size_t)p->bulk_warps * kBulkStages * (p->bulk_stage_bytes + 8 + 16);
+}
+
+int ensure_device(sparbit_plan_s* p) {
+    if (p->dev_ready) return SPARBIT_OK;
+    CU(cudaGetDevice(&p->device));
+    CU(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
+    CU(cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device));
+    CU(cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device));
+    int cc_major = 0;
+    CU(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, p->device));
+    p->cluster_ok = cc_major >= 9;
+    // shrink the bulk ring if this device offers less shared memory than planned
+    while (bulk_smem_bytes(p) > (size_t)p->max_smem_optin && p->bulk_stage_bytes > 1024) p->bulk_stage_bytes -= 1024;
+    const size_t n = p->sched.phases.size();
+    CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
+    CU(cudaMemcpy(p->d_descs, p->sched.phases.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
+    CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
+    CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
+    CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            (int)bulk_smem_bytes(p)));
+    CU(cudaFuncSetAttribute(persistent_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            (int)bulk_smem_bytes(p)));
+    p->dev_ready = true;
+    return SPARBIT_OK;
+}
+
+bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+    return x < y + nb && y < x + na;
+}
+
+// largest power-of-two vector width (<= 16) that divides every address and m
+int pick_vector_bytes(const sparbit_plan_s* p, const void* send, const void* recv) {
+    uintptr_t bits = (uintptr_t)send | (uintptr_t)recv | (uintptr_t)p->sched.m;
+    if (p->sched.algo == ALGO_BRUCK) bits |= (uintptr_t)p->work;
+    int v = 16;
+    while (v > 1 && (bits & (uintptr_t)(v - 1))) v >>= 1;
+    return v;
+}
+
+// warp tasks of one phase on the vector engine (mirrors vec_phase)
+uint64_t vec_tasks(const PhaseDesc& d, uint32_t P, int vbytes) {
+    const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
+    const uint64_t n_copies = (uint64_t)P * d.copies;
+    if (vpc >= 32) {
+        const uint64_t span = 32ull * kVecUnroll;
+        return n_copies * ((vpc + span - 1) / span);
+    }
+    if (vpc == 0) return 0;
+    const uint64_t per_task = (32 / vpc) * kVecUnroll;
+    return (n_copies + per_task - 1) / per_task;
+}
+
+uint64_t bulk_tasks(const PhaseDesc& d, uint32_t P, uint32_t stage_bytes) {
+    return (uint64_t)P * d.copies * ((d.copy_bytes + stage_bytes - 1) / stage_bytes);
+}
+
+template <typename V>
+const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V>; }
+template <typename V>
+const void* persistent_vec_fn() { return (const void*)persistent_vec_kernel<V>; }
+
+const void* pick_phase_vec(int vbytes) {
+    switch (vbytes) {
+        case 16: return phase_vec_fn<uint4>();
+        case 8: return phase_vec_fn<uint2>();
+        case 4: return phase_vec_fn<unsigned>();
+        case 2: return phase_vec_fn<unsigned short>();
+        default: return phase_vec_fn<unsigned char>();
+    }
+}
+const void* pick_persistent_vec(int vbytes) {
+    switch (vbytes) {
+        case 16: return persistent_vec_fn<uint4>();
+        case 8: return persistent_vec_fn<uint2>();
+        case 4: return persistent_vec_fn<unsigned>();
+        case 2: return persistent_vec_fn<unsigned short>();
+        default: return persistent_vec_fn<unsigned char>();
+    }
+}
+template <typename V>
+const void* cluster_vec_fn() { return (const void*)cluster_vec_kernel<V>; }
+const void* pick_cluster_vec(int vbytes) {
+    switch (vbytes) {
+        case 16: return cluster_vec_fn<uint4>();
+        case 8: return cluster_vec_fn<uint2>();
+        case 4: return cluster_vec_fn<unsigned>();
+        case 2: return cluster_vec_fn<unsigned short>();
+        default: return cluster_vec_fn<unsigned char>();
+    }
+}
+
+// executor for SPARBIT_EXEC_AUTO: collectives that move little are latency-bound and run inside
+// one thread-block cluster; everything else runs in the persistent cooperative kernel
+int auto_exec(const Schedule& s, bool coop, bool cluster_ok) {
+    const uint64_t P = s.P;
+    const unsigned __int128 moved = (unsigned __int128)2 * P * (P - 1) * s.m;
+    if (cluster_ok && moved <= (8u << 20) && s.algo != ALGO_RING) return SPARBIT_EXEC_CLUSTER;
+    return coop ? SPARBIT_EXEC_PERSISTENT : SPARBIT_EXEC_GRAPH;
+}
+
+struct Resolved {
+    int exec;    // SPARBIT_EXEC_* (never AUTO)
+    int copy;    // SPARBIT_COPY_VECTOR or _BULK
+    int vbytes;  // vector width for the vector engine
+};
+
+Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv) {
+    Resolved r;
+    r.vbytes = pick_vector_bytes(p, send, recv);
+    const uint64_t m = p->sched.m;
+    const bool bulk_possible = r.vbytes == 16;
+    int copy = p->copy_req;
+    if (copy == SPARBIT_COPY_AUTO) copy = (bulk_possible && m >= 4096) ? SPARBIT_COPY_BULK : SPARBIT_COPY_VECTOR;
+    if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
+    r.copy = copy;
+    int exec = p->exec_req;
+    if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p->sched, p->coop != 0, p->cluster_ok != 0);
+    if (exec == SPARBIT_EXEC_PERSISTENT && !p->coop) exec = SPARBIT_EXEC_GRAPH;
+    if (exec == SPARBIT_EXEC_CLUSTER) {
+        if (!p->cluster_ok) exec = SPARBIT_EXEC_GRAPH;
+        r.copy = SPARBIT_COPY_VECTOR;  // the cluster executor has the vector engine only
+    }
+    r.exec = exec;
+    return r;
+}
+
+Geom make_geom(const sparbit_plan_s* p, const void* send, void* recv) {
+    Geom g;
+    memset(&g, 0, sizeof g);
+    g.P = p->sched.P;
+    g.m = p->sched.m;
+    g.base[SPACE_SEND] = (char*)const_cast<void*>(send);
+    g.base[SPACE_RECV] = (char*)recv;
+    g.base[SPACE_WORK] = (char*)p->work;
+    g.rank_pitch[SPACE_SEND] = g.m;
+    g.rank_pitch[SPACE_RECV] = (uint64_t)g.P * g.m;
+    g.rank_pitch[SPACE_WORK] = (uint64_t)g.P * g.m;
+    return g;
+}
+
+// launch geometry of one phase as its own kernel
+struct PhaseLaunch {
+    const void* fn;
+    dim3 grid, block;
+    size_t smem;
+};
+
+int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d, PhaseLaunch& pl) {
+    const uint32_t P = p->sched.P;
+    if (rs.copy == SPARBIT_COPY_BULK) {
+        const uint64_t tasks = bulk_tasks(d, P, p->bulk_stage_bytes);
+        uint64_t ctas = (tasks + p->bulk_warps - 1) / p->bulk_warps;
+        if (ctas > (uint64_t)p->sm_count) ctas = p->sm_count;
+        if (ctas < 1) ctas = 1;
+        pl.fn = (const void*)phase_bulk_kernel;
+        pl.grid = dim3((unsigned)ctas);
+        pl.block = dim3(p->bulk_warps * 32);
+        pl.smem = bulk_smem_bytes(p);
+    } else {
+        const uint64_t tasks = vec_tasks(d, P, rs.vbytes);
+        if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
+        const uint64_t wpb = kVecBlock / 32;
+        uint64_t ctas = (tasks + wpb - 1) / wpb;
+        const uint64_t cap = (uint64_t)p->sm_count * 4;  // 2048 threads per SM
+        if (ctas > cap) ctas = cap;
+        if (ctas < 1) ctas = 1;
+        pl.fn = pick_phase_vec(rs.vbytes);
+        pl.grid = dim3((unsigned)ctas);
+        pl.block = dim3(kVecBlock);
+        pl.smem = 0;
+    }
+    return SPARBIT_OK;
+}
+
+struct PhaseArgs {
+    Geom g;
+    PhaseDesc d;
+    uint32_t stage_bytes;
+    unsigned* status;
+    unsigned long long timeout_ns;
+    void* ptrs[5];
+    void fill(bool bulk) {
+        ptrs[0] = &g;
+        ptrs[1] = &d;
+        if (bulk) {
+            ptrs[2] = &stage_bytes;
+            ptrs[3] = &status;
+            ptrs[4] = &timeout_ns;
+        }
+    }
+};
+
+int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+    for (int ph = first; ph <= last; ph++) {
+        PhaseArgs a;
+        a.g = g;
+        a.d = p->sched.phase(ph);
+        a.stage_bytes = p->bulk_stage_bytes;
+        a.status = p->d_ctl + 1;
+        a.timeout_ns = p->timeout_ns;
+        a.fill(rs.copy == SPARBIT_COPY_BULK);
+        PhaseLaunch pl;
+        int rc = plan_phase_launch(p, rs, a.d, pl);
+        if (rc) return rc;
+        CU(cudaLaunchKernel(pl.fn, pl.grid, pl.block, a.ptrs, pl.smem, st));
+        p->kernel_launches++;
+    }
+    return SPARBIT_OK;
+}
+
+void drop_graph(sparbit_plan_s* p) {
+    if (p->gexec) cudaGraphExecDestroy(p->gexec);
+    if (p->graph) cudaGraphDestroy(p->graph);
+    p->gexec = nullptr;
+    p->graph = nullptr;
+    p->gkey = GraphKey();
+}
+
+int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+    GraphKey key;
+    key.send = g.base[SPACE_SEND];
+    key.recv = g.base[SPACE_RECV];
+    key.work = g.base[SPACE_WORK];
+    key.first = first;
+    key.last = last;
+    key.path = rs.copy;
+    key.vec = rs.vbytes;
+    if (!p->gexec || !(p->gkey == key)) {
+        // (re)build the chain: one kernel node per phase, each depending on the one before
+        drop_graph(p);
+        CU(cudaGraphCreate(&p->graph, 0));
+        cudaGraphNode_t prev = nullptr;
+        for (int ph = first; ph <= last; ph++) {
+            PhaseArgs a;
+            a.g = g;
+            a.d = p->sched.phase(ph);
+            a.stage_bytes = p->bulk_stage_bytes;
+            a.status = p->d_ctl + 1;
+            a.timeout_ns = p->timeout_ns;
+            a.fill(rs.copy == SPARBIT_COPY_BULK);
+            PhaseLaunch pl;
+            int rc = plan_phase_launch(p, rs, a.d, pl);
+            if (rc) return rc;
+            cudaKernelNodeParams np;
+            memset(&np, 0, sizeof np);
+            np.func = const_cast<void*>(pl.fn);
+            np.gridDim = pl.grid;
+            np.blockDim = pl.block;
+            np.sharedMemBytes = (unsigned)pl.smem;
+            np.kernelParams = a.ptrs;
+            cudaGraphNode_t node;
+            CU(cudaGraphAddKernelNode(&node, p->graph, prev ? &prev : nullptr, prev ? 1 : 0, &np));
+            prev = node;
+        }
+        CU(cudaGraphInstantiate(&p->gexec, p->graph, 0));
+        p->gkey = key;
+    }
+    CU(cudaGraphLaunch(p->gexec, st));
+    p->graph_launches++;
+    p->kernel_launches += (uint64_t)(last - first + 1);
+    return SPARBIT_OK;
+}
+
+int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+    const uint32_t P = p->sched.P;
+    // grid: enough CTAs for the largest phase, at most what is co-resident
+    uint64_t need = 1;
+    const void* fn;
+    dim3 block;
+    size_t smem = 0;
+    int per_sm = 0;
+    if (rs.copy == SPARBIT_COPY_BULK) {
+        fn = (const void*)persistent_bulk_kernel;
+        block = dim3(p->bulk_warps * 32);
+        smem = bulk_smem_bytes(p);
+        for (int ph = first; ph <= last; ph++) {
+            uint64_t t = (bulk_tasks(p->sched.phase(ph), P, p->bulk_stage_bytes) + p->bulk_warps - 1) / p->bulk_warps;
+            if (t > need) need = t;
+        }
+    } else {
+        fn = pick_persistent_vec(rs.vbytes);
+        block = dim3(kVecBlock);
+        for (int ph = first; ph <= last; ph++) {
+            const uint64_t tasks = vec_tasks(p->sched.phase(ph), P, rs.vbytes);
+            if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
+            uint64_t t = (tasks + kVecBlock / 32 - 1) / (kVecBlock / 32);
+            if (t > need) need = t;
+        }
+    }
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, (int)block.x, smem));
+    if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "persistent kernel does not fit on an SM");
+    uint64_t grid = (uint64_t)per_sm * p->sm_count;
+    if (grid > need) grid = need;
+    BarrierCtl ctl;
+    ctl.counter = p->d_ctl;
+    ctl.status = p->d_ctl + 1;
+    ctl.base = p->bar_base;
+    ctl.expected = (unsigned)grid + (unsigned)p->extra_arrivals;
+    ctl.timeout_ns = p->timeout_ns;
+    int first_idx = first + 1, last_idx = last + 1;  // descriptor table index = phase + 1
+    Geom gg = g;
+    const PhaseDesc* descs = p->d_descs;
+    uint32_t stage = p->bulk_stage_bytes;
+    void* args_vec[] = {&gg, &descs, &first_idx, &last_idx, &ctl};
+    void* args_bulk[] = {&gg, &descs, &first_idx, &last_idx, &stage, &ctl};
+    CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), block,
+                                   rs.copy == SPARBIT_COPY_BULK ? args_bulk : args_vec, smem, st));
+    p->bar_base += (unsigned)(last - first) * ctl.expected;  // one barrier between consecutive phases
+    p->kernel_launches++;
+    return SPARBIT_OK;
+}
+
+int launch_cluster(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+    const uint32_t P = p->sched.P;
+    uint64_t need = 1;
+    for (int ph = first; ph <= last; ph++) {
+        const uint64_t tasks = vec_tasks(p->sched.phase(ph), P, rs.vbytes);
+        if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
+        uint64_t t = (tasks + kClusterBlock / 32 - 1) / (kClusterBlock / 32);
+        if (t > need) need = t;
+    }
+    unsigned ctas = 8;  // the portable cluster size
+    while (ctas > 1 && ctas / 2 >= need) ctas /= 2;
+    const void* fn = pick_cluster_vec(rs.vbytes);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = dim3(kClusterBlock);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ctas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int first_idx = first + 1, last_idx = last + 1;
+    Geom gg = g;
+    const PhaseDesc* descs = p->d_descs;
+    void* args[] = {&gg, &descs, &first_idx, &last_idx};
+    CU(cudaLaunchKernelExC(&cfg, fn, args));
+    p->kernel_launches++;
+    return SPARBIT_OK;
+}
+
+int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, int first, int last) {
+    if (!p) return SPARBIT_ERR_ARG;
+    const Schedule& s = p->sched;
+    if (first < -1 || last > s.last_phase() || first > last) return SPARBIT_ERR_ARG;
+    const size_t send_bytes = (size_t)s.P * s.m;
+    const size_t recv_bytes = (size_t)s.P * s.P * s.m;
+    if (send_bytes == 0) return SPARBIT_OK;  // count 0: nothing to do
+    if (!send || !recv) return SPARBIT_ERR_ARG;
+    if (s.algo == ALGO_BRUCK && (!p->work || p->work_bytes < recv_bytes)) return SPARBIT_ERR_WORKSPACE;
+    if (ranges_overlap(send, send_bytes, recv, recv_bytes)) return SPARBIT_ERR_ALIAS;
+    if (s.algo == ALGO_BRUCK &&
+        (ranges_overlap(send, send_bytes, p->work, recv_bytes) || ranges_overlap(recv, recv_bytes, p->work, recv_bytes)))
+        return SPARBIT_ERR_ALIAS;
+    int rc = ensure_device(p);
+    if (rc) return rc;
+    const Resolved rs = resolve(p, send, recv);
+    const Geom g = make_geom(p, send, recv);
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (rs.exec) {
+        case SPARBIT_EXEC_PERSISTENT: rc = launch_persistent(p, rs, g, first, last, st); break;
+        case SPARBIT_EXEC_GRAPH: rc = launch_graph(p, rs, g, first, last, st); break;
+        case SPARBIT_EXEC_CLUSTER: rc = launch_cluster(p, rs, g, first, last, st); break;
+        default: rc = launch_stream(p, rs, g, first, last, st); break;
+    }
+    if (rc == SPARBIT_OK) {
+        p->copy_last = rs.copy;
+        p->last_stream = st;
+        p->launched = true;
+    }
+    return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out) {
+    if (!out) return SPARBIT_ERR_ARG;
+    *out = nullptr;
+    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_ARG;
+    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_CLUSTER) return SPARBIT_ERR_ARG;
+    sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
+    if (!p) return SPARBIT_ERR_NOMEM;
+    int rc;
+    try {
+        rc = map_sched_err(build_schedule(algo, P, (uint64_t)block_bytes, p->sched));
+    } catch (const std::bad_alloc&) {
+        rc = SPARBIT_ERR_NOMEM;
+    }
+    if (rc) {
+        delete p;
+        return rc;
+    }
+    p->exec_req = exec;
+    *out = p;
+    return SPARBIT_OK;
+}
+
+sparbit_plan_t* sparbit_plan(int P, size_t block_bytes) {
+    sparbit_plan_t* p = nullptr;
+    if (sparbit_plan_create(P, block_bytes, SPARBIT_ALGO_SPARBIT, SPARBIT_EXEC_AUTO, &p) != SPARBIT_OK) return nullptr;
+    return p;
+}
+
+int sparbit_plan_destroy(sparbit_plan_t* p) {
+    if (!p) return SPARBIT_OK;
+    int rc = SPARBIT_OK;
+    if (p->dev_ready) {
+        if (p->launched && cudaDeviceSynchronize() != cudaSuccess) rc = SPARBIT_ERR_CUDA;
+        drop_graph(p);
+        cudaFree(p->d_descs);
+        cudaFree(p->d_ctl);
+        cudaFree(p->stage_send);
+        cudaFree(p->stage_recv);
+        cudaFree(p->stage_work);
+    }
+    delete p;
+    return rc;
+}
+
+int sparbit_allgather(sparbit_plan_t* p, const void* sendbuf, void* recvbuf, void* stream) {
+    if (!p) return SPARBIT_ERR_ARG;
+    return run_phases(p, sendbuf, recvbuf, stream, -1, p->sched.last_phase());
+}
+
+int sparbit_allgather_steps(sparbit_plan_t* p, const void* sendbuf, void* recvbuf, void* stream, int first,
+                            int last) {
+    if (!p) return SPARBIT_ERR_ARG;
+    if (first > last) return SPARBIT_ERR_ARG;
+    return run_phases(p, sendbuf, recvbuf, stream, first, last);
+}
+
+int sparbit_allgather_host(sparbit_plan_t* p, const void* host_send, void* host_recv) {
+    if (!p) return SPARBIT_ERR_ARG;
+    const Schedule& s = p->sched;
+    const size_t send_bytes = (size_t)s.P * s.m;
+    const size_t recv_bytes = (size_t)s.P * s.P * s.m;
+    if (send_bytes == 0) return SPARBIT_OK;
+    if (!host_send || !host_recv) return SPARBIT_ERR_ARG;
+    if (ranges_overlap(host_send, send_bytes, host_recv, recv_bytes)) return SPARBIT_ERR_ALIAS;
+    if (!p->stage_send) CU(cudaMalloc(&p->stage_send, send_bytes));
+    if (!p->stage_recv) CU(cudaMalloc(&p->stage_recv, recv_bytes));
+    if (s.algo == ALGO_BRUCK && !p->work) {
+        if (!p->stage_work) CU(cudaMalloc(&p->stage_work, recv_bytes));
+        p->work = p->stage_work;
+        p->work_bytes = recv_bytes;
+    }
+    cudaStream_t st = nullptr;
+    CU(cudaMemcpyAsync(p->stage_send, host_send, send_bytes, cudaMemcpyHostToDevice, st));
+    int rc = run_phases(p, p->stage_send, p->stage_recv, st, -1, s.last_phase());
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(host_recv, p->stage_recv, recv_bytes, cudaMemcpyDeviceToHost, st));
+    return sparbit_plan_status(p, nullptr);
+}
+
+int sparbit_plan_num_steps(const sparbit_plan_t* p) { return p ? p->sched.K : -1; }
+int sparbit_plan_last_phase(const sparbit_plan_t* p) { return p ? p->sched.last_phase() : -2; }
+
+int sparbit_plan_step_info(const sparbit_plan_t* p, int step, int* distance, int* blocks_per_rank, int* ignore) {
+    if (!p || step < 0 || step >= p->sched.K) return SPARBIT_ERR_ARG;
+    const StepInfo& si = p->sched.steps[(size_t)step];
+    if (distance) *distance = si.distance;
+    if (blocks_per_rank) *blocks_per_rank = si.blocks;
+    if (ignore) *ignore = si.ignore;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_messages(const sparbit_plan_t* p, int phase, sparbit_msg* out, size_t cap, size_t* n) {
+    if (!p || !n || phase < -1 || phase > p->sched.last_phase()) return SPARBIT_ERR_ARG;
+    if (cap > 0 && !out) return SPARBIT_ERR_ARG;
+    *n = (size_t)phase_message_count(p->sched, phase);
+    if (cap == 0) return SPARBIT_OK;
+    static_assert(sizeof(Msg) == sizeof(sparbit_msg), "message layouts must agree");
+    try {
+        std::vector<Msg> v;
+        expand_phase(p->sched, phase, v);
+        const size_t k = v.size() < cap ? v.size() : cap;
+        memcpy(out, v.data(), k * sizeof(Msg));
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    return SPARBIT_OK;
+}
+
+size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* p) {
+    if (!p || p->sched.algo != ALGO_BRUCK) return 0;
+    return (size_t)p->sched.P * p->sched.P * p->sched.m;
+}
+
+int sparbit_plan_set_workspace(sparbit_plan_t* p, void* dev, size_t bytes) {
+    if (!p) return SPARBIT_ERR_ARG;
+    if (bytes < sparbit_plan_workspace_bytes(p)) return SPARBIT_ERR_WORKSPACE;
+    if (!dev && sparbit_plan_workspace_bytes(p) > 0) return SPARBIT_ERR_WORKSPACE;
+    p->work = dev;
+    p->work_bytes = bytes;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_set_copy_path(sparbit_plan_t* p, int copy_path) {
+    if (!p || copy_path < SPARBIT_COPY_AUTO || copy_path > SPARBIT_COPY_BULK) return SPARBIT_ERR_ARG;
+    p->copy_req = copy_path;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_exec_mode(const sparbit_plan_t* p) {
+    if (!p) return -1;
+    if (p->exec_req != SPARBIT_EXEC_AUTO) return p->exec_req;
+    // before the first launch the device is not known yet: assume a B200 (both features present)
+    return auto_exec(p->sched, p->dev_ready ? p->coop != 0 : true, p->dev_ready ? p->cluster_ok != 0 : true);
+}
+
+int sparbit_plan_copy_path(const sparbit_plan_t* p) { return p ? p->copy_last : -1; }
+
+int sparbit_plan_launch_counts(const sparbit_plan_t* p, uint64_t* kernel_launches, uint64_t* graph_launches) {
+    if (!p) return SPARBIT_ERR_ARG;
+    if (kernel_launches) *kernel_launches = p->kernel_launches;
+    if (graph_launches) *graph_launches = p->graph_launches;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_status(sparbit_plan_t* p, int* device_status) {
+    if (!p) return SPARBIT_ERR_ARG;
+    if (device_status) *device_status = 0;
+    if (!p->dev_ready || !p->launched) return SPARBIT_OK;
+    CU(cudaStreamSynchronize(p->last_stream));
+    unsigned ctl[2] = {0, 0};
+    CU(cudaMemcpy(ctl, p->d_ctl, sizeof ctl, cudaMemcpyDeviceToHost));
+    if (device_status) *device_status = (int)ctl[1];
+    if (ctl[1] != DEV_OK) {
+        // a failed launch leaves the arrival counter in an unknown state: start over
+        CU(cudaMemset(p->d_ctl, 0, sizeof ctl));
+        p->bar_base = 0;
+        return SPARBIT_ERR_TIMEOUT;
+    }
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_set_barrier_test(sparbit_plan_t* p, int extra_arrivals, uint64_t timeout_ns) {
+    if (!p || extra_arrivals < 0) return SPARBIT_ERR_ARG;
+    p->extra_arrivals = extra_arrivals;
+    p->timeout_ns = timeout_ns ? timeout_ns : kDefaultTimeoutNs;
+    return SPARBIT_OK;
+}
+
+const char* sparbit_strerror(int code) {
+    switch (code) {
+        case SPARBIT_OK: return "success";
+        case SPARBIT_ERR_ARG: return "invalid argument";
+        case SPARBIT_ERR_OVERFLOW: return "size not representable";
+        case SPARBIT_ERR_ALIAS: return "buffers overlap";
+        case SPARBIT_ERR_UNSUPPORTED: return "unsupported (recursive doubling needs a power-of-two P)";
+        case SPARBIT_ERR_WORKSPACE: return "workspace missing or too small";
+        case SPARBIT_ERR_CUDA: return "CUDA runtime error";
+        case SPARBIT_ERR_TIMEOUT: return "device barrier timed out";
+        case SPARBIT_ERR_NOMEM: return "out of host memory";
+        default: return "unknown error";
+    }
+}
+
+const char* sparbit_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,447 @@
+// Copy kernels of the step executor (sm_100a).
+//
+// Two copy engines execute one phase (a set of block copies given by a PhaseDesc):
+//
+//   vector  warp-cooperative ld.global.cg / st.global.cg with 16-, 8-, 4-, 2- or 1-byte vectors.
+//           A warp task is a span of one copy (32 lanes x U vectors, index arithmetic once per
+//           span) or, for copies shorter than a warp row, a row of several whole copies.
+//   bulk    cp.async.bulk global -> shared -> global through a ring of shared-memory stages, one
+//           elected lane per warp driving its own ring; completion of loads through mbarriers,
+//           of stores through bulk async-groups.  No cluster multicast anywhere: every block has
+//           exactly one destination.
+//
+// and three ways to sequence phases: one kernel per phase (stream or CUDA-graph chain), one
+// persistent cooperative kernel with a bounded-wait grid barrier after every phase, or one
+// thread-block cluster with the hardware cluster barrier after every phase.
+//
+// Loads never use the non-coherent path: data written in one phase is read by other SMs in the
+// next one inside the same launch.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "phase_desc.h"
+
+namespace spb {
+
+// device status word values
+enum : unsigned { DEV_OK = 0u, DEV_BARRIER_TIMEOUT = 1u, DEV_MBARRIER_TIMEOUT = 2u };
+
+struct BarrierCtl {
+    unsigned* counter;        // monotonically increasing arrival counter
+    unsigned* status;         // device status word (DEV_*)
+    unsigned  base;           // counter value when this launch starts
+    unsigned  expected;       // arrivals that complete one barrier (grid size, + test extra)
+    unsigned long long timeout_ns;
+};
+
+struct BulkCfg {
+    uint32_t stage_bytes;     // bytes per shared-memory stage (multiple of 16)
+    uint32_t pad_;
+};
+
+constexpr int kBulkStages = 8;     // stages per ring
+constexpr int kBulkLoadsAhead = 4; // loads in flight per ring; the rest hold pending stores
+constexpr int kVecUnroll = 4;      // vectors per lane per warp task
+
+// ------------------------------------------------------------------------------------------------
+// small PTX helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned ld_relaxed_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all() {
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+        "l"(gsrc), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------------
+// vector engine
+// ------------------------------------------------------------------------------------------------
+template <typename V>
+__device__ __forceinline__ V ld_cg(const V* p);
+template <typename V>
+__device__ __forceinline__ void st_cg(V* p, V v);
+
+template <>
+__device__ __forceinline__ uint4 ld_cg<uint4>(const uint4* p) { return __ldcg(p); }
+template <>
+__device__ __forceinline__ uint2 ld_cg<uint2>(const uint2* p) { return __ldcg(p); }
+template <>
+__device__ __forceinline__ unsigned ld_cg<unsigned>(const unsigned* p) { return __ldcg(p); }
+template <>
+__device__ __forceinline__ unsigned short ld_cg<unsigned short>(const unsigned short* p) { return __ldcg(p); }
+template <>
+__device__ __forceinline__ unsigned char ld_cg<unsigned char>(const unsigned char* p) { return __ldcg(p); }
+template <>
+__device__ __forceinline__ void st_cg<uint4>(uint4* p, uint4 v) { __stcg(p, v); }
+template <>
+__device__ __forceinline__ void st_cg<uint2>(uint2* p, uint2 v) { __stcg(p, v); }
+template <>
+__device__ __forceinline__ void st_cg<unsigned>(unsigned* p, unsigned v) { __stcg(p, v); }
+template <>
+__device__ __forceinline__ void st_cg<unsigned short>(unsigned short* p, unsigned short v) { __stcg(p, v); }
+template <>
+__device__ __forceinline__ void st_cg<unsigned char>(unsigned char* p, unsigned char v) { __stcg(p, v); }
+
+// One phase on the vector engine.  warp_id / n_warps enumerate all warps taking part.
+// Requires P * copies * ceil(vectors_per_copy / (32*U)) < 2^32 (checked on the host).
+template <typename V>
+__device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uint32_t warp_id, uint32_t n_warps,
+                                          uint32_t lane) {
+    constexpr int U = kVecUnroll;
+    const uint32_t P = g.P;
+    const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy
+    const uint32_t n_copies = P * d.copies;            // copies in the phase (< 2^32, host-checked)
+    const char* sbase = space_base(g, d.src_space);
+    char* dbase = space_base(g, d.dst_space);
+    const uint64_t spitch = space_pitch(g, d.src_space);
+    const uint64_t dpitch = space_pitch(g, d.dst_space);
+
+    if (vpc64 >= 32) {
+        // a task is one span of 32*U vectors inside one copy
+        const uint32_t span = 32u * U;
+        const uint32_t spc = (uint32_t)((vpc64 + span - 1) / span);  // spans per copy
+        const uint64_t tasks = (uint64_t)n_copies * spc;
+        for (uint64_t w = warp_id; w < tasks; w += n_warps) {
+            const uint32_t w32 = (uint32_t)w;
+            const uint32_t q = w32 / spc;
+            const uint32_t sp = w32 - q * spc;
+            const uint32_t r = q / d.copies;
+            const uint32_t j = q - r * d.copies;
+            const CopyLoc c = locate_copy(d, P, r, j);
+            const V* src = reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
+            V* dst = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m));
+            const uint64_t v0 = (uint64_t)sp * span + lane;
+            V regs[U];
+#pragma unroll
+            for (int k = 0; k < U; k++) {
+                const uint64_t v = v0 + 32u * k;
+                if (v < vpc64) regs[k] = ld_cg<V>(src + v);
+            }
+#pragma unroll
+            for (int k = 0; k < U; k++) {
+                const uint64_t v = v0 + 32u * k;
+                if (v < vpc64) st_cg<V>(dst + v, regs[k]);
+            }
+        }
+    } else if (vpc64 > 0) {
+        // a copy is shorter than a warp row: a row holds cpw whole copies, a task is U rows
+        const uint32_t vpc = (uint32_t)vpc64;
+        const uint32_t cpw = 32u / vpc;
+        const uint32_t sub = lane / vpc;       // which copy of the row
+        const uint32_t v = lane - sub * vpc;   // which vector of that copy
+        const bool lane_on = sub < cpw;
+        const uint32_t per_task = cpw * U;
+        const uint64_t tasks = ((uint64_t)n_copies + per_task - 1) / per_task;
+        for (uint64_t w = warp_id; w < tasks; w += n_warps) {
+            V regs[U];
+            V* dsts[U];
+#pragma unroll
+            for (int k = 0; k < U; k++) {
+                const uint64_t q64 = (w * U + k) * cpw + sub;
+                dsts[k] = nullptr;
+                if (lane_on && q64 < n_copies) {
+                    const uint32_t q = (uint32_t)q64;
+                    const uint32_t r = q / d.copies;
+                    const uint32_t j = q - r * d.copies;
+                    const CopyLoc c = locate_copy(d, P, r, j);
+                    const V* src =
+                        reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
+                    dsts[k] = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
+                    regs[k] = ld_cg<V>(src + v);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < U; k++)
+                if (dsts[k]) st_cg<V>(dsts[k], regs[k]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// bulk engine
+// ------------------------------------------------------------------------------------------------
+struct BulkPipe {
+    uint32_t ring;      // shared address of this warp's first stage
+    uint32_t bars;      // shared address of this warp's first mbarrier (kBulkStages of them)
+    uint32_t meta;      // shared address of per-stage {dst pointer, bytes} records (16 B each)
+    uint32_t it;        // stages used so far by this ring (carried across phases)
+};
+
+// Bounded wait on one mbarrier phase.  Returns false (after setting the status word) on time-out
+// or when another CTA already reported a failure.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned* status,
+                                                  unsigned long long timeout_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 63u) == 0) {
+            if (ld_relaxed_gpu(status) != DEV_OK) return false;
+            if (globaltimer_ns() - t0 > timeout_ns) {
+                atomicCAS(status, DEV_OK, DEV_MBARRIER_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// One phase on the bulk engine, driven by ONE thread (the elected lane of a warp).  pipe_id /
+// n_pipes enumerate all rings taking part.  All addresses and sizes are multiples of 16 bytes
+// (host-checked).  Returns false if a wait gave up.
+__device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, uint32_t stage_bytes, uint32_t pipe_id,
+                                           uint32_t n_pipes, BulkPipe& pp, unsigned* status,
+                                           unsigned long long timeout_ns) {
+    constexpr int S = kBulkStages;
+    constexpr int L = kBulkLoadsAhead;
+    const uint32_t P = g.P;
+    const uint64_t cpc = (d.copy_bytes + stage_bytes - 1) / stage_bytes;  // chunks per copy
+    const uint64_t tasks = (uint64_t)P * d.copies * cpc;
+    if (pipe_id >= tasks) return true;
+    // equal chunks (rounded up to 128 B) instead of full stages plus a short tail
+    const uint32_t chunk = (uint32_t)((((d.copy_bytes + cpc - 1) / cpc) + 127u) & ~127ull);
+    fence_proxy_async_all();  // what other CTAs wrote before the barrier -> visible to bulk loads
+    const uint64_t mine = (tasks - pipe_id + n_pipes - 1) / n_pipes;      // tasks of this ring
+    const char* sbase = space_base(g, d.src_space);
+    char* dbase = space_base(g, d.dst_space);
+    const uint64_t spitch = space_pitch(g, d.src_space);
+    const uint64_t dpitch = space_pitch(g, d.dst_space);
+    bool ok = true;
+
+    for (uint64_t i = 0; i < mine + L; i++) {
+        if (i < mine) {
+            const uint32_t slot_it = pp.it + (uint32_t)i;
+            const uint32_t st = slot_it % S;
+            // the store that last used this stage (S tasks ago) must have finished reading shared
+            // memory: stores are committed one group per task, L tasks behind the loads
+            bulk_wait_read<S - L - 1>();
+            const uint64_t w = pipe_id + i * n_pipes;
+            const uint64_t q = w / cpc;
+            const uint64_t ch = w - q * cpc;
+            const uint32_t r = (uint32_t)(q / d.copies);
+            const uint32_t j = (uint32_t)(q - (uint64_t)r * d.copies);
+            const CopyLoc c = locate_copy(d, P, r, j);
+            const uint64_t off = ch * chunk;
+            const uint64_t left = d.copy_bytes - off;
+            const uint32_t bytes = left < chunk ? (uint32_t)left : chunk;
+            const char* src = sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m) + off;
+            char* dst = dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m) + off;
+            const uint32_t bar = pp.bars + st * 8u;
+            // remember where this stage goes
+            asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(pp.meta + st * 16u), "l"(dst),
+                         "l"((unsigned long long)bytes)
+                         : "memory");
+            mbar_expect_tx(bar, bytes);
+            bulk_load(pp.ring + st * stage_bytes, src, bytes, bar);
+        }
+        if (i >= (uint64_t)L) {
+            const uint32_t slot_it = pp.it + (uint32_t)(i - L);
+            const uint32_t st = slot_it % S;
+            const uint32_t parity = (slot_it / S) & 1u;
+            if (!mbar_wait_bounded(pp.bars + st * 8u, parity, status, timeout_ns)) {
+                ok = false;
+                break;
+            }
+            unsigned long long dst, bytes;
+            asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(dst), "=l"(bytes) : "r"(pp.meta + st * 16u)
+                         : "memory");
+            bulk_store(reinterpret_cast<void*>(dst), pp.ring + st * stage_bytes, (uint32_t)bytes);
+            bulk_commit();
+        }
+    }
+    pp.it += (uint32_t)mine;
+    // all stores of this phase complete (written, not only read) before anyone is told about it
+    bulk_wait_all();
+    fence_proxy_async_all();
+    return ok;
+}
+
+// ------------------------------------------------------------------------------------------------
+// bounded-wait grid barrier (persistent executor)
+// ------------------------------------------------------------------------------------------------
+// All threads of all CTAs call it; `epoch` counts the barriers this launch has passed.  Returns
+// false when the wait gave up or another CTA reported a failure: the caller must then leave the
+// kernel.  Co-residency of the grid is guaranteed by the cooperative launch.
+__device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& epoch, int* smem_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        epoch++;
+        const unsigned target = ctl.base + epoch * ctl.expected;
+        fence_proxy_async_all();          // bulk stores of this CTA -> visible before the release
+        red_release_gpu_add(ctl.counter, 1u);
+        bool ok = true;
+        unsigned polls = 0;
+        unsigned long long t0 = 0;
+        while ((int)(ld_acquire_gpu(ctl.counter) - target) < 0) {
+            if ((++polls & 31u) == 0) {
+                if (t0 == 0) t0 = globaltimer_ns();
+                if (ld_relaxed_gpu(ctl.status) != DEV_OK) {
+                    ok = false;
+                    break;
+                }
+                if (globaltimer_ns() - t0 > ctl.timeout_ns) {
+                    atomicCAS(ctl.status, DEV_OK, DEV_BARRIER_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+            }
+        }
+        fence_proxy_async_all();          // later bulk loads see what the other CTAs wrote
+        *smem_flag = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *smem_flag != 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+// kernels
+// ------------------------------------------------------------------------------------------------
+// one phase, vector engine
+template <typename V>
+__global__ void __launch_bounds__(512) phase_vec_kernel(Geom g, PhaseDesc d) {
+    const uint32_t wpb = blockDim.x >> 5;
+    vec_phase<V>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
+}
+
+// shared-memory layout of the bulk kernels: [rings | mbarriers | meta], ring stages 128-B aligned
+__device__ __forceinline__ BulkPipe make_pipe(unsigned char* smem, uint32_t stage_bytes, uint32_t warps,
+                                              uint32_t warp) {
+    BulkPipe pp;
+    const uint32_t base = smem_u32(smem);
+    const uint32_t rings = warps * kBulkStages * stage_bytes;
+    pp.ring = base + warp * kBulkStages * stage_bytes;
+    pp.bars = base + rings + warp * kBulkStages * 8u;
+    pp.meta = base + rings + warps * kBulkStages * 8u + warp * kBulkStages * 16u;
+    pp.it = 0;
+    return pp;
+}
+__device__ __forceinline__ void init_pipe(const BulkPipe& pp) {
+    for (int s = 0; s < kBulkStages; s++) mbar_init(pp.bars + s * 8u, 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_all();
+}
+
+// one phase, bulk engine
+__global__ void __launch_bounds__(256) phase_bulk_kernel(Geom g, PhaseDesc d, uint32_t stage_bytes, unsigned* status,
+                                                         unsigned long long timeout_ns) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t warps = blockDim.x >> 5;
+    const uint32_t warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31u) == 0) {
+        BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
+        init_pipe(pp);
+        bulk_phase(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, status, timeout_ns);
+    }
+}
+
+// phases first..last (indices into descs), vector engine, grid barrier between phases
+template <typename V>
+__global__ void __launch_bounds__(512) persistent_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
+                                                             int last, BarrierCtl ctl) {
+    __shared__ int flag;
+    if (ld_relaxed_gpu(ctl.status) != DEV_OK) return;  // an earlier failure was not cleared yet
+    const uint32_t wpb = blockDim.x >> 5;
+    const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
+    const uint32_t n_warps = gridDim.x * wpb;
+    unsigned epoch = 0;
+    for (int ph = first; ph <= last; ph++) {
+        const PhaseDesc d = descs[ph];
+        vec_phase<V>(g, d, warp_id, n_warps, threadIdx.x & 31u);
+        if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
+    }
+}
+
+// phases first..last, bulk engine, grid barrier between phases
+__global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
+                                                              int last, uint32_t stage_bytes, BarrierCtl ctl) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int flag;
+    if (ld_relaxed_gpu(ctl.status) != DEV_OK) return;
+    const uint32_t warps = blockDim.x >> 5;
+    const uint32_t warp = threadIdx.x >> 5;
+    const bool driver = (threadIdx.x & 31u) == 0;
+    BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
+    if (driver) init_pipe(pp);
+    unsigned epoch = 0;
+    for (int ph = first; ph <= last; ph++) {
+        if (driver) {
+            const PhaseDesc d = descs[ph];
+            bulk_phase(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
+                       ctl.timeout_ns);
+        }
+        if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
+    }
+}
+
+// phases first..last, vector engine, ONE thread-block cluster as the whole grid: the hardware
+// cluster barrier (arrive.release / wait.acquire) separates phases.  For collectives so small
+// that a grid-wide barrier or a kernel boundary per phase would dominate.
+template <typename V>
+__global__ void __launch_bounds__(512) cluster_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
+                                                           int last) {
+    const uint32_t wpb = blockDim.x >> 5;
+    const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
+    const uint32_t n_warps = gridDim.x * wpb;
+    for (int ph = first; ph <= last; ph++) {
+        const PhaseDesc d = descs[ph];
+        vec_phase<V>(g, d, warp_id, n_warps, threadIdx.x & 31u);
+        if (ph != last) {
+            asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        }
+    }
+}
+
+}  // namespace spb

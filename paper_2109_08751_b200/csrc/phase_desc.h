@@ -1,0 +1,96 @@
+// Compact per-phase descriptor shared by the host schedule generator and the copy kernels.
+//
+// A phase is a set of block copies, one per (rank r, index j) with 0 <= r < P, 0 <= j < copies:
+//
+//   dst_rank = peer_xor ? r ^ peer_xor : (r + peer_add) mod P
+//   src_slot = wrap(wrap1(src_rcoef * (r & rank_mask) + src_off) + j * src_step)
+//   dst_slot = wrap(wrap1(dst_rcoef * (r & rank_mask) + dst_off) + j * dst_step)
+//
+// wrap1 folds a value in [0, 2P) into [0, P); wrap folds a value in (-P, 2P) into [0, P).  The
+// schedule generator guarantees those ranges (|j * step| < P), so no division is needed on the
+// device.  Each copy moves copy_bytes = run * m bytes: `run` consecutive slots when the phase's
+// blocks are contiguous on both sides (recursive doubling, Bruck), else one block.
+//
+// This form covers Algorithm 1's steps (peer r + d, slots r - 2jd on both sides), the ring, the
+// recursive-doubling exchange (peer r xor 2^s, aligned groups), Bruck's steps and rotation, and
+// the own-block copy, in O(1) bytes per phase whatever P is.
+#pragma once
+#include <stdint.h>
+
+#if defined(__CUDACC__)
+#define SPB_HD __host__ __device__ __forceinline__
+#else
+#define SPB_HD inline
+#endif
+
+namespace spb {
+
+enum Space : uint32_t { SPACE_SEND = 0, SPACE_RECV = 1, SPACE_WORK = 2 };
+
+struct PhaseDesc {
+    uint32_t copies;     // copies per rank executed by the kernels (= blocks / run)
+    uint32_t run;        // blocks per copy
+    uint32_t peer_add;   // in [0, P)
+    uint32_t peer_xor;   // 0 = use peer_add
+    uint32_t rank_mask;
+    uint32_t src_rcoef;  // 0 or 1
+    uint32_t src_off;    // in [0, P)
+    int32_t  src_step;   // slots between consecutive copies of a rank (signed)
+    uint32_t dst_rcoef;
+    uint32_t dst_off;
+    int32_t  dst_step;
+    uint32_t src_space;
+    uint32_t dst_space;
+    uint32_t pad_;
+    uint64_t copy_bytes; // run * m
+};
+
+// Geometry of one collective call: where the three spaces live.
+struct Geom {
+    uint32_t P;
+    uint32_t pad_;
+    uint64_t m;               // bytes per block (slot pitch)
+    char*    base[3];         // SEND, RECV, WORK
+    uint64_t rank_pitch[3];   // bytes between consecutive ranks' buffers: m, P*m, P*m
+};
+
+struct CopyLoc {
+    uint32_t src_rank, dst_rank, src_slot, dst_slot;
+};
+
+SPB_HD uint32_t wrap_slot(int64_t v, uint32_t P) {
+    if (v < 0) v += P;
+    if (v >= (int64_t)P) v -= P;
+    return (uint32_t)v;
+}
+
+// Where copy j of rank r reads and writes.  The single definition used by the kernels and by the
+// host-side expansion into explicit messages.
+SPB_HD CopyLoc locate_copy(const PhaseDesc& d, uint32_t P, uint32_t r, uint32_t j) {
+    CopyLoc c;
+    c.src_rank = r;
+    if (d.peer_xor) {
+        c.dst_rank = r ^ d.peer_xor;
+    } else {
+        uint32_t t = r + d.peer_add;
+        c.dst_rank = t >= P ? t - P : t;
+    }
+    uint32_t rr = r & d.rank_mask;
+    int64_t s = (int64_t)d.src_rcoef * rr + d.src_off;
+    if (s >= (int64_t)P) s -= P;
+    c.src_slot = wrap_slot(s + (int64_t)j * d.src_step, P);
+    int64_t t = (int64_t)d.dst_rcoef * rr + d.dst_off;
+    if (t >= (int64_t)P) t -= P;
+    c.dst_slot = wrap_slot(t + (int64_t)j * d.dst_step, P);
+    return c;
+}
+
+// selects instead of dynamic indexing: kernel parameters stay in the constant bank
+SPB_HD char* space_base(const Geom& g, uint32_t space) {
+    return space == SPACE_SEND ? g.base[0] : (space == SPACE_RECV ? g.base[1] : g.base[2]);
+}
+SPB_HD uint64_t space_pitch(const Geom& g, uint32_t space) {
+    return space == SPACE_SEND ? g.rank_pitch[0] : (space == SPACE_RECV ? g.rank_pitch[1] : g.rank_pitch[2]);
+}
+
+}  // namespace spb

@@ -1,0 +1,208 @@
+// Host schedule generator.
+//
+// Sparbit follows Algorithm 1 of the paper: lines 1-5 give the first distance and the bit vector
+// of steps that withhold a block, the loop gives each step's distance d and message count
+// data - ignore, and the state update (d >>= 1; data = 2*data - ignore) carries them forward.  A
+// step's messages are not listed one by one: they are the copies (r, j) -> peer r + d, slot
+// r - 2jd on both sides, which the PhaseDesc form states in O(1) bytes.  The counts are
+// cross-checked against the counting form ceil(P/d) - ceil(P/2d) before a plan is accepted.
+//
+// Ring, recursive doubling and Bruck (Section II-A) are expressed in the same descriptor form.
+#include "schedule.h"
+
+#include <string.h>
+
+namespace spb {
+
+static int ceil_log2(uint64_t p) {
+    int k = 0;
+    while ((1ull << k) < p) k++;
+    return k;
+}
+
+static int floor_log2(uint64_t p) {
+    int k = 0;
+    while ((2ull << k) <= p) k++;
+    return k;
+}
+
+static PhaseDesc blank(uint64_t m) {
+    PhaseDesc d;
+    memset(&d, 0, sizeof d);
+    d.copies = 1;
+    d.run = 1;
+    d.rank_mask = 0xFFFFFFFFu;
+    d.copy_bytes = m;
+    return d;
+}
+
+// own block: sendbuf[r] -> (space)[r][slot r or 0]
+static PhaseDesc own_copy(uint64_t m, bool into_work) {
+    PhaseDesc d = blank(m);
+    d.src_space = SPACE_SEND;  // one slot per rank: slot 0
+    d.dst_space = into_work ? SPACE_WORK : SPACE_RECV;
+    d.dst_rcoef = into_work ? 0u : 1u;
+    return d;
+}
+
+static bool steps_stay_in_range(const PhaseDesc& d, uint32_t P) {
+    // (copies-1) * |step| < P keeps base + j*step inside (-P, 2P)
+    uint64_t a = (uint64_t)(d.copies - 1) * (uint64_t)(d.src_step < 0 ? -(int64_t)d.src_step : d.src_step);
+    uint64_t b = (uint64_t)(d.copies - 1) * (uint64_t)(d.dst_step < 0 ? -(int64_t)d.dst_step : d.dst_step);
+    return a < P && b < P && d.src_off < P && d.dst_off < P && d.peer_add < P;
+}
+
+static int build_sparbit(uint32_t P, uint64_t m, Schedule& s) {
+    const int K = ceil_log2(P);
+    s.K = K;
+    s.phases.push_back(own_copy(m, false));
+    if (K == 0) return SCHED_OK;  // one rank: nothing to exchange
+    // Algorithm 1, lines 1-5
+    uint32_t data = 1, ignore = 0;
+    uint32_t d = 1u << (K - 1);
+    uint32_t last_ignore = (uint32_t)__builtin_ctz(P);
+    uint32_t ignore_steps = (~(P >> last_ignore) | 1u) << last_ignore;
+    for (int i = 0; i < K; i++) {
+        if (d & ignore_steps) ignore = 1;
+        const uint32_t n = data - ignore;
+        // counting form: a rank holds ceil(P/2d) blocks before and ceil(P/d) after the step
+        const uint32_t before = (uint32_t)((P + 2ull * d - 1) / (2ull * d));
+        const uint32_t after = (P + d - 1) / d;
+        if (data != before || n != after - before) return SCHED_INTERNAL;
+        PhaseDesc ph = blank(m);
+        ph.copies = n;
+        ph.peer_add = d;                 // d <= 2^(K-1) < P
+        ph.src_space = ph.dst_space = SPACE_RECV;
+        ph.src_rcoef = ph.dst_rcoef = 1; // displacement (rank - 2jd) mod P, the same on both sides:
+        ph.src_step = ph.dst_step = -(int32_t)(2 * d);  // receiver r+d stores at (r+d) - (2j+1)d
+        if (!steps_stay_in_range(ph, P)) return SCHED_INTERNAL;
+        s.phases.push_back(ph);
+        s.steps.push_back({(int)d, (int)n, (int)ignore});
+        d >>= 1;
+        data = (data << 1) - ignore;
+        ignore = 0;
+    }
+    if (data != P) return SCHED_INTERNAL;  // every rank ends up holding all P blocks
+    return SCHED_OK;
+}
+
+static int build_ring(uint32_t P, uint64_t m, Schedule& s) {
+    s.K = (int)P - 1;
+    s.phases.push_back(own_copy(m, false));
+    for (uint32_t st = 0; st + 1 < P; st++) {
+        PhaseDesc ph = blank(m);  // r forwards the block of rank r - st to r + 1, same slot there
+        ph.peer_add = 1 % P;
+        ph.src_space = ph.dst_space = SPACE_RECV;
+        ph.src_rcoef = ph.dst_rcoef = 1;
+        ph.src_off = ph.dst_off = (P - st % P) % P;
+        if (!steps_stay_in_range(ph, P)) return SCHED_INTERNAL;
+        s.phases.push_back(ph);
+        s.steps.push_back({1, 1, 0});
+    }
+    return SCHED_OK;
+}
+
+static int build_rd(uint32_t P, uint64_t m, Schedule& s) {
+    if (P & (P - 1)) return SCHED_UNSUPPORTED;
+    const int K = ceil_log2(P);
+    s.K = K;
+    s.phases.push_back(own_copy(m, false));
+    for (int st = 0; st < K; st++) {
+        const uint32_t g = 1u << st;  // r and r xor g swap their aligned groups of g slots
+        PhaseDesc ph = blank(m);
+        ph.peer_xor = g;
+        ph.rank_mask = ~(g - 1);
+        ph.src_space = ph.dst_space = SPACE_RECV;
+        ph.src_rcoef = ph.dst_rcoef = 1;
+        ph.src_step = ph.dst_step = 1;
+        ph.copies = 1;  // the g slots are contiguous on both sides: one copy of g blocks
+        ph.run = g;
+        ph.copy_bytes = (uint64_t)g * m;
+        if (!steps_stay_in_range(ph, P)) return SCHED_INTERNAL;
+        s.phases.push_back(ph);
+        s.steps.push_back({(int)g, (int)g, 0});
+    }
+    return SCHED_OK;
+}
+
+static int build_bruck(uint32_t P, uint64_t m, Schedule& s) {
+    const int K = ceil_log2(P);
+    const int F = floor_log2(P);
+    s.K = K;
+    s.rotation = true;
+    s.phases.push_back(own_copy(m, true));  // working slot i of rank r holds block (r + i) mod P
+    for (int st = 0; st < K; st++) {
+        const uint32_t dist = 1u << st;
+        const uint32_t n = st < F ? dist : P - dist;  // last step of a non-power of two: the rest
+        PhaseDesc ph = blank(m);
+        ph.peer_add = (P - dist % P) % P;             // sends to r - 2^st
+        ph.src_space = ph.dst_space = SPACE_WORK;
+        ph.src_off = 0;                               // the first n working slots ...
+        ph.dst_off = dist;                            // ... land behind what the receiver holds
+        ph.src_step = ph.dst_step = 1;
+        ph.copies = 1;
+        ph.run = n;
+        ph.copy_bytes = (uint64_t)n * m;
+        if (!steps_stay_in_range(ph, P) || dist + n > P) return SCHED_INTERNAL;
+        s.phases.push_back(ph);
+        s.steps.push_back({(int)dist, (int)n, 0});
+    }
+    PhaseDesc rot = blank(m);  // workspace[r][i] -> recvbuf[r][(r + i) mod P]
+    rot.copies = P;
+    rot.src_space = SPACE_WORK;
+    rot.dst_space = SPACE_RECV;
+    rot.src_step = 1;
+    rot.dst_rcoef = 1;
+    rot.dst_step = 1;
+    if (!steps_stay_in_range(rot, P)) return SCHED_INTERNAL;
+    s.phases.push_back(rot);
+    return SCHED_OK;
+}
+
+int build_schedule(int algo, int64_t P64, uint64_t m, Schedule& out) {
+    if (P64 < 1) return SCHED_ARG;
+    if (P64 > (1 << 24)) return SCHED_OVERFLOW;
+    const uint32_t P = (uint32_t)P64;
+    // P * P * m must fit comfortably in 63 bits
+    const unsigned __int128 total = (unsigned __int128)P * P * m;
+    if (total >> 62) return SCHED_OVERFLOW;
+    out = Schedule();
+    out.algo = algo;
+    out.P = P;
+    out.m = m;
+    switch (algo) {
+        case ALGO_SPARBIT: return build_sparbit(P, m, out);
+        case ALGO_RING: return build_ring(P, m, out);
+        case ALGO_RD: return build_rd(P, m, out);
+        case ALGO_BRUCK: return build_bruck(P, m, out);
+        default: return SCHED_ARG;
+    }
+}
+
+uint64_t phase_message_count(const Schedule& s, int phase) {
+    const PhaseDesc& d = s.phase(phase);
+    return (uint64_t)s.P * d.copies * d.run;
+}
+
+void expand_phase(const Schedule& s, int phase, std::vector<Msg>& out) {
+    const PhaseDesc& d = s.phase(phase);
+    out.clear();
+    out.reserve((size_t)phase_message_count(s, phase));
+    for (uint32_t r = 0; r < s.P; r++)
+        for (uint32_t j = 0; j < d.copies; j++) {
+            const CopyLoc c = locate_copy(d, s.P, r, j);
+            for (uint32_t k = 0; k < d.run; k++) {  // a run is `run` consecutive slots, no wrap
+                Msg msg;
+                msg.phase = phase;
+                msg.src_rank = (int32_t)c.src_rank;
+                msg.dst_rank = (int32_t)c.dst_rank;
+                msg.src_space = (int32_t)d.src_space;
+                msg.src_slot = (int32_t)(c.src_slot + k);
+                msg.dst_space = (int32_t)d.dst_space;
+                msg.dst_slot = (int32_t)(c.dst_slot + k);
+                out.push_back(msg);
+            }
+        }
+}
+
+}  // namespace spb

@@ -1,0 +1,47 @@
+// Host schedule generator: turns (algorithm, P, m) into compact per-phase descriptors.
+#pragma once
+#include <stdint.h>
+
+#include <vector>
+
+#include "phase_desc.h"
+
+namespace spb {
+
+enum Algo { ALGO_SPARBIT = 0, ALGO_RING = 1, ALGO_RD = 2, ALGO_BRUCK = 3 };
+
+struct StepInfo {
+    int distance;  // ranks between sender and receiver (Algorithm 1's d)
+    int blocks;    // messages per rank in the step (Algorithm 1's data - ignore)
+    int ignore;    // 1 when the step withholds a block
+};
+
+struct Schedule {
+    int algo = 0;
+    uint32_t P = 0;
+    uint64_t m = 0;
+    int K = 0;               // communication steps
+    bool rotation = false;   // Bruck's final phase
+    // phases[0] is phase -1 (own block), phases[1 + s] is step s, phases[1 + K] the rotation
+    std::vector<PhaseDesc> phases;
+    std::vector<StepInfo> steps;
+    int last_phase() const { return rotation ? K : K - 1; }
+    const PhaseDesc& phase(int ph) const { return phases[(size_t)(ph + 1)]; }
+};
+
+// Error codes returned by build_schedule (mapped to the public ones by the caller).
+enum { SCHED_OK = 0, SCHED_ARG = 1, SCHED_OVERFLOW = 2, SCHED_UNSUPPORTED = 4, SCHED_INTERNAL = 99 };
+
+int build_schedule(int algo, int64_t P, uint64_t m, Schedule& out);
+
+struct Msg {
+    int32_t phase, src_rank, dst_rank, src_space, src_slot, dst_space, dst_slot;
+};
+
+// Explicit single-block messages of one phase, through locate_copy (the kernels' index function).
+void expand_phase(const Schedule& s, int phase, std::vector<Msg>& out);
+
+// Number of single-block messages of one phase.
+uint64_t phase_message_count(const Schedule& s, int phase);
+
+}  // namespace spb

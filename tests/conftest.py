@@ -10,6 +10,10 @@ if str(ROOT) not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+    # the library is built in-tree; rebuild only when a source is newer than the shared object
+    from paper_2109_08751_b200 import build as lib_build
+
+    lib_build.build()
 
 
 @pytest.fixture(scope="session")

@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA step executor against the CPU oracle, bit for bit, through the C ABI.
+
+Receive buffers (and Bruck workspaces) are pre-filled with a sentinel and sit between guard bands
+that are checked after every run; the data changes on every iteration, because an allgather
+repeated on unchanged inputs would hide stale reads (the previous run already left the right
+answer in place).
+"""
+import ctypes
+
+import numpy as np
+import pytest
+
+import oracle
+import seeded_inputs as si
+import paper_2109_08751_b200 as sp
+from paper_2109_08751_b200 import binding
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK]
+EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_CLUSTER]
+COPIES = [sp.COPY_VECTOR, sp.COPY_BULK]
+G = si.GUARD_BYTES
+
+
+def is_pow2(p):
+    return p & (p - 1) == 0
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device")
+    return torch.device("cuda:0")
+
+
+class Guarded:
+    """A device byte buffer of `n` bytes at byte offset `shift` inside a sentinel-filled
+    allocation with guard bands on both sides."""
+
+    def __init__(self, n, dev, shift=0, fill=si.SENTINEL):
+        self.n, self.shift, self.fill = n, shift, fill
+        self.raw = torch.full((n + 2 * G + 64,), fill, dtype=torch.uint8, device=dev)
+        base = self.raw.data_ptr()
+        align = (-base) % 256  # torch allocations are 512-aligned, but do not rely on it
+        self.off = align + G + shift
+        self.view = self.raw[self.off:self.off + n]
+
+    @property
+    def ptr(self):
+        return self.view.data_ptr()
+
+    def guards_intact(self):
+        lo = self.raw[: self.off]
+        hi = self.raw[self.off + self.n:]
+        return bool((lo == self.fill).all()) and bool((hi == self.fill).all())
+
+    def refill(self):
+        self.raw.fill_(self.fill)
+
+
+def run_case(dev, P, m, algo, exec_mode, copy, seed, iters=2, shift_send=0, shift_recv=0, shift_work=0):
+    plan = sp.Plan(P, m, algo, exec_mode)
+    plan.set_copy_path(copy)
+    send = Guarded(P * m, dev, shift_send, fill=0x3C)
+    recv = Guarded(P * P * m, dev, shift_recv)
+    work = None
+    if algo == sp.ALGO_BRUCK:
+        work = Guarded(P * P * m, dev, shift_work)
+        plan.set_workspace(work.ptr, P * P * m)
+    ref_plan = oracle.Plan(algo, P)
+    for it in range(iters):
+        host_send = si.send_blocks(P, m, seed + it)
+        send.view.copy_(torch.from_numpy(host_send.reshape(-1)))
+        recv.refill()
+        if work:
+            work.refill()
+        plan.allgather(send.ptr, recv.ptr)
+        assert plan.status() == sp.OK
+        want = si.sentinel_buffer(P * P * m)
+        scratch = si.sentinel_buffer(P * P * m) if algo == sp.ALGO_BRUCK else None
+        ref_plan.run(m, host_send.reshape(-1), want, scratch)
+        got = recv.view.cpu().numpy()
+        assert np.array_equal(got, want), (P, m, algo, exec_mode, copy, it)
+        assert recv.guards_intact() and send.guards_intact()
+        assert np.array_equal(send.view.cpu().numpy(), host_send.reshape(-1))  # send is read-only
+        if work:
+            assert work.guards_intact()
+            assert np.array_equal(work.view.cpu().numpy(), scratch)
+    plan.destroy()
+
+
+# ---------------------------------------------------------------- config 1: P=8, m=64 B
+@pytest.mark.parametrize("exec_mode", EXECS)
+@pytest.mark.parametrize("copy", COPIES)
+def test_config1_p8_m64(dev, exec_mode, copy):
+    run_case(dev, 8, 64, sp.ALGO_SPARBIT, exec_mode, copy, si.BASE_SEED + 1, iters=3)
+
+
+# ---------------------------------------------------------------- config 2: non powers of two, all algorithms
+@pytest.mark.parametrize("P", [6, 13])
+@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_BRUCK])
+@pytest.mark.parametrize("exec_mode", EXECS)
+@pytest.mark.parametrize("copy", COPIES)
+def test_config2_non_power_of_two(dev, P, algo, exec_mode, copy):
+    run_case(dev, P, 4096, algo, exec_mode, copy, si.BASE_SEED + 2)
+
+
+@pytest.mark.parametrize("P", [4, 8, 16])
+@pytest.mark.parametrize("exec_mode", EXECS)
+@pytest.mark.parametrize("copy", COPIES)
+def test_config2_recursive_doubling_powers_of_two(dev, P, exec_mode, copy):
+    run_case(dev, P, 4096, sp.ALGO_RECURSIVE_DOUBLING, exec_mode, copy, si.BASE_SEED + 2)
+
+
+@pytest.mark.parametrize("P", [6, 13])
+def test_config2_recursive_doubling_refused(P):
+    out = ctypes.c_void_p()
+    assert binding.lib.sparbit_plan_create(P, 4096, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) \
+        == sp.ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------- phase-by-phase state
+@pytest.mark.parametrize("algo,P", [(sp.ALGO_SPARBIT, 5), (sp.ALGO_SPARBIT, 21), (sp.ALGO_SPARBIT, 32),
+                                    (sp.ALGO_BRUCK, 13), (sp.ALGO_RING, 6), (sp.ALGO_RECURSIVE_DOUBLING, 16)])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_STREAM])
+def test_state_after_every_phase(dev, algo, P, exec_mode):
+    """Run one phase at a time on both sides; the whole state (sentinel included) must agree."""
+    m = 272  # 17 * 16: not a power of two, several vectors per block
+    plan = sp.Plan(P, m, algo, exec_mode)
+    ref = oracle.Plan(algo, P)
+    host_send = si.send_blocks(P, m, 77)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    work = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    if algo == sp.ALGO_BRUCK:
+        plan.set_workspace(work, P * P * m)
+    want = si.sentinel_buffer(P * P * m)
+    scratch = si.sentinel_buffer(P * P * m)
+    for ph in range(-1, ref.last_phase + 1):
+        plan.allgather_steps(send, recv, ph, ph)
+        assert plan.status() == sp.OK
+        ref.run(m, host_send.reshape(-1), want, scratch, first=ph, last=ph)
+        assert np.array_equal(recv.cpu().numpy(), want), ph
+        if algo == sp.ALGO_BRUCK:
+            assert np.array_equal(work.cpu().numpy(), scratch), ph
+
+
+# ---------------------------------------------------------------- brute force over P
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_CLUSTER])
+def test_every_p_up_to_64(dev, exec_mode):
+    for P in range(1, 65):
+        run_case(dev, P, 16, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=1)
+
+
+@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK])
+def test_comparators_many_p(dev, algo):
+    for P in [1, 2, 3, 4, 5, 7, 8, 12, 16, 17, 31, 32, 33, 64]:
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        run_case(dev, P, 48, algo, sp.EXEC_PERSISTENT, sp.COPY_AUTO, 2000 + P, iters=1)
+
+
+# ---------------------------------------------------------------- any block size, any alignment
+@pytest.mark.parametrize("m", [1, 2, 3, 6, 10, 20, 100, 1000, 4100, 16400])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_CLUSTER])
+def test_odd_block_sizes(dev, m, exec_mode):
+    run_case(dev, 7, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 31 + m, iters=1)
+
+
+@pytest.mark.parametrize("shifts", [(1, 0, 0), (0, 1, 0), (2, 2, 2), (4, 8, 4), (8, 8, 8), (3, 5, 7), (16, 32, 48)])
+@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_BRUCK])
+def test_misaligned_buffers(dev, shifts, algo):
+    """Buffers at odd addresses must fall back to narrower vectors (and off the bulk engine)."""
+    for m in (64, 4096):
+        for copy in COPIES:
+            run_case(dev, 9, m, algo, sp.EXEC_PERSISTENT, copy, 5, iters=1, shift_send=shifts[0],
+                     shift_recv=shifts[1], shift_work=shifts[2])
+
+
+def test_single_rank_and_empty_blocks(dev):
+    for algo in ALGOS:
+        run_case(dev, 1, 256, algo, sp.EXEC_AUTO, sp.COPY_AUTO, 9, iters=1)
+    plan = sp.Plan(8, 0)
+    plan.allgather(None, None)
+    assert plan.status() == sp.OK
+
+
+# ---------------------------------------------------------------- larger shapes (several tiles, ragged tails)
+@pytest.mark.parametrize("P,m", [(37, 20480 + 16), (128, 8192), (100, 33 * 1024)])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH])
+@pytest.mark.parametrize("copy", COPIES)
+def test_medium_shapes(dev, P, m, exec_mode, copy):
+    run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, copy, 4242)
+
+
+@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK])
+@pytest.mark.parametrize("copy", COPIES)
+def test_medium_shapes_comparators(dev, algo, copy):
+    run_case(dev, 64, 20480, algo, sp.EXEC_PERSISTENT, copy, 4343, iters=1)
+
+
+# ---------------------------------------------------------------- the bounded wait of the grid barrier
+@pytest.mark.parametrize("copy", COPIES)
+def test_grid_barrier_gives_up_instead_of_hanging(dev, copy):
+    """With one arrival more expected than there are CTAs the barrier can never complete: the
+    kernel must come back with the time-out status, and the plan must work again afterwards."""
+    P, m = 16, 4096
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_PERSISTENT)
+    plan.set_copy_path(copy)
+    host_send = si.send_blocks(P, m, 1)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.set_barrier_test(1, 20_000_000)  # 20 ms
+    plan.allgather(send, recv)
+    assert plan.status() == sp.ERR_TIMEOUT
+    assert plan.status() == sp.OK        # the condition is cleared by reading it
+    plan.set_barrier_test(0, 0)
+    recv.fill_(si.SENTINEL)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+
+
+# ---------------------------------------------------------------- host-buffer entry point, streams, bookkeeping
+@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_BRUCK])
+def test_host_entry_point(dev, algo):
+    P, m = 24, 2048
+    plan = sp.Plan(P, m, algo)
+    for it in range(2):
+        host_send = si.send_blocks(P, m, 50 + it)
+        host_recv = si.sentinel_buffer(P * P * m)
+        plan.allgather_host(host_send, host_recv)
+        want, _ = oracle.allgather(algo, P, m, host_send)
+        assert np.array_equal(host_recv, want.reshape(-1))
+
+
+@pytest.mark.parametrize("exec_mode", EXECS)
+def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
+    P, m = 16, 1024
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    host_send = si.send_blocks(P, m, 3)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        send = torch.from_numpy(host_send.reshape(-1)).to(dev, non_blocking=False)
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        stream.synchronize()
+        plan.allgather(send, recv, stream)
+        plan.allgather(send, recv, stream)
+    assert plan.status() == sp.OK
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+    kernels, graphs = plan.launch_counts()
+    phases = plan.num_steps + 1
+    if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_CLUSTER):
+        assert (kernels, graphs) == (2, 0)
+    elif exec_mode == sp.EXEC_GRAPH:
+        assert (kernels, graphs) == (2 * phases, 2)
+    else:
+        assert (kernels, graphs) == (2 * phases, 0)
+    assert plan.exec_mode == exec_mode
+
+
+def test_graph_follows_new_pointers(dev):
+    """The cached graph must not keep using the buffers of an earlier call."""
+    P, m = 12, 4096
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_GRAPH)
+    for it in range(3):
+        host_send = si.send_blocks(P, m, 600 + it)
+        send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+        recv = torch.full((P * P * m + 64 * it,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        plan.allgather(send, recv)
+        assert plan.status() == sp.OK
+        want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+        assert np.array_equal(recv[: P * P * m].cpu().numpy(), want.reshape(-1))

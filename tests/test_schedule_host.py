@@ -1,0 +1,136 @@
+"""Host-side tests of the CUDA library that need no GPU: the C ABI exports what the header
+declares, the compact per-phase descriptors expand to exactly the oracle's message sets, and
+argument errors are caught on the host."""
+import ctypes
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2109_08751_b200 as sp
+from paper_2109_08751_b200 import binding
+
+ROOT = Path(__file__).resolve().parent.parent
+ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK]
+
+
+def is_pow2(p):
+    return p & (p - 1) == 0
+
+
+def test_library_exports_every_declared_symbol():
+    header = (ROOT / "include" / "sparbit.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(sparbit_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(binding.SYMBOLS), declared ^ set(binding.SYMBOLS)
+    lib = ctypes.CDLL(str(ROOT / "paper_2109_08751_b200" / "libsparbit_b200.so"))
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def as_set(msgs):
+    return {tuple(int(x) for x in m) for m in msgs}
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_descriptors_expand_to_oracle_message_sets(algo):
+    """Per phase, the library's messages equal the oracle's as a set (order inside a phase is free)."""
+    for P in list(range(1, 41)) + [64, 100, 127, 128, 129, 255, 256]:
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_RING and P > 64:
+            continue
+        plan = sp.Plan(P, 16, algo)
+        ref = oracle.Plan(algo, P)
+        assert plan.num_steps == ref.num_steps
+        assert plan.last_phase == ref.last_phase
+        for ph in range(-1, ref.last_phase + 1):
+            got = plan.messages(ph)
+            want = ref.phase_messages(ph)
+            assert len(got) == len(want), (algo, P, ph)
+            assert as_set(got) == as_set(want), (algo, P, ph)
+        plan.destroy()
+
+
+def test_sparbit_p1000_message_sets():
+    plan = sp.Plan(1000, 1024)
+    ref = oracle.Plan(oracle.SPARBIT, 1000)
+    for ph in range(-1, ref.last_phase + 1):
+        got = np.sort(plan.messages(ph), order=list(binding.MSG_DTYPE.names))
+        want = np.sort(ref.phase_messages(ph), order=list(oracle.MSG_DTYPE.names))
+        assert np.array_equal(got.view(np.int32), want.view(np.int32)), ph
+
+
+@pytest.mark.parametrize("P", [2, 5, 6, 8, 13, 21, 256, 1000])
+def test_step_info_matches_oracle_counts(P):
+    plan = sp.Plan(P, 64)
+    ref = oracle.Plan(oracle.SPARBIT, P)
+    K = plan.num_steps
+    held = 1
+    for s in range(K):
+        d, n, ig = plan.step_info(s)
+        assert d == 2 ** (K - 1 - s)
+        assert n == len(ref.phase_messages(s)) // P
+        assert ig == held - n          # what is withheld is what was held but not sent
+        held += n
+    assert held == P
+
+
+def test_plan_errors():
+    out = ctypes.c_void_p()
+    lib = binding.lib
+    assert lib.sparbit_plan_create(0, 16, 0, 0, ctypes.byref(out)) == sp.ERR_ARG
+    assert lib.sparbit_plan_create(-3, 16, 0, 0, ctypes.byref(out)) == sp.ERR_ARG
+    assert lib.sparbit_plan_create(8, 16, 9, 0, ctypes.byref(out)) == sp.ERR_ARG
+    assert lib.sparbit_plan_create(8, 16, 0, 17, ctypes.byref(out)) == sp.ERR_ARG
+    assert lib.sparbit_plan_create(8, 16, 0, 0, None) == sp.ERR_ARG
+    assert lib.sparbit_plan_create(6, 16, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create(13, 16, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create(1 << 20, 1 << 40, 0, 0, ctypes.byref(out)) == sp.ERR_OVERFLOW
+    assert lib.sparbit_plan_create((1 << 24) + 1, 1, 0, 0, ctypes.byref(out)) == sp.ERR_OVERFLOW
+    assert lib.sparbit_plan(0, 16) is None
+    assert lib.sparbit_plan_destroy(None) == sp.OK
+    assert lib.sparbit_plan_num_steps(None) == -1
+
+
+def test_argument_checks_happen_before_any_launch():
+    """These return on the host before the first CUDA call, so they work without a GPU."""
+    lib = binding.lib
+    plan = sp.Plan(8, 64)
+    h = plan._h
+    assert lib.sparbit_allgather(None, 1, 2, None) == sp.ERR_ARG
+    assert lib.sparbit_allgather(h, None, 4096, None) == sp.ERR_ARG
+    assert lib.sparbit_allgather(h, 4096, None, None) == sp.ERR_ARG
+    # send [4096, 4608) overlaps recv [4352, ...)
+    assert lib.sparbit_allgather(h, 4096, 4352, None) == sp.ERR_ALIAS
+    assert lib.sparbit_allgather_steps(h, 4096, 1 << 20, None, 2, 1) == sp.ERR_ARG
+    assert lib.sparbit_allgather_steps(h, 4096, 1 << 20, None, -2, 1) == sp.ERR_ARG
+    assert lib.sparbit_allgather_steps(h, 4096, 1 << 20, None, 0, 3) == sp.ERR_ARG
+    assert lib.sparbit_plan_step_info(h, 3, None, None, None) == sp.ERR_ARG
+    assert lib.sparbit_plan_set_copy_path(h, 7) == sp.ERR_ARG
+    # zero-byte blocks: a valid no-op, even with null buffers
+    z = sp.Plan(8, 0)
+    assert lib.sparbit_allgather(z._h, None, None, None) == sp.OK
+    # Bruck needs its workspace
+    b = sp.Plan(6, 64, sp.ALGO_BRUCK)
+    assert b.workspace_bytes == 6 * 6 * 64
+    assert lib.sparbit_allgather(b._h, 4096, 1 << 20, None) == sp.ERR_WORKSPACE
+    assert lib.sparbit_plan_set_workspace(b._h, 1 << 22, 100) == sp.ERR_WORKSPACE
+    assert lib.sparbit_plan_set_workspace(b._h, 1 << 20, 6 * 6 * 64) == sp.OK
+    assert lib.sparbit_allgather(b._h, 4096, 1 << 20, None) == sp.ERR_ALIAS   # workspace == recv
+    assert sp.Plan(8, 64).workspace_bytes == 0
+
+
+def test_strerror_covers_every_code():
+    texts = {binding.lib.sparbit_strerror(c).decode() for c in range(0, 9)}
+    assert len(texts) == 9 and "unknown error" not in texts
+    assert binding.lib.sparbit_strerror(99).decode() == "unknown error"
+
+
+def test_exec_mode_resolution():
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_CLUSTER           # latency-bound: one cluster
+    assert sp.Plan(256, 65536).exec_mode == sp.EXEC_PERSISTENT   # bandwidth-bound
+    assert sp.Plan(256, 65536, exec_mode=sp.EXEC_GRAPH).exec_mode == sp.EXEC_GRAPH
