@@ -144,6 +144,7 @@ int pick_vector_bytes(const sparbit_plan_s* p, const void* send, const void* rec
 uint64_t vec_tasks(const PhaseDesc& d, uint32_t P, int vbytes) {
     const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
     const uint64_t n_copies = (uint64_t)P * d.copies;
+    if (n_copies >> 32) return ~0ull;  // the kernels index copies with 32 bits
     if (vpc >= 32) {
         const uint64_t span = 32ull * kVecUnroll;
         return n_copies * ((vpc + span - 1) / span);
