@@ -53,7 +53,8 @@ enum {
     SPARBIT_ERR_WORKSPACE = 5,   /* Bruck without a workspace, or one that is too small */
     SPARBIT_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sparbit_last_cuda_error() */
     SPARBIT_ERR_TIMEOUT = 7,     /* the device-side grid barrier gave up waiting */
-    SPARBIT_ERR_NOMEM = 8        /* host allocation failed */
+    SPARBIT_ERR_NOMEM = 8,       /* host allocation failed */
+    SPARBIT_ERR_LIMIT = 9        /* larger than the fixed scratch of sparbit_allgather_noalloc */
 };
 
 /* Algorithms (paper, Section II-A and Section III).  Only Sparbit is the product's hot path; the
@@ -216,6 +217,43 @@ int sparbit_plan_status(sparbit_plan_t* plan, int* device_status);
  * hanging.
  */
 int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint64_t timeout_ns);
+
+/*
+ * sparbit_allgather_noalloc - the collective for callers that must not allocate device memory.
+ * (The paper has no counterpart for this entry point; it exists for the library's users.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - an application whose device
+ * memory is fully owned by its own pool or framework allocator, a plug-in that is handed
+ * buffers and a stream and nothing else, a service that may not take the driver's allocation
+ * lock once it is up.  sparbit_allgather keeps a small device-side scratch per plan (the
+ * per-phase descriptor table and the grid barrier's counter and status word) and obtains it with
+ * cudaMalloc on the plan's first launch; this entry point keeps the same scratch in a fixed
+ * 2 KiB array that is part of the library image, so it performs no cudaMalloc, cudaFree or any
+ * other allocating CUDA or framework call, at any time.  Every GPU that loads the library
+ * carries those 2 KiB until the process exits.  On the host it uses only short-lived ordinary
+ * heap memory for the schedule.
+ *
+ * It runs the persistent executor with the vector copy engine (the same kernel
+ * sparbit_allgather launches for EXEC_PERSISTENT / COPY_VECTOR), for algo = SPARBIT, RING or
+ * RECURSIVE_DOUBLING; sendbuf / recvbuf / stream as for sparbit_allgather.  Unlike
+ * sparbit_allgather it WAITS: the work is enqueued on `stream`, the stream is synchronised, and
+ * the return value is final - SPARBIT_OK, or SPARBIT_ERR_TIMEOUT if the grid barrier gave up
+ * (recvbuf is then incomplete).
+ *
+ * Limit: the array holds 28 phase descriptors, i.e. any Sparbit or recursive-doubling
+ * collective this library accepts (K + 1 <= 25 phases) and rings of at most 28 ranks.  Anything
+ * larger is refused with SPARBIT_ERR_LIMIT before anything is enqueued.  Bruck needs a
+ * P*P*m workspace and is refused with SPARBIT_ERR_UNSUPPORTED.
+ *
+ * The first call on each device looks up the array's device address (once per device, with that
+ * device current); make that first call before any stream capture begins.  All calls on a
+ * device share the one array, and it keeps what the previous call left: each call re-writes the
+ * descriptors and clears the barrier words on `stream` before its kernel.  Calls whose GPU work
+ * overlaps (two host threads on one device) race on the scratch: serialise them.
+ * Other errors: as for sparbit_plan_create and sparbit_allgather.
+ */
+int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* sendbuf, void* recvbuf,
+                              void* stream);
 
 const char* sparbit_strerror(int code);
 

@@ -13,7 +13,8 @@ import numpy as np
 _LIB_PATH = Path(__file__).resolve().parent / "libsparbit_b200.so"
 
 OK = 0
-ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = range(1, 9)
+ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT = \
+    range(1, 10)
 ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK = range(4)
 EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_CLUSTER = range(5)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
@@ -50,6 +51,7 @@ SYMBOLS = {
     "sparbit_plan_launch_counts": (_i, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
     "sparbit_plan_status": (_i, [_vp, _pi]),
     "sparbit_plan_set_barrier_test": (_i, [_vp, _i, _u64]),
+    "sparbit_allgather_noalloc": (_i, [_i, _sz, _i, _vp, _vp, _vp]),
     "sparbit_strerror": (ctypes.c_char_p, [_i]),
     "sparbit_last_cuda_error": (ctypes.c_char_p, []),
 }
@@ -200,3 +202,12 @@ def sparbit_plan(P: int, block_bytes: int) -> Plan:
 
 def sparbit_allgather(plan: Plan, sendbuf, recvbuf, stream=None) -> None:
     plan.allgather(sendbuf, recvbuf, stream)
+
+
+def sparbit_allgather_noalloc(P: int, block_bytes: int, sendbuf, recvbuf, stream=None,
+                              algo: int = ALGO_SPARBIT) -> None:
+    """The collective without any device allocation by the library (fixed 2 KiB scratch that is
+    part of the library image).  For callers whose device memory is managed elsewhere and who
+    must not trigger cudaMalloc.  Waits for completion.  Calls on one device must not overlap."""
+    _check(lib.sparbit_allgather_noalloc(P, block_bytes, algo, _ptr(sendbuf), _ptr(recvbuf),
+                                         _stream_handle(stream)), "sparbit_allgather_noalloc")

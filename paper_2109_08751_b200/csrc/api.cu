@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -663,10 +664,151 @@ const char* sparbit_strerror(int code) {
         case SPARBIT_ERR_CUDA: return "CUDA runtime error";
         case SPARBIT_ERR_TIMEOUT: return "device barrier timed out";
         case SPARBIT_ERR_NOMEM: return "out of host memory";
+        case SPARBIT_ERR_LIMIT: return "larger than the fixed scratch of sparbit_allgather_noalloc";
         default: return "unknown error";
     }
 }
 
 const char* sparbit_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"
+
+// ================================================================================================
+// Entry point that allocates no device memory.
+//
+// Some users of this library run where cudaMalloc is not an option: inside an application whose
+// device memory belongs to its own pool, as a plug-in that only receives buffers and a stream,
+// or in a loop that must stay clear of the driver's allocation lock.  For them the scratch the
+// persistent executor needs (descriptor table, barrier counter, status word) lives in the fixed
+// array below, which is part of the library image on every GPU that loads it.
+// ================================================================================================
+namespace {
+
+constexpr int kNoallocMaxPhases = 28;
+constexpr size_t kNoallocCtlBytes = 256;  // [0] barrier counter, [1] status word, rest unused
+constexpr size_t kNoallocBytes = kNoallocCtlBytes + kNoallocMaxPhases * sizeof(PhaseDesc);
+static_assert(sizeof(PhaseDesc) == 64, "descriptor size is part of the scratch budget");
+static_assert(kNoallocBytes == 2048, "the documented size of the fixed scratch");
+
+// Host code must never hand this name to a kernel: on the host it is only a stand-in for the
+// symbol.  The device address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocBytes];
+
+constexpr int kMaxDevices = 64;
+struct NoallocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;  // device address of g_noalloc_scratch on this device
+    int sm_count = 0;
+    int coop = 0;
+};
+NoallocDevice g_noalloc_dev[kMaxDevices];
+std::mutex g_noalloc_mutex;  // guards the once-per-device set-up only
+
+// once per device, with that device current
+int noalloc_setup(int device, NoallocDevice*& out) {
+    if (device < 0 || device >= kMaxDevices) return SPARBIT_ERR_ARG;
+    NoallocDevice& nd = g_noalloc_dev[device];
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!nd.ready) {
+        void* ptr = nullptr;
+        CU(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        CU(cudaDeviceGetAttribute(&nd.sm_count, cudaDevAttrMultiProcessorCount, device));
+        CU(cudaDeviceGetAttribute(&nd.coop, cudaDevAttrCooperativeLaunch, device));
+        nd.scratch = (unsigned char*)ptr;
+        // the array is zero when the module is loaded; clear it anyway so that the first call
+        // does not depend on that
+        CU(cudaMemset(nd.scratch, 0, kNoallocBytes));
+        nd.ready = true;
+    }
+    out = &nd;
+    return SPARBIT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* sendbuf, void* recvbuf,
+                              void* stream) {
+    if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;
+    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_ARG;
+    Schedule sched;
+    int rc;
+    try {
+        rc = map_sched_err(build_schedule(algo, P, (uint64_t)block_bytes, sched));
+    } catch (const std::bad_alloc&) {
+        rc = SPARBIT_ERR_NOMEM;
+    }
+    if (rc) return rc;
+    if (sched.phases.size() > (size_t)kNoallocMaxPhases) return SPARBIT_ERR_LIMIT;
+    const size_t send_bytes = (size_t)sched.P * sched.m;
+    const size_t recv_bytes = (size_t)sched.P * sched.P * sched.m;
+    if (send_bytes == 0) return SPARBIT_OK;
+    if (!sendbuf || !recvbuf) return SPARBIT_ERR_ARG;
+    if (ranges_overlap(sendbuf, send_bytes, recvbuf, recv_bytes)) return SPARBIT_ERR_ALIAS;
+
+    int device = -1;
+    CU(cudaGetDevice(&device));
+    NoallocDevice* nd = nullptr;
+    rc = noalloc_setup(device, nd);
+    if (rc) return rc;
+    if (!nd->coop) return SPARBIT_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // vector width from the alignment of the buffers and m (no workspace here)
+    uintptr_t bits = (uintptr_t)sendbuf | (uintptr_t)recvbuf | (uintptr_t)sched.m;
+    int vbytes = 16;
+    while (vbytes > 1 && (bits & (uintptr_t)(vbytes - 1))) vbytes >>= 1;
+
+    // grid: enough CTAs for the largest phase, at most what is co-resident
+    const int first = -1, last = sched.last_phase();
+    uint64_t need = 1;
+    for (int ph = first; ph <= last; ph++) {
+        const uint64_t tasks = vec_tasks(sched.phase(ph), sched.P, vbytes);
+        if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
+        const uint64_t t = (tasks + kVecBlock / 32 - 1) / (kVecBlock / 32);
+        if (t > need) need = t;
+    }
+    const void* fn = pick_persistent_vec(vbytes);
+    int per_sm = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kVecBlock, 0));
+    if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "persistent kernel does not fit on an SM");
+    uint64_t grid = (uint64_t)per_sm * nd->sm_count;
+    if (grid > need) grid = need;
+
+    unsigned* ctl_words = (unsigned*)nd->scratch;
+    PhaseDesc* d_descs = (PhaseDesc*)(nd->scratch + kNoallocCtlBytes);
+
+    // every call starts from a clean scratch: barrier counter and status word at zero, this
+    // collective's descriptors in the table (the call waits below, so the host copy outlives it)
+    CU(cudaMemsetAsync(ctl_words, 0, kNoallocCtlBytes, st));
+    const size_t n = sched.phases.size();
+    CU(cudaMemcpyAsync(d_descs, sched.phases.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice, st));
+
+    Geom g;
+    memset(&g, 0, sizeof g);
+    g.P = sched.P;
+    g.m = sched.m;
+    g.base[SPACE_SEND] = (char*)const_cast<void*>(sendbuf);
+    g.base[SPACE_RECV] = (char*)recvbuf;
+    g.base[SPACE_WORK] = nullptr;
+    g.rank_pitch[SPACE_SEND] = g.m;
+    g.rank_pitch[SPACE_RECV] = (uint64_t)g.P * g.m;
+    g.rank_pitch[SPACE_WORK] = (uint64_t)g.P * g.m;
+    BarrierCtl ctl;
+    ctl.counter = ctl_words;
+    ctl.status = ctl_words + 1;
+    ctl.base = 0;
+    ctl.expected = (unsigned)grid;
+    ctl.timeout_ns = kDefaultTimeoutNs;
+    int first_idx = first + 1, last_idx = last + 1;
+    const PhaseDesc* descs = d_descs;
+    void* args[] = {&g, &descs, &first_idx, &last_idx, &ctl};
+    CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(kVecBlock), args, 0, st));
+    unsigned words[2] = {0, 0};
+    CU(cudaMemcpyAsync(words, ctl_words, sizeof words, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return words[1] == DEV_OK ? SPARBIT_OK : SPARBIT_ERR_TIMEOUT;
+}
 
 }  // extern "C"

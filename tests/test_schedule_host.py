@@ -125,8 +125,8 @@ def test_argument_checks_happen_before_any_launch():
 
 
 def test_strerror_covers_every_code():
-    texts = {binding.lib.sparbit_strerror(c).decode() for c in range(0, 9)}
-    assert len(texts) == 9 and "unknown error" not in texts
+    texts = {binding.lib.sparbit_strerror(c).decode() for c in range(0, 10)}
+    assert len(texts) == 10 and "unknown error" not in texts
     assert binding.lib.sparbit_strerror(99).decode() == "unknown error"
 
 

@@ -1,0 +1,68 @@
+"""The entry point that allocates no device memory, against the regular one.
+
+`sparbit_allgather_noalloc` serves callers that cannot call cudaMalloc (device memory owned by
+their own pool or framework, plug-ins that only get buffers and a stream): its scratch is a fixed
+2 KiB array inside the library image instead of a per-plan allocation.  It must produce exactly
+what `sparbit_allgather` produces.  Because every call shares that one array and it keeps the
+previous call's contents, the check is made on two calls in a row with different sizes and data.
+
+This file sorts last on purpose: a run that stops at the first failure has then already run
+every other test.  It passes alone in a fresh process as well as after the others.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+import paper_2109_08751_b200 as sp
+from paper_2109_08751_b200 import binding
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def regular(P, m, algo, send, dev):
+    """Result of the existing entry point with the same executor and copy engine."""
+    plan = sp.Plan(P, m, algo, sp.EXEC_PERSISTENT)
+    plan.set_copy_path(sp.COPY_VECTOR)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    plan.destroy()
+    return recv
+
+
+def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    # two different collectives back to back: the second finds the first one's descriptors and
+    # barrier words in the shared scratch and must not be disturbed by them
+    cases = [(13, 4096, sp.ALGO_SPARBIT, 11), (64, 1040, sp.ALGO_SPARBIT, 12),
+             (16, 272, sp.ALGO_RECURSIVE_DOUBLING, 13), (9, 100, sp.ALGO_RING, 14)]
+    stream = torch.cuda.Stream(device=dev)
+    for P, m, algo, seed in cases:
+        for call in range(2):
+            host_send = si.send_blocks(P, m, seed + 100 * call)
+            send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+            got = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+            torch.cuda.synchronize(dev)
+            binding.sparbit_allgather_noalloc(P, m, send, got, stream, algo=algo)
+            want = regular(P, m, algo, send, dev)
+            assert torch.equal(got, want), (P, m, algo, call)          # bit-exact, as everywhere
+            assert torch.equal(got.view(P, P * m)[P - 1], send)         # and it is the allgather
+
+
+def test_noalloc_refuses_what_does_not_fit_its_scratch():
+    lib = binding.lib
+    # host-side checks: nothing is enqueued, the pointers are never touched
+    assert lib.sparbit_allgather_noalloc(64, 16, sp.ALGO_RING, 4096, 1 << 20, None) == sp.ERR_LIMIT
+    assert lib.sparbit_allgather_noalloc(8, 16, sp.ALGO_BRUCK, 4096, 1 << 20, None) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_allgather_noalloc(6, 16, sp.ALGO_RECURSIVE_DOUBLING, 4096, 1 << 20, None) \
+        == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_allgather_noalloc(0, 16, sp.ALGO_SPARBIT, 4096, 1 << 20, None) == sp.ERR_ARG
+    assert lib.sparbit_allgather_noalloc(8, 16, sp.ALGO_SPARBIT, 4096, 4100, None) == sp.ERR_ALIAS
+    assert lib.sparbit_allgather_noalloc(8, 0, sp.ALGO_SPARBIT, None, None, None) == sp.OK
+    assert "scratch" in lib.sparbit_strerror(sp.ERR_LIMIT).decode()
