@@ -337,6 +337,76 @@ def run_ours(args):
     return 0
 
 
+# ------------------------------------------------------------------------------------------------
+def run_sweep(args):
+    """Latency and bandwidth curves: every point timed with the paper's protocol (5 warm-ups, 50
+    timed collectives, min / avg / max), one JSON line per (algorithm, executor, engine, P, m)."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peak()
+    points = []
+    if args.sweep in ("config4", "all"):
+        points += [(1000, 1024, ["sparbit"])]
+    if args.sweep in ("config5", "all"):
+        points += [(256, m, ["sparbit", "ring", "rd", "bruck"])
+                   for m in (8, 64, 512, 4096, 32768, 65536, 262144)]
+    if args.sweep == "config3":
+        points += [(128, 65536, ["sparbit"])]
+    algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
+             "bruck": sp.ALGO_BRUCK}
+    execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
+             "cluster": sp.EXEC_CLUSTER}
+    copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
+    stream = torch.cuda.Stream(device=dev)
+    for P, m, names in points:
+        sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        work = None
+        for name in names:
+            if name == "bruck" and work is None:
+                work = torch.empty(P * P * m, dtype=torch.uint8, device=dev)
+            for ename, e in execs.items():
+                if ename == "cluster" and effective_bytes(P, m) > (64 << 20):
+                    continue
+                if ename == "stream" and name == "ring" and m >= 32768:
+                    continue  # same kernels as the graph chain; skipped to bound the sweep
+                for cname, c in copies.items():
+                    if cname == "bulk" and (m % 16 or ename == "cluster"):
+                        continue
+                    plan = sp.Plan(P, m, algos[name], e)
+                    plan.set_copy_path(c)
+                    if name == "bruck":
+                        plan.set_workspace(work, P * P * m)
+                    with torch.cuda.stream(stream):
+                        for it in range(5):
+                            plan.allgather(sends[it & 1], recv, stream)
+                        stream.synchronize()
+                        ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
+                        ev[0].record(stream)
+                        for it in range(50):
+                            plan.allgather(sends[it & 1], recv, stream)
+                            ev[it + 1].record(stream)
+                        stream.synchronize()
+                    assert plan.status() == sp.OK
+                    ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
+                    us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(50)]
+                    avg = float(np.mean(us))
+                    print(json.dumps({
+                        "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
+                        "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
+                        "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
+                        "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
+                        "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
+                        "checked": ok}), flush=True)
+                    plan.destroy()
+        del sends, recv, work
+        torch.cuda.empty_cache()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,7 +421,11 @@ def main():
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--sweep", choices=["config3", "config4", "config5", "all"], default=None,
+                    help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":

@@ -38,10 +38,11 @@ struct GraphKey {
     void* work = nullptr;
     int first = 0, last = -2;
     int path = 0, vec = 0;
-    bool operator==(const GraphKey& o) const {
-        return send == o.send && recv == o.recv && work == o.work && first == o.first && last == o.last &&
-               path == o.path && vec == o.vec;
+    unsigned long long timeout_ns = 0;
+    bool same_shape(const GraphKey& o) const {
+        return first == o.first && last == o.last && path == o.path && vec == o.vec && timeout_ns == o.timeout_ns;
     }
+    bool same_buffers(const GraphKey& o) const { return send == o.send && recv == o.recv && work == o.work; }
 };
 
 }  // namespace
@@ -68,13 +69,16 @@ struct sparbit_plan_s {
     unsigned long long timeout_ns = kDefaultTimeoutNs;
 
     // bulk engine geometry
-    uint32_t bulk_warps = 2;
-    uint32_t bulk_stage_bytes = 14336;
+    // measured on B200: about 32 KiB of loads in flight per SM is the sweet spot for a copy (more
+    // lowers the achieved HBM bandwidth): 4 rings x 2 loads x 4 KiB
+    uint32_t bulk_warps = 4;
+    uint32_t bulk_stage_bytes = 4096;
 
     // cached graph
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t gexec = nullptr;
     GraphKey gkey;
+    std::vector<cudaGraphNode_t> gnodes;  // one kernel node per phase of the cached chain
 
     // host-buffer entry point
     void* stage_send = nullptr;
@@ -194,13 +198,17 @@ const void* pick_cluster_vec(int vbytes) {
     }
 }
 
-// executor for SPARBIT_EXEC_AUTO: collectives that move little are latency-bound and run inside
-// one thread-block cluster; everything else runs in the persistent cooperative kernel
+// executor for SPARBIT_EXEC_AUTO, from the measured P = 256 and P = 1000 sweeps: below about
+// 1 GB moved a collective is bound by the per-phase cost, where the CUDA-graph chain (about 3 us
+// per phase, grids sized per phase) beats the grid barrier of the persistent kernel (about 3.6 us
+// with all CTAs taking part in every barrier); above it the two are within 1 % and the persistent
+// kernel is used (one launch, no graph to re-parameterise when buffers change).
 int auto_exec(const Schedule& s, bool coop, bool cluster_ok) {
+    (void)cluster_ok;
     const uint64_t P = s.P;
     const unsigned __int128 moved = (unsigned __int128)2 * P * (P - 1) * s.m;
-    if (cluster_ok && moved <= (8u << 20) && s.algo != ALGO_RING) return SPARBIT_EXEC_CLUSTER;
-    return coop ? SPARBIT_EXEC_PERSISTENT : SPARBIT_EXEC_GRAPH;
+    if (!coop || moved < ((unsigned __int128)1 << 30)) return SPARBIT_EXEC_GRAPH;
+    return SPARBIT_EXEC_PERSISTENT;
 }
 
 struct Resolved {
@@ -215,7 +223,11 @@ Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv) {
     const uint64_t m = p->sched.m;
     const bool bulk_possible = r.vbytes == 16;
     int copy = p->copy_req;
-    if (copy == SPARBIT_COPY_AUTO) copy = (bulk_possible && m >= 4096) ? SPARBIT_COPY_BULK : SPARBIT_COPY_VECTOR;
+    // measured on B200 (P = 256 sweep): with about 32 KiB of loads in flight per SM both engines
+    // reach the copy peak for blocks >= 32 KiB, the bulk engine a little ahead; below that the
+    // per-operation cost of a bulk copy shows and the vector engine wins
+    if (copy == SPARBIT_COPY_AUTO)
+        copy = (bulk_possible && m >= (32u << 10)) ? SPARBIT_COPY_BULK : SPARBIT_COPY_VECTOR;
     if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
     r.copy = copy;
     int exec = p->exec_req;
@@ -266,7 +278,7 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
         const uint64_t wpb = kVecBlock / 32;
         uint64_t ctas = (tasks + wpb - 1) / wpb;
-        const uint64_t cap = (uint64_t)p->sm_count * 4;  // 2048 threads per SM
+        const uint64_t cap = (uint64_t)p->sm_count * 2;  // 1024 threads x 2 vectors in flight per SM
         if (ctas > cap) ctas = cap;
         if (ctas < 1) ctas = 1;
         pl.fn = pick_phase_vec(rs.vbytes);
@@ -318,6 +330,7 @@ void drop_graph(sparbit_plan_s* p) {
     if (p->graph) cudaGraphDestroy(p->graph);
     p->gexec = nullptr;
     p->graph = nullptr;
+    p->gnodes.clear();
     p->gkey = GraphKey();
 }
 
@@ -330,10 +343,16 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     key.last = last;
     key.path = rs.copy;
     key.vec = rs.vbytes;
-    if (!p->gexec || !(p->gkey == key)) {
-        // (re)build the chain: one kernel node per phase, each depending on the one before
-        drop_graph(p);
-        CU(cudaGraphCreate(&p->graph, 0));
+    key.timeout_ns = p->timeout_ns;
+    const bool rebuild = !p->gexec || !p->gkey.same_shape(key);
+    if (rebuild || !p->gkey.same_buffers(key)) {
+        // The chain is one kernel node per phase, each depending on the one before.  A change of
+        // buffers only rewrites the nodes' parameters in the instantiated graph; anything else
+        // builds and instantiates the chain again.
+        if (rebuild) {
+            drop_graph(p);
+            CU(cudaGraphCreate(&p->graph, 0));
+        }
         cudaGraphNode_t prev = nullptr;
         for (int ph = first; ph <= last; ph++) {
             PhaseArgs a;
@@ -353,11 +372,16 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
             np.blockDim = pl.block;
             np.sharedMemBytes = (unsigned)pl.smem;
             np.kernelParams = a.ptrs;
-            cudaGraphNode_t node;
-            CU(cudaGraphAddKernelNode(&node, p->graph, prev ? &prev : nullptr, prev ? 1 : 0, &np));
-            prev = node;
+            if (rebuild) {
+                cudaGraphNode_t node;
+                CU(cudaGraphAddKernelNode(&node, p->graph, prev ? &prev : nullptr, prev ? 1 : 0, &np));
+                p->gnodes.push_back(node);
+                prev = node;
+            } else {
+                CU(cudaGraphExecKernelNodeSetParams(p->gexec, p->gnodes[(size_t)(ph - first)], &np));
+            }
         }
-        CU(cudaGraphInstantiate(&p->gexec, p->graph, 0));
+        if (rebuild) CU(cudaGraphInstantiate(&p->gexec, p->graph, 0));
         p->gkey = key;
     }
     CU(cudaGraphLaunch(p->gexec, st));
@@ -394,6 +418,8 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     }
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, (int)block.x, smem));
     if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "persistent kernel does not fit on an SM");
+    // one CTA of rings per SM keeps the loads in flight at the measured sweet spot; more would fit
+    if (rs.copy == SPARBIT_COPY_BULK) per_sm = 1;
     uint64_t grid = (uint64_t)per_sm * p->sm_count;
     if (grid > need) grid = need;
     BarrierCtl ctl;

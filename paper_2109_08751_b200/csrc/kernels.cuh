@@ -40,9 +40,21 @@ struct BulkCfg {
     uint32_t pad_;
 };
 
-constexpr int kBulkStages = 8;     // stages per ring
-constexpr int kBulkLoadsAhead = 4; // loads in flight per ring; the rest hold pending stores
-constexpr int kVecUnroll = 4;      // vectors per lane per warp task
+#ifndef SPB_BULK_STAGES
+#define SPB_BULK_STAGES 4
+#endif
+#ifndef SPB_BULK_LOADS
+#define SPB_BULK_LOADS 2
+#endif
+constexpr int kBulkStages = SPB_BULK_STAGES;     // stages per ring
+constexpr int kBulkLoadsAhead = SPB_BULK_LOADS;  // loads in flight per ring; the rest hold pending stores
+#ifndef SPB_VEC_UNROLL
+#define SPB_VEC_UNROLL 2
+#endif
+#ifndef SPB_PERSIST_MIN_CTAS
+#define SPB_PERSIST_MIN_CTAS 2
+#endif
+constexpr int kVecUnroll = SPB_VEC_UNROLL;  // vectors per lane per warp task
 
 // ------------------------------------------------------------------------------------------------
 // small PTX helpers
@@ -350,7 +362,7 @@ __device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& ep
 // ------------------------------------------------------------------------------------------------
 // one phase, vector engine
 template <typename V>
-__global__ void __launch_bounds__(512) phase_vec_kernel(Geom g, PhaseDesc d) {
+__global__ void __launch_bounds__(512, 2) phase_vec_kernel(Geom g, PhaseDesc d) {
     const uint32_t wpb = blockDim.x >> 5;
     vec_phase<V>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
 }
@@ -386,19 +398,32 @@ __global__ void __launch_bounds__(256) phase_bulk_kernel(Geom g, PhaseDesc d, ui
     }
 }
 
+// Descriptors of a multi-phase kernel live in shared memory, double-buffered: the next phase's
+// descriptor is fetched while the current phase runs, so no phase starts with a global load on
+// its critical path, and the copy loops need no registers to hold it.
+__device__ __forceinline__ void fetch_desc(PhaseDesc* dst, const PhaseDesc* __restrict__ src) {
+    static_assert(sizeof(PhaseDesc) == 64, "PhaseDesc is copied as 16 words");
+    if (threadIdx.x < 16)
+        reinterpret_cast<uint32_t*>(dst)[threadIdx.x] = reinterpret_cast<const uint32_t*>(src)[threadIdx.x];
+}
+
 // phases first..last (indices into descs), vector engine, grid barrier between phases
 template <typename V>
-__global__ void __launch_bounds__(512) persistent_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
-                                                             int last, BarrierCtl ctl) {
+__global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs,
+                                                                int first, int last, BarrierCtl ctl) {
     __shared__ int flag;
+    __shared__ PhaseDesc sd[2];
     if (ld_relaxed_gpu(ctl.status) != DEV_OK) return;  // an earlier failure was not cleared yet
     const uint32_t wpb = blockDim.x >> 5;
     const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * wpb;
     unsigned epoch = 0;
+    fetch_desc(&sd[0], &descs[first]);
+    __syncthreads();
     for (int ph = first; ph <= last; ph++) {
-        const PhaseDesc d = descs[ph];
-        vec_phase<V>(g, d, warp_id, n_warps, threadIdx.x & 31u);
+        const int cur = (ph - first) & 1;
+        if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
+        vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
         if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
     }
 }
@@ -408,6 +433,7 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
                                                               int last, uint32_t stage_bytes, BarrierCtl ctl) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int flag;
+    __shared__ PhaseDesc sd[2];
     if (ld_relaxed_gpu(ctl.status) != DEV_OK) return;
     const uint32_t warps = blockDim.x >> 5;
     const uint32_t warp = threadIdx.x >> 5;
@@ -415,12 +441,14 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
     BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
     if (driver) init_pipe(pp);
     unsigned epoch = 0;
+    fetch_desc(&sd[0], &descs[first]);
+    __syncthreads();
     for (int ph = first; ph <= last; ph++) {
-        if (driver) {
-            const PhaseDesc d = descs[ph];
-            bulk_phase(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
+        const int cur = (ph - first) & 1;
+        if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
+        if (driver)
+            bulk_phase(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
                        ctl.timeout_ns);
-        }
         if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
     }
 }
@@ -431,13 +459,18 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
 template <typename V>
 __global__ void __launch_bounds__(512) cluster_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
                                                            int last) {
+    __shared__ PhaseDesc sd[2];
     const uint32_t wpb = blockDim.x >> 5;
     const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * wpb;
+    fetch_desc(&sd[0], &descs[first]);
+    __syncthreads();
     for (int ph = first; ph <= last; ph++) {
-        const PhaseDesc d = descs[ph];
-        vec_phase<V>(g, d, warp_id, n_warps, threadIdx.x & 31u);
+        const int cur = (ph - first) & 1;
+        if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
+        vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
         if (ph != last) {
+            // the cluster barrier also orders this CTA's shared-memory descriptor fetch
             asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
             asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         }
