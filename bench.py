@@ -39,7 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (bytes; None = not captured for this workload)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/persistent_bulk_kernel_P256_m64k_traffic.md: 4.16 GB read + 4.25 GB written
+    "sparbit:P256:m65536:persistent:bulk": 8.41e9,
+}
 
 
 def effective_bytes(P: int, m: int) -> int:
