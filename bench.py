@@ -115,6 +115,22 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x: float, device, use_dist: bool) -> float:
+    """Largest value of x over all ranks (device timings are reported as the slowest rank's)."""
+    if not use_dist:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, P: int, m: int, ms_per_step: float) -> float:
+    """Effective GB/s of `world` independent replicas that all finish within ms_per_step."""
+    return world * effective_bytes(P, m) / (ms_per_step * 1e-3) / 1e9
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -268,12 +284,9 @@ def run_ours(args):
     view = recv.view(P, P * m)
     checked = all(bool(torch.equal(view[r], last_send)) for r in (0, P // 3, P - 1))
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if use_dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    max_total_ms = float(t.item())
+    max_total_ms = max_over_ranks(total_ms, dev, use_dist)
     ms_per_step = max_total_ms / args.steps
-    value = world * effective_bytes(P, m) / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(world, P, m, ms_per_step)
 
     # end to end through the host-buffer entry point (pinned host memory; H2D + D2H inside)
     e2e = None
@@ -290,12 +303,9 @@ def run_ours(args):
             hplan.allgather_host(hs.numpy(), hr.numpy())
         torch.cuda.synchronize(dev)
         dt = (time.perf_counter() - t0) / e2e_steps
-        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if use_dist:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dt = float(tt.item())
+        dt = max_over_ranks(dt, dev, use_dist)
         ok = bool(np.array_equal(hr.numpy()[(P - 1) * P * m:], hs.numpy()))
-        e2e = {"value": world * effective_bytes(P, m) / dt / 1e9, "unit": UNIT, "ms_per_step": dt * 1e3,
+        e2e = {"value": whole_job_value(world, P, m, dt * 1e3), "unit": UNIT, "ms_per_step": dt * 1e3,
                "h2d_bytes_per_step": P * m, "d2h_bytes_per_step": P * P * m, "steps": e2e_steps,
                "checked": ok}
         hplan.destroy()
