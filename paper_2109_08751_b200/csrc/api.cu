@@ -74,11 +74,16 @@ struct sparbit_plan_s {
     uint32_t bulk_warps = 4;
     uint32_t bulk_stage_bytes = 4096;
 
-    // cached graph
-    cudaGraph_t graph = nullptr;
-    cudaGraphExec_t gexec = nullptr;
-    GraphKey gkey;
-    std::vector<cudaGraphNode_t> gnodes;  // one kernel node per phase of the cached chain
+    // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
+    // that callers alternating between buffer sets never re-instantiate
+    struct GraphEntry {
+        GraphKey key;
+        cudaGraphExec_t exec = nullptr;
+        uint64_t stamp = 0;
+    };
+    std::vector<GraphEntry> gcache;
+    uint64_t gstamp = 0;
+    cudaStream_t capture_stream = nullptr;
 
     // host-buffer entry point
     void* stage_send = nullptr;
@@ -198,17 +203,17 @@ const void* pick_cluster_vec(int vbytes) {
     }
 }
 
-// executor for SPARBIT_EXEC_AUTO, from the measured P = 256 and P = 1000 sweeps: below about
-// 1 GB moved a collective is bound by the per-phase cost, where the CUDA-graph chain (about 3 us
-// per phase, grids sized per phase) beats the grid barrier of the persistent kernel (about 3.6 us
-// with all CTAs taking part in every barrier); above it the two are within 1 % and the persistent
-// kernel is used (one launch, no graph to re-parameterise when buffers change).
+// Executor for SPARBIT_EXEC_AUTO, from the measured P = 256 and P = 1000 sweeps on B200: the
+// CUDA-graph chain of per-phase kernels (programmatic dependent launch between phases, grids sized
+// per phase) is the fastest or within noise at every block size - about 2.7 us per phase in the
+// latency regime against 3.7 us for the grid barrier of the persistent kernel, and 1-2 % ahead
+// at 64 KiB blocks.  The persistent kernel stays available (SPARBIT_EXEC_PERSISTENT) and is what
+// sparbit_allgather_noalloc runs.
 int auto_exec(const Schedule& s, bool coop, bool cluster_ok) {
+    (void)s;
+    (void)coop;
     (void)cluster_ok;
-    const uint64_t P = s.P;
-    const unsigned __int128 moved = (unsigned __int128)2 * P * (P - 1) * s.m;
-    if (!coop || moved < ((unsigned __int128)1 << 30)) return SPARBIT_EXEC_GRAPH;
-    return SPARBIT_EXEC_PERSISTENT;
+    return SPARBIT_EXEC_GRAPH;
 }
 
 struct Resolved {
@@ -307,6 +312,11 @@ struct PhaseArgs {
     }
 };
 
+// One kernel per phase on `st`.  Consecutive phases are launched with programmatic stream
+// serialisation: a phase kernel lets its successor start launching at once
+// (griddepcontrol.launch_dependents) and itself waits for its predecessor to complete and flush
+// (griddepcontrol.wait) before it touches memory, so the launch latency of phase i+1 hides behind
+// phase i while the Waitall between phases stays intact.
 int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     for (int ph = first; ph <= last; ph++) {
         PhaseArgs a;
@@ -319,20 +329,30 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         PhaseLaunch pl;
         int rc = plan_phase_launch(p, rs, a.d, pl);
         if (rc) return rc;
-        CU(cudaLaunchKernel(pl.fn, pl.grid, pl.block, a.ptrs, pl.smem, st));
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = pl.grid;
+        cfg.blockDim = pl.block;
+        cfg.dynamicSmemBytes = pl.smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        CU(cudaLaunchKernelExC(&cfg, pl.fn, a.ptrs));
         p->kernel_launches++;
     }
     return SPARBIT_OK;
 }
 
 void drop_graph(sparbit_plan_s* p) {
-    if (p->gexec) cudaGraphExecDestroy(p->gexec);
-    if (p->graph) cudaGraphDestroy(p->graph);
-    p->gexec = nullptr;
-    p->graph = nullptr;
-    p->gnodes.clear();
-    p->gkey = GraphKey();
+    for (auto& e : p->gcache)
+        if (e.exec) cudaGraphExecDestroy(e.exec);
+    p->gcache.clear();
 }
+
+constexpr size_t kGraphCacheEntries = 4;
 
 int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     GraphKey key;
@@ -344,47 +364,57 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     key.path = rs.copy;
     key.vec = rs.vbytes;
     key.timeout_ns = p->timeout_ns;
-    const bool rebuild = !p->gexec || !p->gkey.same_shape(key);
-    if (rebuild || !p->gkey.same_buffers(key)) {
-        // The chain is one kernel node per phase, each depending on the one before.  A change of
-        // buffers only rewrites the nodes' parameters in the instantiated graph; anything else
-        // builds and instantiates the chain again.
-        if (rebuild) {
-            drop_graph(p);
-            CU(cudaGraphCreate(&p->graph, 0));
+    sparbit_plan_s::GraphEntry* hit = nullptr;
+    for (auto& e : p->gcache)
+        if (e.key.same_shape(key) && e.key.same_buffers(key)) hit = &e;
+    if (!hit) {
+        // capture the chain of per-phase launches (programmatic edges included) into a graph
+        if (!p->capture_stream) CU(cudaStreamCreateWithFlags(&p->capture_stream, cudaStreamNonBlocking));
+        const uint64_t launches_before = p->kernel_launches;
+        CU(cudaStreamBeginCapture(p->capture_stream, cudaStreamCaptureModeThreadLocal));
+        int rc = launch_stream(p, rs, g, first, last, p->capture_stream);
+        cudaGraph_t graph = nullptr;
+        cudaError_t ce = cudaStreamEndCapture(p->capture_stream, &graph);
+        p->kernel_launches = launches_before;  // captured, not launched
+        if (rc) {
+            if (graph) cudaGraphDestroy(graph);
+            return rc;
         }
-        cudaGraphNode_t prev = nullptr;
-        for (int ph = first; ph <= last; ph++) {
-            PhaseArgs a;
-            a.g = g;
-            a.d = p->sched.phase(ph);
-            a.stage_bytes = p->bulk_stage_bytes;
-            a.status = p->d_ctl + 1;
-            a.timeout_ns = p->timeout_ns;
-            a.fill(rs.copy == SPARBIT_COPY_BULK);
-            PhaseLaunch pl;
-            int rc = plan_phase_launch(p, rs, a.d, pl);
-            if (rc) return rc;
-            cudaKernelNodeParams np;
-            memset(&np, 0, sizeof np);
-            np.func = const_cast<void*>(pl.fn);
-            np.gridDim = pl.grid;
-            np.blockDim = pl.block;
-            np.sharedMemBytes = (unsigned)pl.smem;
-            np.kernelParams = a.ptrs;
-            if (rebuild) {
-                cudaGraphNode_t node;
-                CU(cudaGraphAddKernelNode(&node, p->graph, prev ? &prev : nullptr, prev ? 1 : 0, &np));
-                p->gnodes.push_back(node);
-                prev = node;
-            } else {
-                CU(cudaGraphExecKernelNodeSetParams(p->gexec, p->gnodes[(size_t)(ph - first)], &np));
+        if (ce != cudaSuccess) return cuda_fail(ce, "cudaStreamEndCapture");
+        if (p->gcache.size() < kGraphCacheEntries) {
+            p->gcache.emplace_back();
+            hit = &p->gcache.back();
+        } else {
+            // recycle the least recently used entry: same topology -> update it in place
+            hit = &p->gcache[0];
+            for (auto& e : p->gcache)
+                if (e.stamp < hit->stamp) hit = &e;
+            if (hit->exec && hit->key.same_shape(key)) {
+                cudaGraphExecUpdateResultInfo info;
+                if (cudaGraphExecUpdate(hit->exec, graph, &info) != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    cudaGraphExecDestroy(hit->exec);
+                    hit->exec = nullptr;
+                }
+            } else if (hit->exec) {
+                cudaGraphExecDestroy(hit->exec);
+                hit->exec = nullptr;
             }
         }
-        if (rebuild) CU(cudaGraphInstantiate(&p->gexec, p->graph, 0));
-        p->gkey = key;
+        if (!hit->exec) {
+            cudaError_t ie = cudaGraphInstantiate(&hit->exec, graph, 0);
+            if (ie != cudaSuccess) {
+                cudaGraphDestroy(graph);
+                hit->exec = nullptr;
+                hit->key = GraphKey();
+                return cuda_fail(ie, "cudaGraphInstantiate");
+            }
+        }
+        cudaGraphDestroy(graph);
+        hit->key = key;
     }
-    CU(cudaGraphLaunch(p->gexec, st));
+    hit->stamp = ++p->gstamp;
+    CU(cudaGraphLaunch(hit->exec, st));
     p->graph_launches++;
     p->kernel_launches += (uint64_t)(last - first + 1);
     return SPARBIT_OK;
@@ -545,6 +575,7 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
     if (p->dev_ready) {
         if (p->launched && cudaDeviceSynchronize() != cudaSuccess) rc = SPARBIT_ERR_CUDA;
         drop_graph(p);
+        if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
         cudaFree(p->d_descs);
         cudaFree(p->d_ctl);
         cudaFree(p->stage_send);
