@@ -108,7 +108,7 @@ int map_sched_err(int e) {
 }
 
 size_t bulk_smem_bytes(const sparbit_plan_s* p) {
-    return (size_t)p->bulk_warps * kBulkStages * (p->bulk_stage_bytes + 8 + 16);
+    return (size_t)p->bulk_warps * kBulkStages * (p->bulk_stage_bytes + 8 + 32);
 }
 
 int ensure_device(sparbit_plan_s* p) {
@@ -122,9 +122,16 @@ int ensure_device(sparbit_plan_s* p) {
     p->cluster_ok = cc_major >= 9;
     // shrink the bulk ring if this device offers less shared memory than planned
     while (bulk_smem_bytes(p) > (size_t)p->max_smem_optin && p->bulk_stage_bytes > 1024) p->bulk_stage_bytes -= 1024;
-    const size_t n = p->sched.phases.size();
+    // descriptor table: the phases in order, then (if the schedule has one) the same sequence with
+    // phases -1 and 0 replaced by the fused first pass
+    std::vector<PhaseDesc> table = p->sched.phases;
+    if (p->sched.has_fused_first) {
+        table.push_back(p->sched.fused_first);
+        table.insert(table.end(), p->sched.phases.begin() + 2, p->sched.phases.end());
+    }
+    const size_t n = table.size();
     CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
-    CU(cudaMemcpy(p->d_descs, p->sched.phases.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(p->d_descs, table.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
     CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
     CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -260,6 +267,33 @@ Geom make_geom(const sparbit_plan_s* p, const void* send, void* recv) {
     return g;
 }
 
+// What a call that asks for phases first..last executes: the phases one by one, or, when it asks
+// for both phase -1 and phase 0 and the schedule allows it, the fused first pass followed by
+// phases 1..last.
+struct ExecSeq {
+    const Schedule* s;
+    bool fused;
+    int first, last;
+    int count() const { return last - first + 1 - (fused ? 1 : 0); }
+    const PhaseDesc& item(int i) const {
+        if (!fused) return s->phase(first + i);
+        return i == 0 ? s->fused_first : s->phase(i);
+    }
+    // position in the device table (see ensure_device)
+    size_t table_index(int i) const {
+        return fused ? s->phases.size() + (size_t)i : (size_t)(first + 1 + i);
+    }
+};
+
+ExecSeq make_seq(const sparbit_plan_s* p, int first, int last) {
+    ExecSeq q;
+    q.s = &p->sched;
+    q.first = first;
+    q.last = last;
+    q.fused = first == -1 && last >= 0 && p->sched.has_fused_first;
+    return q;
+}
+
 // launch geometry of one phase as its own kernel
 struct PhaseLaunch {
     const void* fn;
@@ -318,10 +352,11 @@ struct PhaseArgs {
 // (griddepcontrol.wait) before it touches memory, so the launch latency of phase i+1 hides behind
 // phase i while the Waitall between phases stays intact.
 int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
-    for (int ph = first; ph <= last; ph++) {
+    const ExecSeq seq = make_seq(p, first, last);
+    for (int i = 0; i < seq.count(); i++) {
         PhaseArgs a;
         a.g = g;
-        a.d = p->sched.phase(ph);
+        a.d = seq.item(i);
         a.stage_bytes = p->bulk_stage_bytes;
         a.status = p->d_ctl + 1;
         a.timeout_ns = p->timeout_ns;
@@ -416,12 +451,13 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     hit->stamp = ++p->gstamp;
     CU(cudaGraphLaunch(hit->exec, st));
     p->graph_launches++;
-    p->kernel_launches += (uint64_t)(last - first + 1);
+    p->kernel_launches += (uint64_t)make_seq(p, first, last).count();
     return SPARBIT_OK;
 }
 
 int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
+    const ExecSeq seq = make_seq(p, first, last);
     // grid: enough CTAs for the largest phase, at most what is co-resident
     uint64_t need = 1;
     const void* fn;
@@ -432,15 +468,15 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
         fn = (const void*)persistent_bulk_kernel;
         block = dim3(p->bulk_warps * 32);
         smem = bulk_smem_bytes(p);
-        for (int ph = first; ph <= last; ph++) {
-            uint64_t t = (bulk_tasks(p->sched.phase(ph), P, p->bulk_stage_bytes) + p->bulk_warps - 1) / p->bulk_warps;
+        for (int i = 0; i < seq.count(); i++) {
+            uint64_t t = (bulk_tasks(seq.item(i), P, p->bulk_stage_bytes) + p->bulk_warps - 1) / p->bulk_warps;
             if (t > need) need = t;
         }
     } else {
         fn = pick_persistent_vec(rs.vbytes);
         block = dim3(kVecBlock);
-        for (int ph = first; ph <= last; ph++) {
-            const uint64_t tasks = vec_tasks(p->sched.phase(ph), P, rs.vbytes);
+        for (int i = 0; i < seq.count(); i++) {
+            const uint64_t tasks = vec_tasks(seq.item(i), P, rs.vbytes);
             if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
             uint64_t t = (tasks + kVecBlock / 32 - 1) / (kVecBlock / 32);
             if (t > need) need = t;
@@ -458,7 +494,7 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     ctl.base = p->bar_base;
     ctl.expected = (unsigned)grid + (unsigned)p->extra_arrivals;
     ctl.timeout_ns = p->timeout_ns;
-    int first_idx = first + 1, last_idx = last + 1;  // descriptor table index = phase + 1
+    int first_idx = (int)seq.table_index(0), last_idx = (int)seq.table_index(seq.count() - 1);
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
     uint32_t stage = p->bulk_stage_bytes;
@@ -466,16 +502,17 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     void* args_bulk[] = {&gg, &descs, &first_idx, &last_idx, &stage, &ctl};
     CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), block,
                                    rs.copy == SPARBIT_COPY_BULK ? args_bulk : args_vec, smem, st));
-    p->bar_base += (unsigned)(last - first) * ctl.expected;  // one barrier between consecutive phases
+    p->bar_base += (unsigned)(last_idx - first_idx) * ctl.expected;  // one barrier between consecutive passes
     p->kernel_launches++;
     return SPARBIT_OK;
 }
 
 int launch_cluster(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
+    const ExecSeq seq = make_seq(p, first, last);
     uint64_t need = 1;
-    for (int ph = first; ph <= last; ph++) {
-        const uint64_t tasks = vec_tasks(p->sched.phase(ph), P, rs.vbytes);
+    for (int i = 0; i < seq.count(); i++) {
+        const uint64_t tasks = vec_tasks(seq.item(i), P, rs.vbytes);
         if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
         uint64_t t = (tasks + kClusterBlock / 32 - 1) / (kClusterBlock / 32);
         if (t > need) need = t;
@@ -496,7 +533,7 @@ int launch_cluster(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int fir
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int first_idx = first + 1, last_idx = last + 1;
+    int first_idx = (int)seq.table_index(0), last_idx = (int)seq.table_index(seq.count() - 1);
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
     void* args[] = {&gg, &descs, &first_idx, &last_idx};

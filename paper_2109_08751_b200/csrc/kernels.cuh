@@ -174,6 +174,7 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
             const CopyLoc c = locate_copy(d, P, r, j);
             const V* src = reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
             V* dst = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m));
+            V* dst2 = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m));
             const uint64_t v0 = (uint64_t)sp * span + lane;
             V regs[U];
 #pragma unroll
@@ -184,7 +185,10 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t v = v0 + 32u * k;
-                if (v < vpc64) st_cg<V>(dst + v, regs[k]);
+                if (v < vpc64) {
+                    st_cg<V>(dst + v, regs[k]);
+                    if (d.dup_self) st_cg<V>(dst2 + v, regs[k]);
+                }
             }
         }
     } else if (vpc64 > 0) {
@@ -199,6 +203,7 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
         for (uint64_t w = warp_id; w < tasks; w += n_warps) {
             V regs[U];
             V* dsts[U];
+            V* dsts2[U];
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t q64 = (w * U + k) * cpw + sub;
@@ -211,12 +216,16 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
                     const V* src =
                         reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
                     dsts[k] = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
+                    dsts2[k] = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
                     regs[k] = ld_cg<V>(src + v);
                 }
             }
 #pragma unroll
             for (int k = 0; k < U; k++)
-                if (dsts[k]) st_cg<V>(dsts[k], regs[k]);
+                if (dsts[k]) {
+                    st_cg<V>(dsts[k], regs[k]);
+                    if (d.dup_self) st_cg<V>(dsts2[k], regs[k]);
+                }
         }
     }
 }
@@ -227,7 +236,7 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
 struct BulkPipe {
     uint32_t ring;      // shared address of this warp's first stage
     uint32_t bars;      // shared address of this warp's first mbarrier (kBulkStages of them)
-    uint32_t meta;      // shared address of per-stage {dst pointer, bytes} records (16 B each)
+    uint32_t meta;      // shared address of per-stage {dst pointer, bytes, second-dst delta, pad} records (32 B: v2.u64 accesses need 16-byte alignment)
     uint32_t it;        // stages used so far by this ring (carried across phases)
 };
 
@@ -290,11 +299,14 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
             const uint32_t bytes = left < chunk ? (uint32_t)left : chunk;
             const char* src = sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m) + off;
             char* dst = dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m) + off;
+            // second destination of a dup_self phase, as a byte delta from the first
+            const long long delta2 = ((long long)r - (long long)c.dst_rank) * (long long)dpitch;
             const uint32_t bar = pp.bars + st * 8u;
             // remember where this stage goes
-            asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(pp.meta + st * 16u), "l"(dst),
+            asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(pp.meta + st * 32u), "l"(dst),
                          "l"((unsigned long long)bytes)
                          : "memory");
+            asm volatile("st.shared.u64 [%0], %1;" ::"r"(pp.meta + st * 32u + 16u), "l"(delta2) : "memory");
             mbar_expect_tx(bar, bytes);
             bulk_load(pp.ring + st * stage_bytes, src, bytes, bar);
         }
@@ -307,9 +319,14 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
                 break;
             }
             unsigned long long dst, bytes;
-            asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(dst), "=l"(bytes) : "r"(pp.meta + st * 16u)
+            asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(dst), "=l"(bytes) : "r"(pp.meta + st * 32u)
                          : "memory");
             bulk_store(reinterpret_cast<void*>(dst), pp.ring + st * stage_bytes, (uint32_t)bytes);
+            if (d.dup_self) {
+                long long delta2;
+                asm volatile("ld.shared.u64 %0, [%1];" : "=l"(delta2) : "r"(pp.meta + st * 32u + 16u) : "memory");
+                bulk_store(reinterpret_cast<void*>(dst + delta2), pp.ring + st * stage_bytes, (uint32_t)bytes);
+            }
             bulk_commit();
         }
     }
@@ -386,7 +403,7 @@ __device__ __forceinline__ BulkPipe make_pipe(unsigned char* smem, uint32_t stag
     const uint32_t rings = warps * kBulkStages * stage_bytes;
     pp.ring = base + warp * kBulkStages * stage_bytes;
     pp.bars = base + rings + warp * kBulkStages * 8u;
-    pp.meta = base + rings + warps * kBulkStages * 8u + warp * kBulkStages * 16u;
+    pp.meta = base + rings + warps * kBulkStages * 8u + warp * kBulkStages * 32u;
     pp.it = 0;
     return pp;
 }

@@ -11,6 +11,10 @@
 // device.  Each copy moves copy_bytes = run * m bytes: `run` consecutive slots when the phase's
 // blocks are contiguous on both sides (recursive doubling, Bruck), else one block.
 //
+// A phase with dup_self = 1 writes each copy twice: to (dst_rank, dst_slot) and to (r, dst_slot).
+// That is the own-block copy and the first step in one pass: the first step forwards exactly the
+// own block, so sendbuf[r] is read once and lands in recvbuf[r][r] and in the first peer's slot r.
+//
 // This form covers Algorithm 1's steps (peer r + d, slots r - 2jd on both sides), the ring, the
 // recursive-doubling exchange (peer r xor 2^s, aligned groups), Bruck's steps and rotation, and
 // the own-block copy, in O(1) bytes per phase whatever P is.
@@ -41,7 +45,8 @@ struct PhaseDesc {
     int32_t  dst_step;
     uint32_t src_space;
     uint32_t dst_space;
-    uint32_t pad_;
+    uint32_t dup_self;   // 1: every copy is also written to the SENDING rank's buffer of dst_space,
+                         // same slot (the own-block copy fused with the first step)
     uint64_t copy_bytes; // run * m
 };
 

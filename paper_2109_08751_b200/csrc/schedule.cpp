@@ -159,6 +159,27 @@ static int build_bruck(uint32_t P, uint64_t m, Schedule& s) {
     return SCHED_OK;
 }
 
+// The first step of Sparbit, ring and recursive doubling forwards exactly one block per rank, the
+// rank's own, from the slot the own-block copy has just filled.  Reading it from sendbuf instead
+// and writing it to both places gives the same state after phase 0 with one pass less.
+static void add_fused_first(Schedule& s) {
+    if (s.K < 1 || s.rotation) return;
+    const PhaseDesc& own = s.phases[0];
+    const PhaseDesc& st0 = s.phases[1];
+    if (st0.copies != 1 || st0.run != 1 || st0.src_space != SPACE_RECV || st0.dst_space != SPACE_RECV) return;
+    // step 0 must read slot r of rank r (what the own-block copy wrote) and store it in slot r
+    if (st0.src_rcoef != 1 || st0.src_off != 0 || st0.dst_rcoef != 1 || st0.dst_off != 0) return;
+    if (st0.rank_mask != 0xFFFFFFFFu) return;
+    PhaseDesc f = st0;
+    f.src_space = own.src_space;  // sendbuf[r], one slot per rank
+    f.src_rcoef = 0;
+    f.src_off = 0;
+    f.src_step = 0;
+    f.dup_self = 1;
+    s.fused_first = f;
+    s.has_fused_first = true;
+}
+
 int build_schedule(int algo, int64_t P64, uint64_t m, Schedule& out) {
     if (P64 < 1) return SCHED_ARG;
     if (P64 > (1 << 24)) return SCHED_OVERFLOW;
@@ -170,13 +191,16 @@ int build_schedule(int algo, int64_t P64, uint64_t m, Schedule& out) {
     out.algo = algo;
     out.P = P;
     out.m = m;
+    int rc;
     switch (algo) {
-        case ALGO_SPARBIT: return build_sparbit(P, m, out);
-        case ALGO_RING: return build_ring(P, m, out);
-        case ALGO_RD: return build_rd(P, m, out);
-        case ALGO_BRUCK: return build_bruck(P, m, out);
+        case ALGO_SPARBIT: rc = build_sparbit(P, m, out); break;
+        case ALGO_RING: rc = build_ring(P, m, out); break;
+        case ALGO_RD: rc = build_rd(P, m, out); break;
+        case ALGO_BRUCK: rc = build_bruck(P, m, out); break;
         default: return SCHED_ARG;
     }
+    if (rc == SCHED_OK) add_fused_first(out);
+    return rc;
 }
 
 uint64_t phase_message_count(const Schedule& s, int phase) {

@@ -25,6 +25,11 @@ struct Schedule {
     // phases[0] is phase -1 (own block), phases[1 + s] is step s, phases[1 + K] the rotation
     std::vector<PhaseDesc> phases;
     std::vector<StepInfo> steps;
+    // Execution-only shortcut: phases -1 and 0 as ONE pass (sendbuf[r] read once, written to
+    // recvbuf[r][r] and to the first peer's slot r).  Valid when has_fused_first; used when a call
+    // runs both phases.  The logical schedule (phases, messages) is unchanged by it.
+    bool has_fused_first = false;
+    PhaseDesc fused_first;
     int last_phase() const { return rotation ? K : K - 1; }
     const PhaseDesc& phase(int ph) const { return phases[(size_t)(ph + 1)]; }
 };

@@ -253,7 +253,7 @@ def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
     want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
     assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
     kernels, graphs = plan.launch_counts()
-    phases = plan.num_steps + 1
+    phases = plan.num_steps  # the own-block copy and step 0 run as one fused pass
     if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_CLUSTER):
         assert (kernels, graphs) == (2, 0)
     elif exec_mode == sp.EXEC_GRAPH:
