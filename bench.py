@@ -397,6 +397,8 @@ def run_sweep(args):
                    for m in (8, 64, 512, 4096, 32768, 65536, 262144)]
     if args.sweep == "config3":
         points += [(128, 65536, ["sparbit"])]
+    if args.sweep == "small":  # configs 1 and 2 and their neighbourhood: latency only
+        points += [(P, m, ["sparbit"]) for P in (6, 8, 13, 16, 32, 64) for m in (64, 4096)]
     algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
              "bruck": sp.ALGO_BRUCK}
     execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
@@ -463,7 +465,7 @@ def main():
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--sweep", choices=["config3", "config4", "config5", "all"], default=None,
+    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     args = ap.parse_args()
     if args.sweep:

@@ -30,7 +30,7 @@ int cuda_fail(cudaError_t e, const char* what) {
 
 constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s
 constexpr int kVecBlock = 512;
-constexpr int kClusterBlock = 512;
+constexpr int kClusterBlock = 1024;
 
 struct GraphKey {
     const void* send = nullptr;
@@ -517,22 +517,34 @@ int launch_cluster(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int fir
         uint64_t t = (tasks + kClusterBlock / 32 - 1) / (kClusterBlock / 32);
         if (t > need) need = t;
     }
-    unsigned ctas = 8;  // the portable cluster size
-    while (ctas > 1 && ctas / 2 >= need) ctas /= 2;
     const void* fn = pick_cluster_vec(rs.vbytes);
+    // 16 CTAs (the non-portable maximum) when the device can place such a cluster, else 8
+    unsigned ctas = 16;
     cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(ctas);
-    cfg.blockDim = dim3(kClusterBlock);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = ctas;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        ctas = 8;
+    }
+    for (;;) {
+        while (ctas > 1 && ctas / 2 >= need) ctas /= 2;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(ctas);
+        cfg.blockDim = dim3(kClusterBlock);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = ctas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int fit = 0;
+        if (ctas <= 8 || (cudaOccupancyMaxActiveClusters(&fit, fn, &cfg) == cudaSuccess && fit >= 1)) break;
+        (void)cudaGetLastError();
+        ctas = 8;
+        need = ~0ull;  // keep 8
+    }
     int first_idx = (int)seq.table_index(0), last_idx = (int)seq.table_index(seq.count() - 1);
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;

@@ -489,7 +489,7 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
 // cluster barrier (arrive.release / wait.acquire) separates phases.  For collectives so small
 // that a grid-wide barrier or a kernel boundary per phase would dominate.
 template <typename V>
-__global__ void __launch_bounds__(512) cluster_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
+__global__ void __launch_bounds__(1024) cluster_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
                                                            int last) {
     __shared__ PhaseDesc sd[2];
     const uint32_t wpb = blockDim.x >> 5;
