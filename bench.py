@@ -232,7 +232,7 @@ def run_ours(args):
 
     P, m = args.P, args.m
     algo = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
-            "bruck": sp.ALGO_BRUCK}[args.algo]
+            "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}[args.algo]
     exec_mode = {"auto": sp.EXEC_AUTO, "persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH,
                  "stream": sp.EXEC_STREAM, "cluster": sp.EXEC_CLUSTER}[args.exec]
     copy = {"auto": sp.COPY_AUTO, "vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}[args.copy]
@@ -393,14 +393,14 @@ def run_sweep(args):
     if args.sweep in ("config4", "all"):
         points += [(1000, 1024, ["sparbit"])]
     if args.sweep in ("config5", "all"):
-        points += [(256, m, ["sparbit", "ring", "rd", "bruck"])
+        points += [(256, m, ["sparbit", "ring", "ne", "rd", "bruck"])
                    for m in (8, 64, 512, 4096, 32768, 65536, 262144)]
     if args.sweep == "config3":
         points += [(128, 65536, ["sparbit"])]
     if args.sweep == "small":  # configs 1 and 2 and their neighbourhood: latency only
         points += [(P, m, ["sparbit"]) for P in (6, 8, 13, 16, 32, 64) for m in (64, 4096)]
     algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
-             "bruck": sp.ALGO_BRUCK}
+             "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}
     execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
              "cluster": sp.EXEC_CLUSTER}
     copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
@@ -415,7 +415,7 @@ def run_sweep(args):
             for ename, e in execs.items():
                 if ename == "cluster" and effective_bytes(P, m) > (64 << 20):
                     continue
-                if ename == "stream" and name == "ring" and m >= 32768:
+                if ename == "stream" and name in ("ring", "ne") and m >= 32768:
                     continue  # same kernels as the graph chain; skipped to bound the sweep
                 for cname, c in copies.items():
                     if cname == "bulk" and (m % 16 or ename == "cluster"):
@@ -459,7 +459,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--P", type=int, default=P_DEFAULT)
     ap.add_argument("--m", type=int, default=M_DEFAULT)
-    ap.add_argument("--algo", choices=["sparbit", "ring", "rd", "bruck"], default="sparbit")
+    ap.add_argument("--algo", choices=["sparbit", "ring", "ne", "rd", "bruck"], default="sparbit")
     ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "cluster"], default="auto")
     ap.add_argument("--copy", choices=["auto", "vector", "bulk"], default="auto")
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)

@@ -49,7 +49,8 @@ enum {
     SPARBIT_ERR_ARG = 1,         /* null handle/buffer, P < 1, phase range or enum out of range */
     SPARBIT_ERR_OVERFLOW = 2,    /* P*P*m (or an internal work count) is not representable */
     SPARBIT_ERR_ALIAS = 3,       /* send / receive / workspace byte ranges overlap */
-    SPARBIT_ERR_UNSUPPORTED = 4, /* recursive doubling with P not a power of two; bad mode combo */
+    SPARBIT_ERR_UNSUPPORTED = 4, /* recursive doubling with P not a power of two; neighbor
+                                    exchange with odd P; bad mode combination */
     SPARBIT_ERR_WORKSPACE = 5,   /* Bruck without a workspace, or one that is too small */
     SPARBIT_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sparbit_last_cuda_error() */
     SPARBIT_ERR_TIMEOUT = 7,     /* the device-side grid barrier gave up waiting */
@@ -58,12 +59,13 @@ enum {
 };
 
 /* Algorithms (paper, Section II-A and Section III).  Only Sparbit is the product's hot path; the
- * other three run on the same executor as comparators. */
+ * other four run on the same executor as comparators. */
 enum {
     SPARBIT_ALGO_SPARBIT = 0,
     SPARBIT_ALGO_RING = 1,
     SPARBIT_ALGO_RECURSIVE_DOUBLING = 2, /* powers of two only, as the paper states */
-    SPARBIT_ALGO_BRUCK = 3
+    SPARBIT_ALGO_BRUCK = 3,
+    SPARBIT_ALGO_NEIGHBOR_EXCHANGE = 4   /* even P only, as the paper states */
 };
 
 /* How the phases are put on the GPU. */
@@ -116,8 +118,8 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
  * *out receives a plan the caller must release with sparbit_plan_destroy.  block_bytes may be 0
  * (the collective is then a no-op, as MPI allows count 0).  Errors: ERR_ARG (P < 1, null out,
  * unknown enum), ERR_OVERFLOW (P*P*block_bytes does not fit in 63 bits, or P > 2^24),
- * ERR_UNSUPPORTED (recursive doubling with P not a power of two: Section II-A defines it for
- * powers of two only), ERR_NOMEM.  Host-only.
+ * ERR_UNSUPPORTED (recursive doubling with P not a power of two, neighbor exchange with odd P:
+ * Section II-A defines them for those P only), ERR_NOMEM.  Host-only.
  */
 int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out);
 
@@ -159,7 +161,8 @@ int sparbit_allgather_host(sparbit_plan_t* plan, const void* host_send, void* ho
 /* ---- introspection (host-only, no CUDA call) ------------------------------------------------ */
 
 /* K, the number of communication steps: Sparbit and Bruck ceil(log2 P), recursive doubling
- * log2 P, ring P-1 (the latency terms of the cost formulae of Sections II-A and III-B). */
+ * log2 P, ring P-1, neighbor exchange P/2 (the latency terms of the cost formulae of Sections
+ * II-A and III-B). */
 int sparbit_plan_num_steps(const sparbit_plan_t* plan);
 
 /* Index of the last phase: K-1, or K for Bruck (rotation).  -1 when P = 1 and not Bruck. */

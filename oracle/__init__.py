@@ -18,8 +18,9 @@ _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "allgather_oracle.c"
 _LIB = _HERE / "liballgather_oracle.so"
 
-SPARBIT, RING, RECURSIVE_DOUBLING, BRUCK = 0, 1, 2, 3
-ALGO_NAMES = {SPARBIT: "sparbit", RING: "ring", RECURSIVE_DOUBLING: "recursive_doubling", BRUCK: "bruck"}
+SPARBIT, RING, RECURSIVE_DOUBLING, BRUCK, NEIGHBOR_EXCHANGE = 0, 1, 2, 3, 4
+ALGO_NAMES = {SPARBIT: "sparbit", RING: "ring", RECURSIVE_DOUBLING: "recursive_doubling", BRUCK: "bruck",
+              NEIGHBOR_EXCHANGE: "neighbor_exchange"}
 SPACE_SEND, SPACE_RECV, SPACE_SCRATCH = 0, 1, 2
 
 MSG_DTYPE = np.dtype(

@@ -27,6 +27,12 @@
  *   RING     Section II-A: p-1 steps, r -> r+1, own block first, then forward what arrived last.
  *   RD       Section II-A recursive doubling: log2 p steps, partner r xor 2^s, send all held;
  *            defined for powers of two only (the paper states the restriction).
+ *   NE       Section II-A neighbor exchange: p/2 steps, even p only; on step s an even rank r
+ *            exchanges with r + (-1)^s and an odd rank with r - (-1)^s (wrap-around); one block
+ *            (the own) on the first step, two blocks on every other step.  Which two the paper
+ *            leaves open; the reading taken: on step 1 a rank sends the two blocks it holds,
+ *            on every later step the two blocks it received on the previous step (the ring's
+ *            rule, applied pairwise).  A rank receives what its partner sends.
  *   BRUCK    Section II-A: floor(log2 p) steps sending everything held to r - 2^s, receiving
  *            from r + 2^s, one more step with the first p - 2^floor(log2 p) blocks when p is
  *            not a power of two, then the rotation.  Local order: slot i of the working buffer
@@ -52,7 +58,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORACLE_SPARBIT = 0, ORACLE_RING = 1, ORACLE_RD = 2, ORACLE_BRUCK = 3 };
+enum { ORACLE_SPARBIT = 0, ORACLE_RING = 1, ORACLE_RD = 2, ORACLE_BRUCK = 3, ORACLE_NE = 4 };
 enum { SPACE_SEND = 0, SPACE_RECV = 1, SPACE_SCRATCH = 2 };
 
 typedef struct {
@@ -190,6 +196,42 @@ static int rd_rank_posts(int p, int rank, postlist_t *sends, postlist_t *recvs) 
         for (int j = 0; j < held; j++) {
             if (post_push(sends, s, partner, SPACE_RECV, mine + j)) return -1;
             if (post_push(recvs, s, partner, SPACE_RECV, theirs + j)) return -1;
+        }
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- Neighbor exchange --------- */
+static int ne_partner(int p, int rank, int s) {
+    int sign = (s % 2 == 0) ? 1 : -1;                 /* (-1)^s */
+    int to = (rank % 2 == 0) ? rank + sign : rank - sign;
+    return (int)pmod(to, p);
+}
+
+/* first[s * p + x]: first of the (one or two) consecutive slots rank x sends on step s */
+static int *ne_send_table(int p) {
+    int steps = p / 2;
+    int *first = (int *)malloc((size_t)(steps > 0 ? steps : 1) * (size_t)p * sizeof(int));
+    if (!first) return NULL;
+    for (int s = 0; s < steps; s++)
+        for (int x = 0; x < p; x++) {
+            if (s == 0)
+                first[x] = x;                           /* the own block */
+            else if (s == 1)
+                first[p + x] = x - x % 2;               /* the two it holds: own and step 0's */
+            else                                        /* what arrived on the previous step */
+                first[s * p + x] = first[(s - 1) * p + ne_partner(p, x, s - 1)];
+        }
+    return first;
+}
+
+static int ne_rank_posts(int p, int rank, const int *first, postlist_t *sends, postlist_t *recvs) {
+    for (int s = 0; s < p / 2; s++) {
+        int partner = ne_partner(p, rank, s);
+        int n = s == 0 ? 1 : 2;
+        for (int j = 0; j < n; j++) {
+            if (post_push(sends, s, partner, SPACE_RECV, first[s * p + rank] + j)) return -1;
+            if (post_push(recvs, s, partner, SPACE_RECV, first[s * p + partner] + j)) return -1;
         }
     }
     return 0;
@@ -355,7 +397,7 @@ oracle_plan *oracle_plan_create(int algo, int P) {
         set_err("P must be >= 1");
         return NULL;
     }
-    if (algo < ORACLE_SPARBIT || algo > ORACLE_BRUCK) {
+    if (algo < ORACLE_SPARBIT || algo > ORACLE_NE) {
         set_err("unknown algorithm %d", algo);
         return NULL;
     }
@@ -363,6 +405,11 @@ oracle_plan *oracle_plan_create(int algo, int P) {
         set_err("recursive doubling is defined for powers of two only");
         return NULL;
     }
+    if (algo == ORACLE_NE && P % 2 != 0) {
+        set_err("neighbor exchange works with an even number of processes only");
+        return NULL;
+    }
+    int *ne_first = NULL;
     oracle_plan *pl = (oracle_plan *)calloc(1, sizeof *pl);
     postlist_t *sends = (postlist_t *)calloc((size_t)P, sizeof(postlist_t));
     postlist_t *recvs = (postlist_t *)calloc((size_t)P, sizeof(postlist_t));
@@ -376,7 +423,14 @@ oracle_plan *oracle_plan_create(int algo, int P) {
     }
     pl->algo = algo;
     pl->P = P;
-    pl->K = algo == ORACLE_RING ? P - 1 : ceil_log2((unsigned)P);
+    pl->K = algo == ORACLE_RING ? P - 1 : algo == ORACLE_NE ? P / 2 : ceil_log2((unsigned)P);
+    if (algo == ORACLE_NE) {
+        ne_first = ne_send_table(P);
+        if (!ne_first) {
+            set_err("out of memory");
+            goto fail;
+        }
+    }
     pl->has_rotation = algo == ORACLE_BRUCK;
 
     /* every rank runs the algorithm on its own and posts its operations */
@@ -387,6 +441,7 @@ oracle_plan *oracle_plan_create(int algo, int P) {
             case ORACLE_RING: rc = ring_rank_posts(P, r, &sends[r], &recvs[r]); break;
             case ORACLE_RD: rc = rd_rank_posts(P, r, &sends[r], &recvs[r]); break;
             case ORACLE_BRUCK: rc = bruck_rank_posts(P, r, &sends[r], &recvs[r]); break;
+            case ORACLE_NE: rc = ne_rank_posts(P, r, ne_first, &sends[r], &recvs[r]); break;
         }
         if (rc) {
             if (!g_err[0]) set_err("out of memory while posting");
@@ -481,6 +536,7 @@ oracle_plan *oracle_plan_create(int algo, int P) {
 
     if (check_plan(pl)) goto fail;
 
+    free(ne_first);
     free_lists(sends, P);
     free_lists(recvs, P);
     free(cursor);
@@ -489,6 +545,7 @@ oracle_plan *oracle_plan_create(int algo, int P) {
     free(matched);
     return pl;
 fail:
+    free(ne_first);
     free_lists(sends, P);
     free_lists(recvs, P);
     free(cursor);

@@ -15,13 +15,13 @@ _LIB_PATH = Path(__file__).resolve().parent / "libsparbit_b200.so"
 OK = 0
 ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT = \
     range(1, 10)
-ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK = range(4)
+ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK, ALGO_NEIGHBOR_EXCHANGE = range(5)
 EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_CLUSTER = range(5)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
 SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
-              ALGO_BRUCK: "bruck"}
+              ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}
 EXEC_NAMES = {EXEC_AUTO: "auto", EXEC_PERSISTENT: "persistent", EXEC_GRAPH: "graph", EXEC_STREAM: "stream",
               EXEC_CLUSTER: "cluster"}
 COPY_NAMES = {COPY_AUTO: "auto", COPY_VECTOR: "vector", COPY_BULK: "bulk"}

@@ -593,7 +593,7 @@ extern "C" {
 int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out) {
     if (!out) return SPARBIT_ERR_ARG;
     *out = nullptr;
-    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_ARG;
+    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
     if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_CLUSTER) return SPARBIT_ERR_ARG;
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
@@ -765,7 +765,8 @@ const char* sparbit_strerror(int code) {
         case SPARBIT_ERR_ARG: return "invalid argument";
         case SPARBIT_ERR_OVERFLOW: return "size not representable";
         case SPARBIT_ERR_ALIAS: return "buffers overlap";
-        case SPARBIT_ERR_UNSUPPORTED: return "unsupported (recursive doubling needs a power-of-two P)";
+        case SPARBIT_ERR_UNSUPPORTED:
+            return "unsupported (recursive doubling needs a power-of-two P, neighbor exchange an even P)";
         case SPARBIT_ERR_WORKSPACE: return "workspace missing or too small";
         case SPARBIT_ERR_CUDA: return "CUDA runtime error";
         case SPARBIT_ERR_TIMEOUT: return "device barrier timed out";

@@ -7,7 +7,8 @@
 // r - 2jd on both sides, which the PhaseDesc form states in O(1) bytes.  The counts are
 // cross-checked against the counting form ceil(P/d) - ceil(P/2d) before a plan is accepted.
 //
-// Ring, recursive doubling and Bruck (Section II-A) are expressed in the same descriptor form.
+// Ring, neighbor exchange, recursive doubling and Bruck (Section II-A) are expressed in the same
+// descriptor form.
 #include "schedule.h"
 
 #include <string.h>
@@ -49,7 +50,8 @@ static bool steps_stay_in_range(const PhaseDesc& d, uint32_t P) {
     // (copies-1) * |step| < P keeps base + j*step inside (-P, 2P)
     uint64_t a = (uint64_t)(d.copies - 1) * (uint64_t)(d.src_step < 0 ? -(int64_t)d.src_step : d.src_step);
     uint64_t b = (uint64_t)(d.copies - 1) * (uint64_t)(d.dst_step < 0 ? -(int64_t)d.dst_step : d.dst_step);
-    return a < P && b < P && d.src_off < P && d.dst_off < P && d.peer_add < P;
+    return a < P && b < P && d.src_off < P && d.dst_off < P && d.src_off_odd < P && d.dst_off_odd < P &&
+           d.peer_add < P && d.peer_pre < P;
 }
 
 static int build_sparbit(uint32_t P, uint64_t m, Schedule& s) {
@@ -159,8 +161,50 @@ static int build_bruck(uint32_t P, uint64_t m, Schedule& s) {
     return SCHED_OK;
 }
 
-// The first step of Sparbit, ring and recursive doubling forwards exactly one block per rank, the
-// rank's own, from the slot the own-block copy has just filled.  Reading it from sendbuf instead
+// Neighbor exchange (Section II-A): P/2 steps, even P only.  On step s an even rank r exchanges
+// with r + (-1)^s and an odd rank with r - (-1)^s: the pairing {2k, 2k+1} on even steps, the
+// pairing shifted by one, {2k-1, 2k}, on odd steps; both are "add c, flip the lowest bit, subtract
+// c" with c = s mod 2.  Step 0 swaps the own blocks, step 1 sends the pair of blocks a rank then
+// holds, every later step forwards the pair received on the step before.  Unrolled, a rank whose
+// own pair of slots starts at 2k forwards, on step s >= 1, the pair that starts a(s) pairs away:
+// even ranks backwards on even steps and forwards on odd ones, odd ranks the other way round,
+// with a(s) = s/2 on even steps and (s-1)/2 on odd ones.  Pairs land in their final slots.
+static int build_ne(uint32_t P, uint64_t m, Schedule& s) {
+    if (P % 2) return SCHED_UNSUPPORTED;
+    s.K = (int)(P / 2);
+    s.phases.push_back(own_copy(m, false));
+    for (uint32_t st = 0; st < P / 2; st++) {
+        const uint32_t c = st & 1u;
+        PhaseDesc ph = blank(m);
+        ph.peer_pre = c;
+        ph.peer_xor = 1;
+        ph.peer_add = (P - c) % P;
+        ph.src_space = ph.dst_space = SPACE_RECV;
+        ph.src_rcoef = ph.dst_rcoef = 1;
+        if (st == 0) {
+            // the own block, slot r on both sides
+        } else {
+            const uint32_t a = c ? (st - 1) / 2 : st / 2;  // pairs away from the own pair
+            const uint32_t away = (2 * a) % P;              // in slots
+            const uint32_t back = (P - away) % P;
+            ph.rank_mask = ~1u;                             // 2k: first slot of the own pair
+            ph.parity_split = 1;
+            ph.src_off = ph.dst_off = c ? away : back;          // even ranks
+            ph.src_off_odd = ph.dst_off_odd = c ? back : away;  // odd ranks
+            ph.src_step = ph.dst_step = 1;
+            ph.copies = 1;                                  // the two slots are adjacent: one copy
+            ph.run = 2;
+            ph.copy_bytes = 2 * m;
+        }
+        if (!steps_stay_in_range(ph, P)) return SCHED_INTERNAL;
+        s.phases.push_back(ph);
+        s.steps.push_back({1, st == 0 ? 1 : 2, 0});
+    }
+    return SCHED_OK;
+}
+
+// The first step of Sparbit, ring, neighbor exchange and recursive doubling forwards exactly one
+// block per rank, the rank's own, from the slot the own-block copy has just filled.  Reading it from sendbuf instead
 // and writing it to both places gives the same state after phase 0 with one pass less.
 static void add_fused_first(Schedule& s) {
     if (s.K < 1 || s.rotation) return;
@@ -173,7 +217,7 @@ static void add_fused_first(Schedule& s) {
     PhaseDesc f = st0;
     f.src_space = own.src_space;  // sendbuf[r], one slot per rank
     f.src_rcoef = 0;
-    f.src_off = 0;
+    f.src_off = f.src_off_odd = 0;
     f.src_step = 0;
     f.dup_self = 1;
     s.fused_first = f;
@@ -197,10 +241,18 @@ int build_schedule(int algo, int64_t P64, uint64_t m, Schedule& out) {
         case ALGO_RING: rc = build_ring(P, m, out); break;
         case ALGO_RD: rc = build_rd(P, m, out); break;
         case ALGO_BRUCK: rc = build_bruck(P, m, out); break;
+        case ALGO_NE: rc = build_ne(P, m, out); break;
         default: return SCHED_ARG;
     }
-    if (rc == SCHED_OK) add_fused_first(out);
-    return rc;
+    if (rc != SCHED_OK) return rc;
+    // one offset for both parities unless a builder split them on purpose
+    for (PhaseDesc& ph : out.phases)
+        if (!ph.parity_split) {
+            ph.src_off_odd = ph.src_off;
+            ph.dst_off_odd = ph.dst_off;
+        }
+    add_fused_first(out);
+    return SCHED_OK;
 }
 
 uint64_t phase_message_count(const Schedule& s, int phase) {

@@ -8,7 +8,7 @@
 
 namespace spb {
 
-enum Algo { ALGO_SPARBIT = 0, ALGO_RING = 1, ALGO_RD = 2, ALGO_BRUCK = 3 };
+enum Algo { ALGO_SPARBIT = 0, ALGO_RING = 1, ALGO_RD = 2, ALGO_BRUCK = 3, ALGO_NE = 4 };
 
 struct StepInfo {
     int distance;  // ranks between sender and receiver (Algorithm 1's d)

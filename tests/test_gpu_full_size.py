@@ -75,7 +75,8 @@ def test_config4_p1000_m1k(dev, exec_mode):
 
 # config 5: the sweep at P = 256
 @pytest.mark.parametrize("m", [8, 64, 512, 4096, 32768])
-@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK])
+@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK,
+                                  sp.ALGO_NEIGHBOR_EXCHANGE])
 def test_config5_sweep(dev, m, algo):
     full_compare(dev, 256, m, algo, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 5, iters=1)
 

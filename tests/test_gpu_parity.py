@@ -18,7 +18,7 @@ from paper_2109_08751_b200 import binding
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
-ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK]
+ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK, sp.ALGO_NEIGHBOR_EXCHANGE]
 EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_CLUSTER]
 COPIES = [sp.COPY_VECTOR, sp.COPY_BULK]
 G = si.GUARD_BYTES
@@ -121,9 +121,23 @@ def test_config2_recursive_doubling_refused(P):
         == sp.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("P", [6, 8, 14])
+@pytest.mark.parametrize("exec_mode", EXECS)
+@pytest.mark.parametrize("copy", COPIES)
+def test_config2_neighbor_exchange_even_p(dev, P, exec_mode, copy):
+    run_case(dev, P, 4096, sp.ALGO_NEIGHBOR_EXCHANGE, exec_mode, copy, si.BASE_SEED + 2)
+
+
+def test_config2_neighbor_exchange_refused_for_odd_p():
+    out = ctypes.c_void_p()
+    assert binding.lib.sparbit_plan_create(13, 4096, sp.ALGO_NEIGHBOR_EXCHANGE, 0, ctypes.byref(out)) \
+        == sp.ERR_UNSUPPORTED
+
+
 # ---------------------------------------------------------------- phase-by-phase state
 @pytest.mark.parametrize("algo,P", [(sp.ALGO_SPARBIT, 5), (sp.ALGO_SPARBIT, 21), (sp.ALGO_SPARBIT, 32),
-                                    (sp.ALGO_BRUCK, 13), (sp.ALGO_RING, 6), (sp.ALGO_RECURSIVE_DOUBLING, 16)])
+                                    (sp.ALGO_BRUCK, 13), (sp.ALGO_RING, 6), (sp.ALGO_RECURSIVE_DOUBLING, 16),
+                                    (sp.ALGO_NEIGHBOR_EXCHANGE, 10)])
 @pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_STREAM])
 def test_state_after_every_phase(dev, algo, P, exec_mode):
     """Run one phase at a time on both sides; the whole state (sentinel included) must agree."""
@@ -154,10 +168,13 @@ def test_every_p_up_to_64(dev, exec_mode):
         run_case(dev, P, 16, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=1)
 
 
-@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK])
+@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK,
+                                  sp.ALGO_NEIGHBOR_EXCHANGE])
 def test_comparators_many_p(dev, algo):
     for P in [1, 2, 3, 4, 5, 7, 8, 12, 16, 17, 31, 32, 33, 64]:
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
             continue
         run_case(dev, P, 48, algo, sp.EXEC_PERSISTENT, sp.COPY_AUTO, 2000 + P, iters=1)
 
@@ -181,7 +198,10 @@ def test_misaligned_buffers(dev, shifts, algo):
 
 def test_single_rank_and_empty_blocks(dev):
     for algo in ALGOS:
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE:
+            continue  # one rank is not an even number of ranks
         run_case(dev, 1, 256, algo, sp.EXEC_AUTO, sp.COPY_AUTO, 9, iters=1)
+    run_case(dev, 2, 256, sp.ALGO_NEIGHBOR_EXCHANGE, sp.EXEC_AUTO, sp.COPY_AUTO, 9, iters=1)
     plan = sp.Plan(8, 0)
     plan.allgather(None, None)
     assert plan.status() == sp.OK
@@ -195,7 +215,8 @@ def test_medium_shapes(dev, P, m, exec_mode, copy):
     run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, copy, 4242)
 
 
-@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK])
+@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK,
+                                  sp.ALGO_NEIGHBOR_EXCHANGE])
 @pytest.mark.parametrize("copy", COPIES)
 def test_medium_shapes_comparators(dev, algo, copy):
     run_case(dev, 64, 20480, algo, sp.EXEC_PERSISTENT, copy, 4343, iters=1)

@@ -13,7 +13,16 @@ import oracle
 import seeded_inputs as si
 
 ALL_P = list(range(1, 65))
-ALGOS = [oracle.SPARBIT, oracle.RING, oracle.RECURSIVE_DOUBLING, oracle.BRUCK]
+ALGOS = [oracle.SPARBIT, oracle.RING, oracle.RECURSIVE_DOUBLING, oracle.BRUCK, oracle.NEIGHBOR_EXCHANGE]
+
+
+def defined_for(algo, P):
+    """Recursive doubling: powers of two only; neighbor exchange: even P only (Section II-A)."""
+    if algo == oracle.RECURSIVE_DOUBLING:
+        return P & (P - 1) == 0
+    if algo == oracle.NEIGHBOR_EXCHANGE:
+        return P % 2 == 0
+    return True
 
 
 def is_pow2(p):
@@ -44,7 +53,7 @@ def step_sets(pl, spaces=False):
 def test_final_state_is_rank_ordered_concatenation(algo):
     """Section II: slot j of every receive buffer holds the block sent by rank j."""
     for P in ALL_P:
-        if algo == oracle.RECURSIVE_DOUBLING and not is_pow2(P):
+        if not defined_for(algo, P):
             continue
         for m in (1, 4, 7, 16):
             send = si.send_blocks(P, m, seed=si.BASE_SEED + P)
@@ -209,7 +218,7 @@ def test_sparbit_is_p_shifted_binomial_trees(P):
 @pytest.mark.parametrize("P", [1, 2, 3, 5, 6, 8, 13, 16, 21, 37, 64])
 def test_each_block_received_exactly_once(algo, P):
     """Every rank receives (p - 1) blocks, one from each other origin, none twice."""
-    if algo == oracle.RECURSIVE_DOUBLING and not is_pow2(P):
+    if not defined_for(algo, P):
         return
     pl = plan(algo, P)
     msgs = pl.messages
@@ -322,6 +331,40 @@ def test_bruck_shape(P):
     # rotation is purely local and touches every slot once
     rot = pl.phase_messages(pl.num_steps)
     assert len(rot) == P * P and (rot["src_rank"] == rot["dst_rank"]).all()
+
+
+@pytest.mark.parametrize("P", [2, 4, 6, 8, 10, 14, 16, 30, 64, 100])
+def test_neighbor_exchange_shape(P):
+    """Section II-A: p/2 steps; on step s an even process r exchanges with r + (-1)^s and an odd
+    one with r - (-1)^s, always pairwise; one block on the first step, two on all others, which
+    adds up to the p - 1 blocks of the cost formula's bandwidth term."""
+    pl = plan(oracle.NEIGHBOR_EXCHANGE, P)
+    assert pl.num_steps == P // 2                      # p/2 alpha
+    total = 0
+    for s, msgs in enumerate(step_sets(pl)):
+        per_rank = 1 if s == 0 else 2
+        assert len(msgs) == P * per_rank
+        partner = {}
+        for src, dst, a, b in msgs:
+            sign = (-1) ** s
+            want = (src + sign) % P if src % 2 == 0 else (src - sign) % P
+            assert dst == want and a == b
+            partner[src] = dst
+        assert all(partner[partner[r]] == r for r in range(P))   # exchanges are pairwise
+        total += per_rank
+    assert total == P - 1
+    # the first step swaps the own blocks of the two neighbours
+    assert step_sets(pl)[0] == {(r, r ^ 1, r, r) for r in range(P)}
+    if P >= 4:
+        # the second step sends the two blocks held so far: the pair {2k, 2k+1}
+        assert {(a, src) for src, dst, a, b in step_sets(pl)[1]} == \
+            {(2 * (r // 2) + j, r) for r in range(P) for j in (0, 1)}
+
+
+@pytest.mark.parametrize("P", [3, 5, 7, 13, 21])
+def test_neighbor_exchange_only_for_even_p(P):
+    with pytest.raises(oracle.OracleError):
+        plan(oracle.NEIGHBOR_EXCHANGE, P)
 
 
 @pytest.mark.parametrize("P", [4, 8, 16, 64])

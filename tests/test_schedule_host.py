@@ -13,7 +13,7 @@ import paper_2109_08751_b200 as sp
 from paper_2109_08751_b200 import binding
 
 ROOT = Path(__file__).resolve().parent.parent
-ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK]
+ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK, sp.ALGO_NEIGHBOR_EXCHANGE]
 
 
 def is_pow2(p):
@@ -40,6 +40,8 @@ def test_descriptors_expand_to_oracle_message_sets(algo):
     """Per phase, the library's messages equal the oracle's as a set (order inside a phase is free)."""
     for P in list(range(1, 41)) + [64, 100, 127, 128, 129, 255, 256]:
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
             continue
         if algo == sp.ALGO_RING and P > 64:
             continue
@@ -89,6 +91,7 @@ def test_plan_errors():
     assert lib.sparbit_plan_create(8, 16, 0, 0, None) == sp.ERR_ARG
     assert lib.sparbit_plan_create(6, 16, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     assert lib.sparbit_plan_create(13, 16, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create(7, 16, sp.ALGO_NEIGHBOR_EXCHANGE, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     assert lib.sparbit_plan_create(1 << 20, 1 << 40, 0, 0, ctypes.byref(out)) == sp.ERR_OVERFLOW
     assert lib.sparbit_plan_create((1 << 24) + 1, 1, 0, 0, ctypes.byref(out)) == sp.ERR_OVERFLOW
     assert lib.sparbit_plan(0, 16) is None
