@@ -451,6 +451,60 @@ def run_sweep(args):
     return 0
 
 
+def run_heatmap(args):
+    """Which algorithm is fastest for each (P, m) on this executor, in the style of the paper's
+    heat maps (Section IV): block sizes 1 B .. 1 MiB, P up to 256, powers of two and not, every
+    algorithm that is defined for the P, executor and engine chosen by the library (AUTO).
+    5 warm-ups + 50 timed collectives per cell; one JSON line per cell."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "ne": sp.ALGO_NEIGHBOR_EXCHANGE,
+             "rd": sp.ALGO_RECURSIVE_DOUBLING, "bruck": sp.ALGO_BRUCK}
+    stream = torch.cuda.Stream(device=dev)
+    free_bytes = torch.cuda.mem_get_info(dev)[0]
+    for P in (5, 8, 13, 16, 32, 61, 64, 128, 253, 256):
+        for m in (1, 8, 64, 512, 4096, 32768, 262144, 1048576):
+            if P * P * m * 2.2 + 2 * P * m > free_bytes:
+                continue
+            sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
+            recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+            work = torch.empty(P * P * m, dtype=torch.uint8, device=dev)
+            cell = {}
+            for name, a in algos.items():
+                if name == "rd" and P & (P - 1):
+                    continue
+                if name == "ne" and P % 2:
+                    continue
+                plan = sp.Plan(P, m, a, sp.EXEC_AUTO)
+                if name == "bruck":
+                    plan.set_workspace(work, P * P * m)
+                with torch.cuda.stream(stream):
+                    for it in range(5):
+                        plan.allgather(sends[it & 1], recv, stream)
+                    stream.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    for it in range(50):
+                        plan.allgather(sends[it & 1], recv, stream)
+                    e1.record(stream)
+                    stream.synchronize()
+                assert plan.status() == sp.OK
+                assert bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
+                cell[name] = round(e0.elapsed_time(e1) / 50 * 1e3, 2)
+                plan.destroy()
+            order = sorted(cell, key=cell.get)
+            best, second = order[0], order[1]
+            print(json.dumps({"P": P, "m": m, "us_avg": cell, "best": best,
+                              "gain_over_second_pct": round(100 * (cell[second] - cell[best]) / cell[second], 1)}),
+                  flush=True)
+            del sends, recv, work
+            torch.cuda.empty_cache()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -467,7 +521,11 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
+    ap.add_argument("--heatmap", action="store_true",
+                    help="best algorithm per (P, m) cell, one JSON line per cell")
     args = ap.parse_args()
+    if args.heatmap:
+        return run_heatmap(args)
     if args.sweep:
         return run_sweep(args)
     if args.warmup < 3:

@@ -275,6 +275,7 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
     const uint32_t chunk = (uint32_t)((((d.copy_bytes + cpc - 1) / cpc) + 127u) & ~127ull);
     fence_proxy_async_all();  // what other CTAs wrote before the barrier -> visible to bulk loads
     const uint64_t mine = (tasks - pipe_id + n_pipes - 1) / n_pipes;      // tasks of this ring
+    const bool small = (tasks >> 32) == 0;
     const char* sbase = space_base(g, d.src_space);
     char* dbase = space_base(g, d.dst_space);
     const uint64_t spitch = space_pitch(g, d.src_space);
@@ -289,10 +290,21 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
             // memory: stores are committed one group per task, L tasks behind the loads
             bulk_wait_read<S - L - 1>();
             const uint64_t w = pipe_id + i * n_pipes;
-            const uint64_t q = w / cpc;
-            const uint64_t ch = w - q * cpc;
-            const uint32_t r = (uint32_t)(q / d.copies);
-            const uint32_t j = (uint32_t)(q - (uint64_t)r * d.copies);
+            uint64_t q, ch;
+            uint32_t r, j;
+            if (small) {  // everything fits 32 bits: four cheap divisions instead of four long ones
+                const uint32_t w32 = (uint32_t)w, cpc32 = (uint32_t)cpc;
+                const uint32_t q32 = w32 / cpc32;
+                ch = w32 - q32 * cpc32;
+                r = q32 / d.copies;
+                j = q32 - r * d.copies;
+                q = q32;
+            } else {
+                q = w / cpc;
+                ch = w - q * cpc;
+                r = (uint32_t)(q / d.copies);
+                j = (uint32_t)(q - (uint64_t)r * d.copies);
+            }
             const CopyLoc c = locate_copy(d, P, r, j);
             const uint64_t off = ch * chunk;
             const uint64_t left = d.copy_bytes - off;
