@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (bytes; None = not captured for this workload)
 NCU_TRAFFIC_BYTES = {
-    # profiles/persistent_bulk_kernel_P256_m64k_traffic.md: 4.16 GB read + 4.25 GB written
+    # profiles/persistent_kernels_P256_m16k.md (full-size section): 4.16 GB read + 4.25 GB written
     "sparbit:P256:m65536:persistent:bulk": 8.41e9,
     # profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md: last phase, 2.15 GB read + 2.10 GB written
     "sparbit:P256:m65536:graph:bulk": 4.25e9,
@@ -52,8 +52,10 @@ def effective_bytes(P: int, m: int) -> int:
 
 
 def algorithmic_bytes(P: int, m: int) -> int:
-    """Bytes one collective must read plus write: every delivered block once each way, plus the
-    own-block copy."""
+    """Bytes one collective must read plus write: every delivered block written once and read
+    once, plus the own-block copy.  The library fuses that copy with the first step (sendbuf[r] is
+    read once and written to two places), which saves P*m of the 2*P*m a separate copy would
+    move; the saving is not credited here, so the figure is an upper bound on what is needed."""
     return 2 * P * (P - 1) * m + 2 * P * m
 
 
