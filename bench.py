@@ -51,12 +51,12 @@ def effective_bytes(P: int, m: int) -> int:
     return 2 * P * (P - 1) * m
 
 
-def algorithmic_bytes(P: int, m: int) -> int:
-    """Bytes one collective must read plus write: every delivered block written once and read
-    once, plus the own-block copy.  The library fuses that copy with the first step (sendbuf[r] is
-    read once and written to two places), which saves P*m of the 2*P*m a separate copy would
-    move; the saving is not credited here, so the figure is an upper bound on what is needed."""
-    return 2 * P * (P - 1) * m + 2 * P * m
+def algorithmic_bytes(P: int, m: int, fused_first: bool = True) -> int:
+    """Bytes one collective must read plus write: every delivered block is written once and read
+    once (2*P*(P-1)*m), and the own block gets into place.  With the own-block copy fused into the
+    first step (sendbuf[r] read once, written to two places; Sparbit, ring, neighbor exchange and
+    recursive doubling) that costs P*m more; as a separate copy (Bruck) it costs 2*P*m."""
+    return 2 * P * (P - 1) * m + (P * m if fused_first else 2 * P * m)
 
 
 def measured_peak():
@@ -322,7 +322,7 @@ def run_ours(args):
     one_kernel = launches_per_step <= 1
     if one_kernel:
         dom_ms = float(np.mean(per_ms))
-        dom_bytes = algorithmic_bytes(P, m)
+        dom_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
         dom_name = "whole collective in one kernel"
     else:
         last = plan.last_phase
@@ -343,6 +343,7 @@ def run_ours(args):
     if rank == 0:
         peak, peak_src = measured_peak()
         avg_ms = float(np.mean(per_ms))
+        path_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
         key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[plan.exec_mode]}:{sp.COPY_NAMES[plan.copy_path]}"
         roofline = {
@@ -351,9 +352,9 @@ def run_ours(args):
             "kernel": f"{sp.EXEC_NAMES[plan.exec_mode]} executor, {sp.COPY_NAMES[plan.copy_path]} engine: "
                       f"{dom_name} ({launches_per_step:g} launch(es) per collective)",
             "algorithmic_bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
-            "whole_path": {"algorithmic_bytes": algorithmic_bytes(P, m), "us": avg_ms * 1e3,
-                           "achieved": algorithmic_bytes(P, m) / (avg_ms * 1e-3) / 1e9,
-                           "frac": algorithmic_bytes(P, m) / (avg_ms * 1e-3) / 1e9 / peak},
+            "whole_path": {"algorithmic_bytes": path_bytes, "us": avg_ms * 1e3,
+                           "achieved": path_bytes / (avg_ms * 1e-3) / 1e9,
+                           "frac": path_bytes / (avg_ms * 1e-3) / 1e9 / peak},
         }
         cpu = None if args.no_cpu else cpu_baseline_leg(P, m, seed)
         line = {
