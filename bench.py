@@ -202,13 +202,16 @@ def run_reference(args):
     times, ok = time_oracle(P, ms, steps=args.steps, warmup=args.warmup, threads=threads, seed=args.seed)
     per = float(np.mean(times))
     value = effective_bytes(P, ms) / per / 1e9
-    sample = (f"each step = one whole collective P={P}, m={ms} B (block shrunk from {m} B to bound the run), "
+    shrunk = f" (block shrunk from {m} B to bound the run)" if ms != m else ""
+    sample = (f"each step = one whole collective P={P}, m={ms} B{shrunk}, "
               f"oracle execute phase on host buffers; box has {cores} cores")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": f"sparbit allgather P={P} m={m}B (sampled at m={ms}B)", "P": P, "block_bytes": ms},
+        "config": {"workload": f"sparbit allgather, P={P} virtual ranks, m={m} B blocks"
+                               + (f" (sampled at m={ms} B)" if ms != m else ""),
+                   "P": P, "block_bytes": ms, "algo": "sparbit"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "checked": ok,

@@ -32,7 +32,8 @@
  * returning int return SPARBIT_OK (0) or a positive SPARBIT_ERR_* code.  Nothing here
  * synchronises the device unless its comment says so.  All argument errors are found on the
  * host before anything is launched.  A plan may be used by one host thread and on one stream at
- * a time.
+ * a time, and belongs to the device that was current at its first launch (later calls with
+ * another device current return SPARBIT_ERR_ARG).
  */
 #ifndef SPARBIT_H
 #define SPARBIT_H
@@ -68,19 +69,22 @@ enum {
     SPARBIT_ALGO_NEIGHBOR_EXCHANGE = 4   /* even P only, as the paper states */
 };
 
-/* How the phases are put on the GPU. */
+/* How the phases are put on the GPU.  When a call runs phases -1 and 0 together they are executed
+ * as ONE pass (the own block is read once from sendbuf and written both to its own slot and to
+ * the first peer's): same state after phase 0, one pass less. */
 enum {
-    SPARBIT_EXEC_AUTO = 0,       /* chosen from P and m */
-    SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per phase */
-    SPARBIT_EXEC_GRAPH = 2,      /* one kernel per phase, chained in a cached CUDA graph */
-    SPARBIT_EXEC_STREAM = 3,     /* one kernel per phase, launched one by one on the stream */
-    SPARBIT_EXEC_CLUSTER = 4     /* one thread-block cluster, hardware cluster barrier per phase;
-                                    for collectives small enough to be latency-bound */
+    SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: the graph chain, at every size */
+    SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
+    SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
+                                    in a CUDA graph cached per buffer set (4 sets; further sets
+                                    re-parameterise the least recently used graph) */
+    SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
+    SPARBIT_EXEC_CLUSTER = 4     /* one thread-block cluster, hardware cluster barrier per pass */
 };
 
 /* Which copy engine a phase uses. */
 enum {
-    SPARBIT_COPY_AUTO = 0,   /* chosen from m and the alignment of the buffers */
+    SPARBIT_COPY_AUTO = 0,   /* BULK for 16-byte aligned buffers and m >= 32 KiB, else VECTOR */
     SPARBIT_COPY_VECTOR = 1, /* warp-cooperative ld/st.global, 16/8/4/2/1-byte vectors */
     SPARBIT_COPY_BULK = 2    /* cp.async.bulk global->shared->global ring (needs 16-byte
                                 alignment of buffers and m); falls back to VECTOR otherwise */

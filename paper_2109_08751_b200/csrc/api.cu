@@ -57,6 +57,7 @@ struct sparbit_plan_s {
 
     // device side, created by the first launch
     bool dev_ready = false;
+    bool dev_touched = false;  // set-up was attempted: something may have been allocated
     int device = -1;
     int sm_count = 0;
     int coop = 0;
@@ -112,7 +113,13 @@ size_t bulk_smem_bytes(const sparbit_plan_s* p) {
 }
 
 int ensure_device(sparbit_plan_s* p) {
-    if (p->dev_ready) return SPARBIT_OK;
+    if (p->dev_ready) {
+        // a plan belongs to the device of its first launch
+        int cur = -1;
+        CU(cudaGetDevice(&cur));
+        return cur == p->device ? SPARBIT_OK : SPARBIT_ERR_ARG;
+    }
+    p->dev_touched = true;
     CU(cudaGetDevice(&p->device));
     CU(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
     CU(cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device));
@@ -621,7 +628,7 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes) {
 int sparbit_plan_destroy(sparbit_plan_t* p) {
     if (!p) return SPARBIT_OK;
     int rc = SPARBIT_OK;
-    if (p->dev_ready) {
+    if (p->dev_touched || p->stage_send || p->stage_recv || p->stage_work) {
         if (p->launched && cudaDeviceSynchronize() != cudaSuccess) rc = SPARBIT_ERR_CUDA;
         drop_graph(p);
         if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
