@@ -457,6 +457,62 @@ def run_sweep(args):
     return 0
 
 
+def run_allgatherv(args):
+    """Blocks of different sizes on the Sparbit schedule (P = 256, about 64 KiB per block on
+    average): equal sizes through the variable-size path, uniformly drawn sizes, and a mix with
+    empty and several-times-larger blocks.  Effective bytes = 2*(P-1)*sum(counts)."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peak()
+    P = args.P
+    cases = {
+        "equal (fixed-size plan)": None,
+        "equal (variable-size plan)": [args.m] * P,
+        "uniform 0..2m": si.block_counts(P, args.seed, kind="uniform", unit=16, scale=args.m // 16),
+        "mixed (1/8 empty, 1/8 six-fold)": si.block_counts(P, args.seed, kind="mixed", unit=16,
+                                                            scale=args.m // 16 * 8 // 13),
+    }
+    stream = torch.cuda.Stream(device=dev)
+    for name, counts in cases.items():
+        if counts is None:
+            plan = sp.Plan(P, args.m)
+            T = P * args.m
+            host = [si.send_blocks(P, args.m, args.seed + k).reshape(-1) for k in range(2)]
+        else:
+            plan = sp.Plan.create_v(counts)
+            T = sum(counts)
+            host = [si.send_blocks_v(counts, args.seed + k) for k in range(2)]
+        sends = [torch.from_numpy(h).to(dev) for h in host]
+        recv = torch.full((P * T,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        with torch.cuda.stream(stream):
+            for it in range(5):
+                plan.allgather(sends[it & 1], recv, stream)
+            stream.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
+            ev[0].record(stream)
+            for it in range(50):
+                plan.allgather(sends[it & 1], recv, stream)
+                ev[it + 1].record(stream)
+            stream.synchronize()
+        assert plan.status() == sp.OK
+        ok = bool(torch.equal(recv.view(P, T)[P - 1], sends[1]))
+        us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(50)]
+        avg = float(np.mean(us))
+        eff = 2 * (P - 1) * T
+        print(json.dumps({"case": name, "P": P, "total_bytes_per_rank": T,
+                          "max_block": max(counts) if counts else args.m,
+                          "us_min": round(min(us), 1), "us_avg": round(avg, 1), "us_max": round(max(us), 1),
+                          "GBps_avg": round(eff / avg / 1e3, 1),
+                          "pct_measured_peak": round(100 * eff / avg / 1e3 / peak, 1), "checked": ok}), flush=True)
+        plan.destroy()
+        del sends, recv
+        torch.cuda.empty_cache()
+    return 0
+
+
 def run_heatmap(args):
     """Which algorithm is fastest for each (P, m) on this executor, in the style of the paper's
     heat maps (Section IV): block sizes 1 B .. 1 MiB, P up to 256, powers of two and not, every
@@ -529,7 +585,11 @@ def main():
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     ap.add_argument("--heatmap", action="store_true",
                     help="best algorithm per (P, m) cell, one JSON line per cell")
+    ap.add_argument("--allgatherv", action="store_true",
+                    help="variable block sizes on the Sparbit schedule, one JSON line per size mix")
     args = ap.parse_args()
+    if args.allgatherv:
+        return run_allgatherv(args)
     if args.heatmap:
         return run_heatmap(args)
     if args.sweep:

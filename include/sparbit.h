@@ -127,6 +127,24 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
  */
 int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out);
 
+/*
+ * sparbit_plan_create_v - a plan for blocks of DIFFERENT sizes, i.e. MPI_Allgatherv with
+ * contiguous displacements, on the same schedules (the paper's Section VII names Allgatherv as
+ * the next target; the schedules themselves never look inside a block, so they carry over
+ * unchanged).  block_bytes: host array of P byte counts, block_bytes[j] = what rank j
+ * contributes (0 allowed); it is copied.  With T = the sum of the counts and off[j] = the sum
+ * of the counts below j:
+ *   sendbuf   T bytes       rank r's block at byte offset off[r]
+ *   recvbuf   P * T bytes   rank r's buffer at r * T, block j at + off[j]
+ * The plan is then used with sparbit_allgather, sparbit_allgather_steps and
+ * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Runs on the
+ * vector copy engine with the graph or stream executor: exec must be AUTO, GRAPH or STREAM
+ * (PERSISTENT, CLUSTER: ERR_UNSUPPORTED).  Bruck is refused (ERR_UNSUPPORTED: its rotated
+ * workspace assumes equal blocks).  Other errors as for sparbit_plan_create; P is limited to
+ * 65536 here.  Host-only.
+ */
+int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, sparbit_plan_t** out);
+
 /* Releases the plan and everything it owns (device table, graph).  Synchronises the device if
  * the plan ever launched work.  NULL is allowed. */
 int sparbit_plan_destroy(sparbit_plan_t* plan);

@@ -67,6 +67,8 @@ def _load():
         lib.oracle_plan_messages.argtypes = [ctypes.c_void_p]
         lib.oracle_run.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p,
                                    ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        lib.oracle_run_v.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_int, ctypes.c_int, ctypes.c_int]
         _lib = lib
     return _lib
 
@@ -118,6 +120,23 @@ class Plan:
             sp = scratch.ctypes.data
         lib = _load()
         rc = lib.oracle_run(self._h, m, send.ctypes.data, recv.ctypes.data, sp, first, last, threads)
+        if rc:
+            raise OracleError(lib.oracle_last_error().decode())
+
+    def run_v(self, counts, send: np.ndarray, recv: np.ndarray, first: int = -1, last: int | None = None,
+              threads: int = 1) -> None:
+        """Allgatherv: blocks of counts[j] bytes, contiguous displacements (see oracle_run_v)."""
+        P = self.P
+        off = np.zeros(P + 1, dtype=np.uint64)
+        off[1:] = np.cumsum(np.asarray(counts, dtype=np.uint64))
+        T = int(off[P])
+        if last is None:
+            last = self.last_phase
+        for name, buf, need in (("send", send, T), ("recv", recv, P * T)):
+            if buf.dtype != np.uint8 or not buf.flags.c_contiguous or buf.size != need:
+                raise ValueError(f"{name} must be contiguous uint8 of {need} bytes")
+        lib = _load()
+        rc = lib.oracle_run_v(self._h, off.ctypes.data, send.ctypes.data, recv.ctypes.data, first, last, threads)
         if rc:
             raise OracleError(lib.oracle_last_error().decode())
 

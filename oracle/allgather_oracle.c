@@ -574,6 +574,7 @@ int oracle_plan_phase_range(const oracle_plan *pl, int phase, size_t *begin, siz
 typedef struct {
     const oracle_plan *pl;
     size_t m;
+    const uint64_t *off; /* allgatherv: P+1 prefix sums of the blocks' byte counts, else NULL */
     const uint8_t *send;
     uint8_t *recv;
     uint8_t *scratch;
@@ -584,6 +585,11 @@ typedef struct {
 
 static uint8_t *locate(const exec_arg *a, int space, int rank, int slot) {
     const size_t P = (size_t)a->pl->P;
+    if (a->off) { /* block b is off[b+1]-off[b] bytes, at off[b] in the send buffer and in every
+                     receive buffer (each receive buffer is off[P] bytes) */
+        if (space == SPACE_SEND) return (uint8_t *)a->send + a->off[rank];
+        return a->recv + (size_t)rank * a->off[P] + a->off[slot];
+    }
     switch (space) {
         case SPACE_SEND: return (uint8_t *)a->send + (size_t)rank * a->m;
         case SPACE_RECV: return a->recv + ((size_t)rank * P + (size_t)slot) * a->m;
@@ -600,8 +606,10 @@ static void *exec_thread(void *vp) {
         size_t hi = b + n * ((size_t)a->tid + 1) / (size_t)a->nthreads;
         for (size_t k = lo; k < hi; k++) {
             const oracle_msg *m = &a->pl->msgs[k];
+            /* the block a message carries is the one whose final slot it is written to */
+            size_t bytes = a->off ? (size_t)(a->off[m->dst_slot + 1] - a->off[m->dst_slot]) : a->m;
             memcpy(locate(a, m->dst_space, m->dst_rank, m->dst_slot),
-                   locate(a, m->src_space, m->src_rank, m->src_slot), a->m);
+                   locate(a, m->src_space, m->src_rank, m->src_slot), bytes);
         }
         if (a->bar) pthread_barrier_wait(a->bar); /* the step's Waitall */
     }
@@ -615,8 +623,36 @@ static void *exec_thread(void *vp) {
  * threads >= 1; messages of a phase are split evenly between threads (their writes are disjoint,
  * which check_plan proved), with a barrier after every phase.
  */
+static int run_impl(const oracle_plan *pl, size_t m, const uint64_t *off, const void *send, void *recv,
+                    void *scratch, int first, int last, int threads);
+
 int oracle_run(const oracle_plan *pl, size_t m, const void *send, void *recv, void *scratch,
                int first, int last, int threads) {
+    return run_impl(pl, m, NULL, send, recv, scratch, first, last, threads);
+}
+
+/*
+ * The same phases for blocks of different sizes (MPI_Allgatherv with contiguous displacements;
+ * the paper's conclusion names it as the next target, and the schedules never look inside a
+ * block).  off: P+1 prefix sums of the byte counts.  send: off[P] bytes, rank r's block at off[r].
+ * recv: P * off[P] bytes, rank r's buffer at r * off[P], block j at + off[j].  Not for Bruck (its
+ * rotated working buffer is laid out for equal blocks).
+ */
+int oracle_run_v(const oracle_plan *pl, const uint64_t *off, const void *send, void *recv, int first,
+                 int last, int threads) {
+    if (!pl || !off) {
+        set_err("null argument");
+        return -1;
+    }
+    if (pl->algo == ORACLE_BRUCK) {
+        set_err("Bruck is laid out for equal blocks");
+        return -1;
+    }
+    return run_impl(pl, off[pl->P] ? 1 : 0, off, send, recv, NULL, first, last, threads);
+}
+
+static int run_impl(const oracle_plan *pl, size_t m, const uint64_t *off, const void *send, void *recv,
+                    void *scratch, int first, int last, int threads) {
     if (!pl) {
         set_err("null plan");
         return -1;
@@ -631,7 +667,7 @@ int oracle_run(const oracle_plan *pl, size_t m, const void *send, void *recv, vo
     }
     if (threads < 1) threads = 1;
     if (threads == 1) {
-        exec_arg a = {pl, m, (const uint8_t *)send, (uint8_t *)recv, (uint8_t *)scratch,
+        exec_arg a = {pl, m, off, (const uint8_t *)send, (uint8_t *)recv, (uint8_t *)scratch,
                       first, last, 0, 1, NULL};
         exec_thread(&a);
         return 0;
@@ -647,7 +683,7 @@ int oracle_run(const oracle_plan *pl, size_t m, const void *send, void *recv, vo
         return -1;
     }
     for (int t = 0; t < threads; t++) {
-        exec_arg a = {pl, m, (const uint8_t *)send, (uint8_t *)recv, (uint8_t *)scratch,
+        exec_arg a = {pl, m, off, (const uint8_t *)send, (uint8_t *)recv, (uint8_t *)scratch,
                       first, last, t, threads, &bar};
         args[t] = a;
         pthread_create(&th[t], NULL, exec_thread, &args[t]);

@@ -35,6 +35,7 @@ _pi = ctypes.POINTER(ctypes.c_int)
 SYMBOLS = {
     "sparbit_plan": (_vp, [_i, _sz]),
     "sparbit_plan_create": (_i, [_i, _sz, _i, _i, ctypes.POINTER(_vp)]),
+    "sparbit_plan_create_v": (_i, [_i, ctypes.POINTER(_sz), _i, _i, ctypes.POINTER(_vp)]),
     "sparbit_plan_destroy": (_i, [_vp]),
     "sparbit_allgather": (_i, [_vp, _vp, _vp, _vp]),
     "sparbit_allgather_steps": (_i, [_vp, _vp, _vp, _vp, _i, _i]),
@@ -109,6 +110,21 @@ class Plan:
         self._h = h
         self.P, self.block_bytes, self.algo = P, block_bytes, algo
         self._workspace = None
+
+    @classmethod
+    def create_v(cls, block_bytes, algo: int = ALGO_SPARBIT, exec_mode: int = EXEC_AUTO) -> "Plan":
+        """A plan for blocks of different sizes (sparbit_plan_create_v): block_bytes[j] is the
+        byte count rank j contributes."""
+        counts = [int(x) for x in block_bytes]
+        arr = (_sz * len(counts))(*counts)
+        h = _vp()
+        _check(lib.sparbit_plan_create_v(len(counts), arr, algo, exec_mode, ctypes.byref(h)),
+               "sparbit_plan_create_v")
+        self = cls.__new__(cls)
+        self._h = h
+        self.P, self.block_bytes, self.algo = len(counts), counts, algo
+        self._workspace = None
+        return self
 
     # -- the collective
     def allgather(self, sendbuf, recvbuf, stream=None) -> None:

@@ -55,6 +55,15 @@ struct sparbit_plan_s {
     void* work = nullptr;
     size_t work_bytes = 0;
 
+    // variable block sizes (allgatherv): prefix sums of the byte counts, P+1 entries
+    bool variable = false;
+    std::vector<uint64_t> voff;
+    uintptr_t voff_bits = 0;  // OR of all prefix sums: decides the vector width
+    uint64_t* d_voff = nullptr;
+
+    size_t send_bytes() const { return variable ? (size_t)voff.back() : (size_t)sched.P * sched.m; }
+    size_t recv_bytes() const { return (size_t)sched.P * send_bytes(); }
+
     // device side, created by the first launch
     bool dev_ready = false;
     bool dev_touched = false;  // set-up was attempted: something may have been allocated
@@ -139,6 +148,10 @@ int ensure_device(sparbit_plan_s* p) {
     const size_t n = table.size();
     CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
     CU(cudaMemcpy(p->d_descs, table.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
+    if (p->variable) {
+        CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
+        CU(cudaMemcpy(p->d_voff, p->voff.data(), p->voff.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
+    }
     CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
     CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -157,7 +170,8 @@ bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
 
 // largest power-of-two vector width (<= 16) that divides every address and m
 int pick_vector_bytes(const sparbit_plan_s* p, const void* send, const void* recv) {
-    uintptr_t bits = (uintptr_t)send | (uintptr_t)recv | (uintptr_t)p->sched.m;
+    uintptr_t bits = (uintptr_t)send | (uintptr_t)recv;
+    bits |= p->variable ? p->voff_bits : (uintptr_t)p->sched.m;
     if (p->sched.algo == ALGO_BRUCK) bits |= (uintptr_t)p->work;
     int v = 16;
     while (v > 1 && (bits & (uintptr_t)(v - 1))) v >>= 1;
@@ -183,7 +197,7 @@ uint64_t bulk_tasks(const PhaseDesc& d, uint32_t P, uint32_t stage_bytes) {
 }
 
 template <typename V>
-const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V>; }
+const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V, false>; }
 template <typename V>
 const void* persistent_vec_fn() { return (const void*)persistent_vec_kernel<V>; }
 
@@ -194,6 +208,17 @@ const void* pick_phase_vec(int vbytes) {
         case 4: return phase_vec_fn<unsigned>();
         case 2: return phase_vec_fn<unsigned short>();
         default: return phase_vec_fn<unsigned char>();
+    }
+}
+template <typename V>
+const void* phase_vec_var_fn() { return (const void*)phase_vec_kernel<V, true>; }
+const void* pick_phase_vec_var(int vbytes) {
+    switch (vbytes) {
+        case 16: return phase_vec_var_fn<uint4>();
+        case 8: return phase_vec_var_fn<uint2>();
+        case 4: return phase_vec_var_fn<unsigned>();
+        case 2: return phase_vec_var_fn<unsigned short>();
+        default: return phase_vec_var_fn<unsigned char>();
     }
 }
 const void* pick_persistent_vec(int vbytes) {
@@ -248,6 +273,7 @@ Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv) {
     if (copy == SPARBIT_COPY_AUTO)
         copy = (bulk_possible && m >= (32u << 10)) ? SPARBIT_COPY_BULK : SPARBIT_COPY_VECTOR;
     if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
+    if (p->variable) copy = SPARBIT_COPY_VECTOR;  // variable block sizes run on the vector engine
     r.copy = copy;
     int exec = p->exec_req;
     if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p->sched, p->coop != 0, p->cluster_ok != 0);
@@ -271,6 +297,14 @@ Geom make_geom(const sparbit_plan_s* p, const void* send, void* recv) {
     g.rank_pitch[SPACE_SEND] = g.m;
     g.rank_pitch[SPACE_RECV] = (uint64_t)g.P * g.m;
     g.rank_pitch[SPACE_WORK] = (uint64_t)g.P * g.m;
+    g.voff = nullptr;
+    if (p->variable) {
+        g.m = 0;
+        g.rank_pitch[SPACE_SEND] = 0;                 // send blocks sit at voff[rank]
+        g.rank_pitch[SPACE_RECV] = p->voff.back();    // every receive buffer holds all blocks
+        g.rank_pitch[SPACE_WORK] = 0;
+        g.voff = p->d_voff;
+    }
     return g;
 }
 
@@ -327,7 +361,7 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         const uint64_t cap = (uint64_t)p->sm_count * 2;  // 1024 threads x 2 vectors in flight per SM
         if (ctas > cap) ctas = cap;
         if (ctas < 1) ctas = 1;
-        pl.fn = pick_phase_vec(rs.vbytes);
+        pl.fn = p->variable ? pick_phase_vec_var(rs.vbytes) : pick_phase_vec(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
         pl.smem = 0;
@@ -565,8 +599,8 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
     if (!p) return SPARBIT_ERR_ARG;
     const Schedule& s = p->sched;
     if (first < -1 || last > s.last_phase() || first > last) return SPARBIT_ERR_ARG;
-    const size_t send_bytes = (size_t)s.P * s.m;
-    const size_t recv_bytes = (size_t)s.P * s.P * s.m;
+    const size_t send_bytes = p->send_bytes();
+    const size_t recv_bytes = p->recv_bytes();
     if (send_bytes == 0) return SPARBIT_OK;  // count 0: nothing to do
     if (!send || !recv) return SPARBIT_ERR_ARG;
     if (s.algo == ALGO_BRUCK && (!p->work || p->work_bytes < recv_bytes)) return SPARBIT_ERR_WORKSPACE;
@@ -619,6 +653,62 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
     return SPARBIT_OK;
 }
 
+int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, sparbit_plan_t** out) {
+    if (!out) return SPARBIT_ERR_ARG;
+    *out = nullptr;
+    if (!block_bytes || P < 1) return SPARBIT_ERR_ARG;
+    if (P > (1 << 16)) return SPARBIT_ERR_OVERFLOW;
+    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
+    if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // rotated workspace: fixed sizes only
+    if (exec != SPARBIT_EXEC_AUTO && exec != SPARBIT_EXEC_GRAPH && exec != SPARBIT_EXEC_STREAM) {
+        if (exec == SPARBIT_EXEC_PERSISTENT || exec == SPARBIT_EXEC_CLUSTER) return SPARBIT_ERR_UNSUPPORTED;
+        return SPARBIT_ERR_ARG;
+    }
+    sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
+    if (!p) return SPARBIT_ERR_NOMEM;
+    int rc;
+    try {
+        rc = map_sched_err(build_schedule(algo, P, 1, p->sched));
+        if (rc == SPARBIT_OK) {
+            p->variable = true;
+            p->voff.assign((size_t)P + 1, 0);
+            unsigned __int128 total = 0;
+            for (int b = 0; b < P; b++) {
+                total += block_bytes[b];
+                if (total >> 62) rc = SPARBIT_ERR_OVERFLOW;
+                p->voff[(size_t)b + 1] = (uint64_t)total;
+                p->voff_bits |= (uintptr_t)p->voff[(size_t)b + 1];
+            }
+            if ((total * (unsigned)P) >> 62) rc = SPARBIT_ERR_OVERFLOW;
+        }
+        if (rc == SPARBIT_OK) {
+            // the task grid of a phase is laid out for its largest copy
+            auto set_max = [&](PhaseDesc& d) {
+                uint64_t mx = 0;
+                for (uint32_t r = 0; r < p->sched.P; r++)
+                    for (uint32_t j = 0; j < d.copies; j++) {
+                        const CopyLoc c = locate_copy(d, p->sched.P, r, j);
+                        const uint64_t b = p->voff[c.dst_slot + d.run] - p->voff[c.dst_slot];
+                        if (b > mx) mx = b;
+                    }
+                d.copy_bytes = mx;
+            };
+            for (PhaseDesc& d : p->sched.phases) set_max(d);
+            if (p->sched.has_fused_first) set_max(p->sched.fused_first);
+            p->sched.m = 0;
+        }
+    } catch (const std::bad_alloc&) {
+        rc = SPARBIT_ERR_NOMEM;
+    }
+    if (rc) {
+        delete p;
+        return rc;
+    }
+    p->exec_req = exec;
+    *out = p;
+    return SPARBIT_OK;
+}
+
 sparbit_plan_t* sparbit_plan(int P, size_t block_bytes) {
     sparbit_plan_t* p = nullptr;
     if (sparbit_plan_create(P, block_bytes, SPARBIT_ALGO_SPARBIT, SPARBIT_EXEC_AUTO, &p) != SPARBIT_OK) return nullptr;
@@ -633,6 +723,7 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
         drop_graph(p);
         if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
         cudaFree(p->d_descs);
+        cudaFree(p->d_voff);
         cudaFree(p->d_ctl);
         cudaFree(p->stage_send);
         cudaFree(p->stage_recv);
@@ -657,8 +748,8 @@ int sparbit_allgather_steps(sparbit_plan_t* p, const void* sendbuf, void* recvbu
 int sparbit_allgather_host(sparbit_plan_t* p, const void* host_send, void* host_recv) {
     if (!p) return SPARBIT_ERR_ARG;
     const Schedule& s = p->sched;
-    const size_t send_bytes = (size_t)s.P * s.m;
-    const size_t recv_bytes = (size_t)s.P * s.P * s.m;
+    const size_t send_bytes = p->send_bytes();
+    const size_t recv_bytes = p->recv_bytes();
     if (send_bytes == 0) return SPARBIT_OK;
     if (!host_send || !host_recv) return SPARBIT_ERR_ARG;
     if (ranges_overlap(host_send, send_bytes, host_recv, recv_bytes)) return SPARBIT_ERR_ALIAS;

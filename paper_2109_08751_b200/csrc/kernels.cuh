@@ -148,12 +148,43 @@ __device__ __forceinline__ void st_cg<unsigned char>(unsigned char* p, unsigned 
 
 // One phase on the vector engine.  warp_id / n_warps enumerate all warps taking part.
 // Requires P * copies * ceil(vectors_per_copy / (32*U)) < 2^32 (checked on the host).
-template <typename V>
+//
+// kVar = true is the variable-block-size form (allgatherv): d.copy_bytes is then the LARGEST copy
+// of the phase and fixes the task grid; each copy's own size and position come from g.voff.
+template <bool kVar>
+struct CopyBytes {
+    uint64_t src, dst, dst2;  // byte offsets inside the source / destination space
+    uint64_t vectors;         // vectors this copy really has
+};
+
+template <typename V, bool kVar>
+__device__ __forceinline__ CopyBytes<kVar> copy_bytes_of(const Geom& g, const PhaseDesc& d, const CopyLoc& c,
+                                                         uint32_t r, uint64_t spitch, uint64_t dpitch,
+                                                         uint64_t uniform_vectors) {
+    CopyBytes<kVar> o;
+    if constexpr (kVar) {
+        const uint64_t lo = __ldg(g.voff + c.dst_slot);
+        const uint64_t hi = __ldg(g.voff + c.dst_slot + d.run);
+        o.vectors = (hi - lo) / sizeof(V);
+        o.src = d.src_space == SPACE_SEND ? __ldg(g.voff + c.src_rank)
+                                          : (uint64_t)c.src_rank * spitch + __ldg(g.voff + c.src_slot);
+        o.dst = (uint64_t)c.dst_rank * dpitch + lo;
+        o.dst2 = (uint64_t)r * dpitch + lo;
+    } else {
+        o.vectors = uniform_vectors;
+        o.src = (uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m;
+        o.dst = (uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m;
+        o.dst2 = (uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m;
+    }
+    return o;
+}
+
+template <typename V, bool kVar = false>
 __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uint32_t warp_id, uint32_t n_warps,
                                           uint32_t lane) {
     constexpr int U = kVecUnroll;
     const uint32_t P = g.P;
-    const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy
+    const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy (of the largest copy if kVar)
     const uint32_t n_copies = P * d.copies;            // copies in the phase (< 2^32, host-checked)
     const char* sbase = space_base(g, d.src_space);
     char* dbase = space_base(g, d.dst_space);
@@ -172,20 +203,21 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
             const uint32_t r = q / d.copies;
             const uint32_t j = q - r * d.copies;
             const CopyLoc c = locate_copy(d, P, r, j);
-            const V* src = reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
-            V* dst = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m));
-            V* dst2 = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m));
+            const CopyBytes<kVar> cb = copy_bytes_of<V, kVar>(g, d, c, r, spitch, dpitch, vpc64);
+            const V* src = reinterpret_cast<const V*>(sbase + cb.src);
+            V* dst = reinterpret_cast<V*>(dbase + cb.dst);
+            V* dst2 = reinterpret_cast<V*>(dbase + cb.dst2);
             const uint64_t v0 = (uint64_t)sp * span + lane;
             V regs[U];
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t v = v0 + 32u * k;
-                if (v < vpc64) regs[k] = ld_cg<V>(src + v);
+                if (v < cb.vectors) regs[k] = ld_cg<V>(src + v);
             }
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t v = v0 + 32u * k;
-                if (v < vpc64) {
+                if (v < cb.vectors) {
                     st_cg<V>(dst + v, regs[k]);
                     if (d.dup_self) st_cg<V>(dst2 + v, regs[k]);
                 }
@@ -213,11 +245,12 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
                     const uint32_t r = q / d.copies;
                     const uint32_t j = q - r * d.copies;
                     const CopyLoc c = locate_copy(d, P, r, j);
-                    const V* src =
-                        reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
-                    dsts[k] = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
-                    dsts2[k] = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
-                    regs[k] = ld_cg<V>(src + v);
+                    const CopyBytes<kVar> cb = copy_bytes_of<V, kVar>(g, d, c, r, spitch, dpitch, vpc64);
+                    if (v < cb.vectors) {
+                        dsts[k] = reinterpret_cast<V*>(dbase + cb.dst) + v;
+                        dsts2[k] = reinterpret_cast<V*>(dbase + cb.dst2) + v;
+                        regs[k] = ld_cg<V>(reinterpret_cast<const V*>(sbase + cb.src) + v);
+                    }
                 }
             }
 #pragma unroll
@@ -398,12 +431,12 @@ __device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& ep
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// one phase, vector engine
-template <typename V>
+// one phase, vector engine (kVar: variable block sizes)
+template <typename V, bool kVar = false>
 __global__ void __launch_bounds__(512, 2) phase_vec_kernel(Geom g, PhaseDesc d) {
     chain_wait();
     const uint32_t wpb = blockDim.x >> 5;
-    vec_phase<V>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
+    vec_phase<V, kVar>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
     chain_trigger();
 }
 

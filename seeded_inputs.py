@@ -57,6 +57,36 @@ def send_blocks(P: int, m: int, seed: int) -> np.ndarray:
     return out
 
 
+def send_blocks_v(counts, seed: int) -> np.ndarray:
+    """Concatenated send blocks of different sizes: rank r contributes counts[r] bytes, taken
+    from the same per-rank word stream as send_blocks."""
+    counts = [int(c) for c in counts]
+    out = np.empty(sum(counts), dtype=np.uint8)
+    pos = 0
+    for r, c in enumerate(counts):
+        if c:
+            words = (c + 3) // 4
+            key = np.uint64(seed & 0xFFFFFFFFFFFFFFFF) ^ ((np.uint64(r) << np.uint64(32))
+                                                           | np.arange(words, dtype=np.uint64))
+            w32 = (splitmix64(key) & np.uint64(0xFFFFFFFF)).astype("<u4")
+            out[pos:pos + c] = w32.view(np.uint8)[:c]
+        pos += c
+    return out
+
+
+def block_counts(P: int, seed: int, kind: str = "mixed", unit: int = 16, scale: int = 64) -> list:
+    """Seeded per-rank byte counts for allgatherv runs: multiples of `unit`, about `scale` units
+    on average; "mixed" includes empty blocks and a few large ones."""
+    key = np.uint64(seed & 0xFFFFFFFFFFFFFFFF) + np.arange(P, dtype=np.uint64)
+    h = splitmix64(key)
+    base = (h % np.uint64(2 * scale + 1)).astype(np.int64)
+    if kind == "mixed":
+        sel = ((h >> np.uint64(40)) % np.uint64(8)).astype(np.int64)
+        base = np.where(sel == 0, 0, base)            # one in eight is empty
+        base = np.where(sel == 1, base * 6, base)     # one in eight is several times larger
+    return [int(b) * unit for b in base]
+
+
 def sentinel_buffer(nbytes: int, value: int = SENTINEL) -> np.ndarray:
     """A uint8 buffer of nbytes filled with the sentinel byte."""
     return np.full(nbytes, value, dtype=np.uint8)
