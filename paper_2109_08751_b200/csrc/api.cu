@@ -60,6 +60,11 @@ struct sparbit_plan_s {
     std::vector<uint64_t> voff;
     uintptr_t voff_bits = 0;  // OR of all prefix sums: decides the vector width
     uint64_t* d_voff = nullptr;
+    // task lists of the variable-size kernels, one per descriptor of the device table order
+    // (phases in order, then the fused first pass): entries, and where each list starts
+    std::vector<unsigned long long> vtasks;
+    std::vector<size_t> vtask_lo, vtask_hi;  // per device-table index: [lo, hi) inside vtasks
+    unsigned long long* d_vtasks = nullptr;
 
     size_t send_bytes() const { return variable ? (size_t)voff.back() : (size_t)sched.P * sched.m; }
     size_t recv_bytes() const { return (size_t)sched.P * send_bytes(); }
@@ -151,6 +156,11 @@ int ensure_device(sparbit_plan_s* p) {
     if (p->variable) {
         CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
         CU(cudaMemcpy(p->d_voff, p->voff.data(), p->voff.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
+        const size_t nt = p->vtasks.size() ? p->vtasks.size() : 1;
+        CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(unsigned long long)));
+        if (p->vtasks.size())
+            CU(cudaMemcpy(p->d_vtasks, p->vtasks.data(), p->vtasks.size() * sizeof(unsigned long long),
+                          cudaMemcpyHostToDevice));
     }
     CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
@@ -197,7 +207,7 @@ uint64_t bulk_tasks(const PhaseDesc& d, uint32_t P, uint32_t stage_bytes) {
 }
 
 template <typename V>
-const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V, false>; }
+const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V>; }
 template <typename V>
 const void* persistent_vec_fn() { return (const void*)persistent_vec_kernel<V>; }
 
@@ -211,7 +221,7 @@ const void* pick_phase_vec(int vbytes) {
     }
 }
 template <typename V>
-const void* phase_vec_var_fn() { return (const void*)phase_vec_kernel<V, true>; }
+const void* phase_vec_var_fn() { return (const void*)phase_vec_list_kernel<V>; }
 const void* pick_phase_vec_var(int vbytes) {
     switch (vbytes) {
         case 16: return phase_vec_var_fn<uint4>();
@@ -342,8 +352,21 @@ struct PhaseLaunch {
     size_t smem;
 };
 
-int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d, PhaseLaunch& pl) {
+int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d, PhaseLaunch& pl,
+                      uint64_t var_tasks = 0) {
     const uint32_t P = p->sched.P;
+    if (p->variable) {
+        const uint64_t wpb = kVecBlock / 32;
+        uint64_t ctas = (var_tasks + wpb - 1) / wpb;
+        const uint64_t cap = (uint64_t)p->sm_count * 2;
+        if (ctas > cap) ctas = cap;
+        if (ctas < 1) ctas = 1;
+        pl.fn = pick_phase_vec_var(rs.vbytes);
+        pl.grid = dim3((unsigned)ctas);
+        pl.block = dim3(kVecBlock);
+        pl.smem = 0;
+        return SPARBIT_OK;
+    }
     if (rs.copy == SPARBIT_COPY_BULK) {
         const uint64_t tasks = bulk_tasks(d, P, p->bulk_stage_bytes);
         uint64_t ctas = (tasks + p->bulk_warps - 1) / p->bulk_warps;
@@ -361,7 +384,7 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         const uint64_t cap = (uint64_t)p->sm_count * 2;  // 1024 threads x 2 vectors in flight per SM
         if (ctas > cap) ctas = cap;
         if (ctas < 1) ctas = 1;
-        pl.fn = p->variable ? pick_phase_vec_var(rs.vbytes) : pick_phase_vec(rs.vbytes);
+        pl.fn = pick_phase_vec(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
         pl.smem = 0;
@@ -375,11 +398,16 @@ struct PhaseArgs {
     uint32_t stage_bytes;
     unsigned* status;
     unsigned long long timeout_ns;
+    const unsigned long long* list;  // variable block sizes: this pass's task list
+    unsigned long long count;
     void* ptrs[5];
-    void fill(bool bulk) {
+    void fill(bool bulk, bool variable = false) {
         ptrs[0] = &g;
         ptrs[1] = &d;
-        if (bulk) {
+        if (variable) {
+            ptrs[2] = &list;
+            ptrs[3] = &count;
+        } else if (bulk) {
             ptrs[2] = &stage_bytes;
             ptrs[3] = &status;
             ptrs[4] = &timeout_ns;
@@ -401,9 +429,16 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         a.stage_bytes = p->bulk_stage_bytes;
         a.status = p->d_ctl + 1;
         a.timeout_ns = p->timeout_ns;
-        a.fill(rs.copy == SPARBIT_COPY_BULK);
+        a.list = nullptr;
+        a.count = 0;
+        if (p->variable) {
+            const size_t ti = seq.table_index(i);
+            a.list = p->d_vtasks + p->vtask_lo[ti];
+            a.count = p->vtask_hi[ti] - p->vtask_lo[ti];
+        }
+        a.fill(rs.copy == SPARBIT_COPY_BULK, p->variable);
         PhaseLaunch pl;
-        int rc = plan_phase_launch(p, rs, a.d, pl);
+        int rc = plan_phase_launch(p, rs, a.d, pl, a.count);
         if (rc) return rc;
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
@@ -696,6 +731,29 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
             for (PhaseDesc& d : p->sched.phases) set_max(d);
             if (p->sched.has_fused_first) set_max(p->sched.fused_first);
             p->sched.m = 0;
+            // task lists, indexed like the device descriptor table: every phase, the fused first
+            // pass, and (as in that table) phases 1.. once more after it
+            auto add_list = [&](const PhaseDesc& d) {
+                p->vtask_lo.push_back(p->vtasks.size());
+                for (uint32_t r = 0; r < p->sched.P; r++)
+                    for (uint32_t j = 0; j < d.copies; j++) {
+                        const CopyLoc c = locate_copy(d, p->sched.P, r, j);
+                        const uint64_t b = p->voff[c.dst_slot + d.run] - p->voff[c.dst_slot];
+                        const uint64_t q = (uint64_t)r * d.copies + j;
+                        for (uint64_t sg = 0; sg * kVarSegmentBytes < b; sg++)
+                            p->vtasks.push_back((unsigned long long)((q << 32) | sg));
+                    }
+                p->vtask_hi.push_back(p->vtasks.size());
+            };
+            for (const PhaseDesc& d : p->sched.phases) add_list(d);
+            if (p->sched.has_fused_first) {
+                add_list(p->sched.fused_first);
+                for (size_t i = 2; i < p->sched.phases.size(); i++) {  // same lists as phases 1..
+                    p->vtask_lo.push_back(p->vtask_lo[i]);
+                    p->vtask_hi.push_back(p->vtask_hi[i]);
+                }
+            }
+            if (p->vtasks.size() >> 28) rc = SPARBIT_ERR_OVERFLOW;  // 2 GiB of task entries: refuse
         }
     } catch (const std::bad_alloc&) {
         rc = SPARBIT_ERR_NOMEM;
@@ -724,6 +782,7 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
         if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
         cudaFree(p->d_descs);
         cudaFree(p->d_voff);
+        cudaFree(p->d_vtasks);
         cudaFree(p->d_ctl);
         cudaFree(p->stage_send);
         cudaFree(p->stage_recv);

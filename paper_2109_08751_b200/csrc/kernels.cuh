@@ -148,43 +148,12 @@ __device__ __forceinline__ void st_cg<unsigned char>(unsigned char* p, unsigned 
 
 // One phase on the vector engine.  warp_id / n_warps enumerate all warps taking part.
 // Requires P * copies * ceil(vectors_per_copy / (32*U)) < 2^32 (checked on the host).
-//
-// kVar = true is the variable-block-size form (allgatherv): d.copy_bytes is then the LARGEST copy
-// of the phase and fixes the task grid; each copy's own size and position come from g.voff.
-template <bool kVar>
-struct CopyBytes {
-    uint64_t src, dst, dst2;  // byte offsets inside the source / destination space
-    uint64_t vectors;         // vectors this copy really has
-};
-
-template <typename V, bool kVar>
-__device__ __forceinline__ CopyBytes<kVar> copy_bytes_of(const Geom& g, const PhaseDesc& d, const CopyLoc& c,
-                                                         uint32_t r, uint64_t spitch, uint64_t dpitch,
-                                                         uint64_t uniform_vectors) {
-    CopyBytes<kVar> o;
-    if constexpr (kVar) {
-        const uint64_t lo = __ldg(g.voff + c.dst_slot);
-        const uint64_t hi = __ldg(g.voff + c.dst_slot + d.run);
-        o.vectors = (hi - lo) / sizeof(V);
-        o.src = d.src_space == SPACE_SEND ? __ldg(g.voff + c.src_rank)
-                                          : (uint64_t)c.src_rank * spitch + __ldg(g.voff + c.src_slot);
-        o.dst = (uint64_t)c.dst_rank * dpitch + lo;
-        o.dst2 = (uint64_t)r * dpitch + lo;
-    } else {
-        o.vectors = uniform_vectors;
-        o.src = (uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m;
-        o.dst = (uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m;
-        o.dst2 = (uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m;
-    }
-    return o;
-}
-
-template <typename V, bool kVar = false>
+template <typename V>
 __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uint32_t warp_id, uint32_t n_warps,
                                           uint32_t lane) {
     constexpr int U = kVecUnroll;
     const uint32_t P = g.P;
-    const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy (of the largest copy if kVar)
+    const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy
     const uint32_t n_copies = P * d.copies;            // copies in the phase (< 2^32, host-checked)
     const char* sbase = space_base(g, d.src_space);
     char* dbase = space_base(g, d.dst_space);
@@ -203,21 +172,20 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
             const uint32_t r = q / d.copies;
             const uint32_t j = q - r * d.copies;
             const CopyLoc c = locate_copy(d, P, r, j);
-            const CopyBytes<kVar> cb = copy_bytes_of<V, kVar>(g, d, c, r, spitch, dpitch, vpc64);
-            const V* src = reinterpret_cast<const V*>(sbase + cb.src);
-            V* dst = reinterpret_cast<V*>(dbase + cb.dst);
-            V* dst2 = reinterpret_cast<V*>(dbase + cb.dst2);
+            const V* src = reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
+            V* dst = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m));
+            V* dst2 = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m));
             const uint64_t v0 = (uint64_t)sp * span + lane;
             V regs[U];
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t v = v0 + 32u * k;
-                if (v < cb.vectors) regs[k] = ld_cg<V>(src + v);
+                if (v < vpc64) regs[k] = ld_cg<V>(src + v);
             }
 #pragma unroll
             for (int k = 0; k < U; k++) {
                 const uint64_t v = v0 + 32u * k;
-                if (v < cb.vectors) {
+                if (v < vpc64) {
                     st_cg<V>(dst + v, regs[k]);
                     if (d.dup_self) st_cg<V>(dst2 + v, regs[k]);
                 }
@@ -245,12 +213,11 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
                     const uint32_t r = q / d.copies;
                     const uint32_t j = q - r * d.copies;
                     const CopyLoc c = locate_copy(d, P, r, j);
-                    const CopyBytes<kVar> cb = copy_bytes_of<V, kVar>(g, d, c, r, spitch, dpitch, vpc64);
-                    if (v < cb.vectors) {
-                        dsts[k] = reinterpret_cast<V*>(dbase + cb.dst) + v;
-                        dsts2[k] = reinterpret_cast<V*>(dbase + cb.dst2) + v;
-                        regs[k] = ld_cg<V>(reinterpret_cast<const V*>(sbase + cb.src) + v);
-                    }
+                    const V* src =
+                        reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
+                    dsts[k] = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
+                    dsts2[k] = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m)) + v;
+                    regs[k] = ld_cg<V>(src + v);
                 }
             }
 #pragma unroll
@@ -259,6 +226,63 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
                     st_cg<V>(dsts[k], regs[k]);
                     if (d.dup_self) st_cg<V>(dsts2[k], regs[k]);
                 }
+        }
+    }
+}
+
+// One phase with blocks of DIFFERENT sizes (allgatherv).  The host lists the phase's work as
+// tasks of at most kVarSegmentBytes: entry = copy index (r * copies + j) in the high half, segment
+// number inside that copy in the low half; empty blocks have no entry.  Every task is then about
+// the same size, so handing task t to warp t mod n_warps balances the warps whatever the mix of
+// block sizes is.  A copy's size and position come from g.voff (prefix sums of the byte counts):
+// block b is voff[b+1]-voff[b] bytes, at voff[b] in the send buffer and in every receive buffer.
+constexpr uint32_t kVarSegmentBytes = 4096;
+
+template <typename V>
+__device__ __forceinline__ void vec_list_phase(const Geom& g, const PhaseDesc& d,
+                                               const unsigned long long* __restrict__ list, uint64_t count,
+                                               uint32_t warp_id, uint32_t n_warps, uint32_t lane) {
+    constexpr int U = kVecUnroll;
+    constexpr uint32_t span = 32u * U;  // vectors per warp iteration
+    const uint32_t P = g.P;
+    const char* sbase = space_base(g, d.src_space);
+    char* dbase = space_base(g, d.dst_space);
+    const uint64_t spitch = space_pitch(g, d.src_space);
+    const uint64_t dpitch = space_pitch(g, d.dst_space);
+    for (uint64_t t = warp_id; t < count; t += n_warps) {
+        const unsigned long long e = __ldg(list + t);
+        const uint32_t q = (uint32_t)(e >> 32);
+        const uint32_t sg = (uint32_t)e;
+        const uint32_t r = q / d.copies;
+        const uint32_t j = q - r * d.copies;
+        const CopyLoc c = locate_copy(d, P, r, j);
+        const uint64_t lo = __ldg(g.voff + c.dst_slot);
+        const uint64_t hi = __ldg(g.voff + c.dst_slot + d.run);
+        const uint64_t soff = d.src_space == SPACE_SEND ? __ldg(g.voff + c.src_rank)
+                                                        : (uint64_t)c.src_rank * spitch + __ldg(g.voff + c.src_slot);
+        const uint64_t begin = (uint64_t)sg * kVarSegmentBytes;  // this task's bytes of the copy
+        uint64_t end = begin + kVarSegmentBytes;
+        if (end > hi - lo) end = hi - lo;
+        const V* src = reinterpret_cast<const V*>(sbase + soff + begin);
+        V* dst = reinterpret_cast<V*>(dbase + (uint64_t)c.dst_rank * dpitch + lo + begin);
+        V* dst2 = reinterpret_cast<V*>(dbase + (uint64_t)r * dpitch + lo + begin);
+        const uint32_t vectors = (uint32_t)((end - begin) / sizeof(V));
+#pragma unroll 1
+        for (uint32_t first = 0; first < vectors; first += span) {
+            V regs[U];
+#pragma unroll
+            for (int k = 0; k < U; k++) {
+                const uint32_t v = first + lane + 32u * k;
+                if (v < vectors) regs[k] = ld_cg<V>(src + v);
+            }
+#pragma unroll
+            for (int k = 0; k < U; k++) {
+                const uint32_t v = first + lane + 32u * k;
+                if (v < vectors) {
+                    st_cg<V>(dst + v, regs[k]);
+                    if (d.dup_self) st_cg<V>(dst2 + v, regs[k]);
+                }
+            }
         }
     }
 }
@@ -431,12 +455,22 @@ __device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& ep
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// one phase, vector engine (kVar: variable block sizes)
-template <typename V, bool kVar = false>
+// one phase, vector engine
+template <typename V>
 __global__ void __launch_bounds__(512, 2) phase_vec_kernel(Geom g, PhaseDesc d) {
     chain_wait();
     const uint32_t wpb = blockDim.x >> 5;
-    vec_phase<V, kVar>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
+    vec_phase<V>(g, d, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
+    chain_trigger();
+}
+
+// one phase, vector engine, variable block sizes (task list built by the host)
+template <typename V>
+__global__ void __launch_bounds__(512, 2) phase_vec_list_kernel(Geom g, PhaseDesc d, const unsigned long long* list,
+                                                                unsigned long long count) {
+    chain_wait();
+    const uint32_t wpb = blockDim.x >> 5;
+    vec_list_phase<V>(g, d, list, count, blockIdx.x * wpb + (threadIdx.x >> 5), gridDim.x * wpb, threadIdx.x & 31u);
     chain_trigger();
 }
 
