@@ -37,12 +37,12 @@ METRIC = "sparbit_allgather_effective_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (bytes; None = not captured for this workload)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, measured with
+# one-pass ncu captures of this benchmark at full size (bytes; absent = not captured)
 NCU_TRAFFIC_BYTES = {
-    # profiles/persistent_kernels_P256_m16k.md (full-size section): 4.16 GB read + 4.25 GB written
+    # persistent_bulk_kernel, whole collective: 4.16 GB read + 4.25 GB written
     "sparbit:P256:m65536:persistent:bulk": 8.41e9,
-    # profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md: last phase, 2.15 GB read + 2.10 GB written
+    # phase_bulk_kernel, last phase: 2.15 GB read + 2.10 GB written
     "sparbit:P256:m65536:graph:bulk": 4.25e9,
 }
 

@@ -1,21 +1,26 @@
 // Copy kernels of the step executor (sm_100a).
 //
-// Two copy engines execute one phase (a set of block copies given by a PhaseDesc):
+// Two copy engines execute one pass (a set of block copies given by a PhaseDesc):
 //
 //   vector  warp-cooperative ld.global.cg / st.global.cg with 16-, 8-, 4-, 2- or 1-byte vectors.
 //           A warp task is a span of one copy (32 lanes x U vectors, index arithmetic once per
-//           span) or, for copies shorter than a warp row, a row of several whole copies.
+//           span) or, for copies shorter than a warp row, rows of several whole copies.  A
+//           second form (vec_list_phase) takes a host-built task list, for blocks of different
+//           sizes.
 //   bulk    cp.async.bulk global -> shared -> global through a ring of shared-memory stages, one
 //           elected lane per warp driving its own ring; completion of loads through mbarriers,
 //           of stores through bulk async-groups.  No cluster multicast anywhere: every block has
-//           exactly one destination.
+//           one destination (two in the fused first pass, issued as two stores).
 //
-// and three ways to sequence phases: one kernel per phase (stream or CUDA-graph chain), one
-// persistent cooperative kernel with a bounded-wait grid barrier after every phase, or one
-// thread-block cluster with the hardware cluster barrier after every phase.
+// and four ways to sequence passes: one kernel per pass, chained by programmatic dependent launch
+// (plain stream launches or a CUDA graph); one persistent cooperative kernel with a bounded-wait
+// grid barrier after every pass; or one thread-block cluster with the hardware cluster barrier.
 //
-// Loads never use the non-coherent path: data written in one phase is read by other SMs in the
-// next one inside the same launch.
+// Loads never use the non-coherent path or L1: data written in one pass is read by other SMs in
+// the next one, possibly inside the same launch.
+//
+// Both engines are tuned to about 32 KiB of loads in flight per SM, the measured sweet spot of a
+// copy on B200 (more in flight lowers the achieved HBM bandwidth).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -35,26 +40,23 @@ struct BarrierCtl {
     unsigned long long timeout_ns;
 };
 
-struct BulkCfg {
-    uint32_t stage_bytes;     // bytes per shared-memory stage (multiple of 16)
-    uint32_t pad_;
-};
-
+// Tunables (overridable at compile time for experiments).
 #ifndef SPB_BULK_STAGES
-#define SPB_BULK_STAGES 4
+#define SPB_BULK_STAGES 4   // stages per ring
 #endif
 #ifndef SPB_BULK_LOADS
-#define SPB_BULK_LOADS 2
+#define SPB_BULK_LOADS 2    // loads in flight per ring; the other stages hold pending stores
 #endif
-constexpr int kBulkStages = SPB_BULK_STAGES;     // stages per ring
-constexpr int kBulkLoadsAhead = SPB_BULK_LOADS;  // loads in flight per ring; the rest hold pending stores
 #ifndef SPB_VEC_UNROLL
-#define SPB_VEC_UNROLL 2
+#define SPB_VEC_UNROLL 2    // vectors per lane per warp task
 #endif
 #ifndef SPB_PERSIST_MIN_CTAS
-#define SPB_PERSIST_MIN_CTAS 2
+#define SPB_PERSIST_MIN_CTAS 2  // CTAs of 512 threads per SM the persistent vector kernel is built for
 #endif
-constexpr int kVecUnroll = SPB_VEC_UNROLL;  // vectors per lane per warp task
+constexpr int kBulkStages = SPB_BULK_STAGES;
+constexpr int kBulkLoadsAhead = SPB_BULK_LOADS;
+constexpr int kVecUnroll = SPB_VEC_UNROLL;
+static_assert(kBulkLoadsAhead >= 1 && kBulkLoadsAhead < kBulkStages, "a ring needs stages for loads and for stores");
 
 // ------------------------------------------------------------------------------------------------
 // small PTX helpers
