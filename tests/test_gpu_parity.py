@@ -296,3 +296,33 @@ def test_graph_follows_new_pointers(dev):
         assert plan.status() == sp.OK
         want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
         assert np.array_equal(recv[: P * P * m].cpu().numpy(), want.reshape(-1))
+
+
+@pytest.mark.parametrize("copy", COPIES)
+def test_graph_cache_recycles_entries(dev, copy):
+    """More buffer sets than the graph cache holds: the least recently used instance is
+    re-parameterised in place and must then use the new buffers, not the old ones."""
+    P, m = 10, 4096
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_GRAPH)
+    plan.set_copy_path(copy)
+    sets = []
+    for k in range(7):
+        host_send = si.send_blocks(P, m, 900 + k)
+        sets.append((host_send, torch.from_numpy(host_send.reshape(-1)).to(dev),
+                     torch.empty(P * P * m, dtype=torch.uint8, device=dev)))
+    for rnd in range(2):
+        for host_send, send, recv in sets:
+            recv.fill_(si.SENTINEL)
+            plan.allgather(send, recv)
+        assert plan.status() == sp.OK
+        for host_send, send, recv in sets:
+            want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+            assert np.array_equal(recv.cpu().numpy(), want.reshape(-1)), rnd
+    # partial ranges get graphs of their own and must not disturb the cached full ones
+    host_send, send, recv = sets[0]
+    recv.fill_(si.SENTINEL)
+    plan.allgather_steps(send, recv, -1, 1)
+    plan.allgather_steps(send, recv, 2, plan.last_phase)
+    assert plan.status() == sp.OK
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
