@@ -124,6 +124,9 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
  * unknown enum), ERR_OVERFLOW (P*P*block_bytes does not fit in 63 bits, or P > 2^24),
  * ERR_UNSUPPORTED (recursive doubling with P not a power of two, neighbor exchange with odd P:
  * Section II-A defines them for those P only), ERR_NOMEM.  Host-only.
+ * Environment: when exec is AUTO, SPARBIT_EXEC=persistent|graph|stream|cluster replaces the
+ * automatic choice; SPARBIT_COPY=vector|bulk presets the copy engine (sparbit_plan_set_copy_path
+ * still overrides it).  Other values are ignored.
  */
 int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out);
 

@@ -112,6 +112,26 @@ struct sparbit_plan_s {
 
 namespace {
 
+// SPARBIT_EXEC / SPARBIT_COPY in the environment override what AUTO would pick (not an explicit
+// request): persistent|graph|stream|cluster and vector|bulk.  Anything else is ignored.
+int env_choice(const char* name, const char* const* words, const int* values, int n, int fallback) {
+    const char* v = getenv(name);
+    if (!v) return fallback;
+    for (int i = 0; i < n; i++)
+        if (strcmp(v, words[i]) == 0) return values[i];
+    return fallback;
+}
+int env_exec(int fallback) {
+    static const char* const w[] = {"persistent", "graph", "stream", "cluster"};
+    static const int x[] = {SPARBIT_EXEC_PERSISTENT, SPARBIT_EXEC_GRAPH, SPARBIT_EXEC_STREAM, SPARBIT_EXEC_CLUSTER};
+    return env_choice("SPARBIT_EXEC", w, x, 4, fallback);
+}
+int env_copy(int fallback) {
+    static const char* const w[] = {"vector", "bulk"};
+    static const int x[] = {SPARBIT_COPY_VECTOR, SPARBIT_COPY_BULK};
+    return env_choice("SPARBIT_COPY", w, x, 2, fallback);
+}
+
 int map_sched_err(int e) {
     switch (e) {
         case SCHED_OK: return SPARBIT_OK;
@@ -683,7 +703,8 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
         delete p;
         return rc;
     }
-    p->exec_req = exec;
+    p->exec_req = exec == SPARBIT_EXEC_AUTO ? env_exec(SPARBIT_EXEC_AUTO) : exec;
+    p->copy_req = env_copy(SPARBIT_COPY_AUTO);
     *out = p;
     return SPARBIT_OK;
 }
@@ -763,6 +784,10 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
         return rc;
     }
     p->exec_req = exec;
+    if (exec == SPARBIT_EXEC_AUTO) {  // variable-size plans take graph or stream only
+        const int e = env_exec(SPARBIT_EXEC_AUTO);
+        if (e == SPARBIT_EXEC_GRAPH || e == SPARBIT_EXEC_STREAM) p->exec_req = e;
+    }
     *out = p;
     return SPARBIT_OK;
 }

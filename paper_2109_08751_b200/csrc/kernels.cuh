@@ -414,12 +414,13 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
 // All threads of all CTAs call it; `epoch` counts the barriers this launch has passed.  Returns
 // false when the wait gave up or another CTA reported a failure: the caller must then leave the
 // kernel.  Co-residency of the grid is guaranteed by the cooperative launch.
+template <bool kAsyncProxy>
 __device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& epoch, int* smem_flag) {
     __syncthreads();
     if (threadIdx.x == 0) {
         epoch++;
         const unsigned target = ctl.base + epoch * ctl.expected;
-        fence_proxy_async_all();          // bulk stores of this CTA -> visible before the release
+        if (kAsyncProxy) fence_proxy_async_all();  // bulk stores of this CTA -> visible before the release
         red_release_gpu_add(ctl.counter, 1u);
         bool ok = true;
         unsigned polls = 0;
@@ -438,7 +439,7 @@ __device__ __forceinline__ bool grid_barrier(const BarrierCtl& ctl, unsigned& ep
                 }
             }
         }
-        fence_proxy_async_all();          // later bulk loads see what the other CTAs wrote
+        if (kAsyncProxy) fence_proxy_async_all();  // later bulk loads see what the other CTAs wrote
         *smem_flag = ok ? 1 : 0;
     }
     __syncthreads();
@@ -537,7 +538,7 @@ __global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kern
         const int cur = (ph - first) & 1;
         if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
         vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
-        if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
+        if (ph != last && !grid_barrier<false>(ctl, epoch, &flag)) return;
     }
 }
 
@@ -562,7 +563,7 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
         if (driver)
             bulk_phase(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
                        ctl.timeout_ns);
-        if (ph != last && !grid_barrier(ctl, epoch, &flag)) return;
+        if (ph != last && !grid_barrier<true>(ctl, epoch, &flag)) return;
     }
 }
 

@@ -137,3 +137,12 @@ def test_exec_mode_resolution():
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH             # measured best at every size
     assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH
     assert sp.Plan(256, 65536, exec_mode=sp.EXEC_PERSISTENT).exec_mode == sp.EXEC_PERSISTENT
+
+
+def test_environment_overrides_only_the_automatic_choice(monkeypatch):
+    monkeypatch.setenv("SPARBIT_EXEC", "persistent")
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_PERSISTENT
+    assert sp.Plan(8, 64, exec_mode=sp.EXEC_STREAM).exec_mode == sp.EXEC_STREAM   # explicit wins
+    assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_GRAPH                  # not offered there
+    monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH
