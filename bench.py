@@ -36,6 +36,7 @@ P_DEFAULT, M_DEFAULT = 256, 64 * 1024
 METRIC = "sparbit_allgather_effective_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 7700.0  # HBM3e of the HGX B200 (8000 on DGX); context only, not the roofline's peak
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, measured with
 # one-pass ncu captures of this benchmark at full size (bytes; absent = not captured)
@@ -373,6 +374,8 @@ def run_ours(args):
                        "parallelism": "replicas only" if world > 1 else "1 GPU"},
             "us_per_collective": {"min": min(per_ms) * 1e3, "avg": avg_ms * 1e3, "max": max(per_ms) * 1e3},
             "pct_of_hbm_peak": 100.0 * value / world / peak,
+            "pct_of_nominal_hbm": 100.0 * value / world / NOMINAL_HBM_GBS,
+            "GBps_from_min_time": world * effective_bytes(P, m) / (min(per_ms) * 1e-3) / 1e9,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(k1 - k0), "graph_launches": int(g1 - g0),
             "clocks": clocks, "checked": bool(checked),
@@ -386,6 +389,40 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------------------------------
+def run_cpu_sweep(args):
+    """The oracle of every algorithm timed on this machine's host cores (no GPU involved): execute
+    phase only, best of 3, one thread and all threads (capped at 16), same effective-bytes formula
+    as the GPU numbers.  One JSON line per (algorithm, P, m)."""
+    import oracle
+    cores = os.cpu_count() or 1
+    threads = min(cores, 16)
+    P = args.P
+    for m in (64, 4096, 65536):
+        send = si.send_blocks(P, m, args.seed).reshape(-1)
+        for name, algo in (("sparbit", oracle.SPARBIT), ("ring", oracle.RING), ("ne", oracle.NEIGHBOR_EXCHANGE),
+                           ("rd", oracle.RECURSIVE_DOUBLING), ("bruck", oracle.BRUCK)):
+            if (name == "rd" and P & (P - 1)) or (name == "ne" and P % 2):
+                continue
+            plan = oracle.Plan(algo, P)
+            recv = si.sentinel_buffer(P * P * m)
+            scratch = si.sentinel_buffer(P * P * m) if algo == oracle.BRUCK else None
+            out = {"algo": name, "P": P, "m": m, "cores": threads}
+            for label, t in (("us_1_thread", 1), (f"us_{threads}_threads", threads)):
+                best = None
+                for _ in range(3):
+                    t0 = time.perf_counter()
+                    plan.run(m, send, recv, scratch, threads=t)
+                    dt = time.perf_counter() - t0
+                    best = dt if best is None else min(best, dt)
+                out[label] = round(best * 1e6, 1)
+                out[label.replace("us_", "GBps_")] = round(effective_bytes(P, m) / best / 1e9, 2)
+            out["checked"] = bool(np.array_equal(recv.reshape(P, P * m)[P - 1], send))
+            print(json.dumps(out), flush=True)
+            plan.close()
+            del recv, scratch
+    return 0
+
+
 def run_sweep(args):
     """Latency and bandwidth curves: every point timed with the paper's protocol (5 warm-ups, 50
     timed collectives, min / avg / max), one JSON line per (algorithm, executor, engine, P, m)."""
@@ -585,9 +622,13 @@ def main():
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     ap.add_argument("--heatmap", action="store_true",
                     help="best algorithm per (P, m) cell, one JSON line per cell")
+    ap.add_argument("--cpu-sweep", action="store_true",
+                    help="time the CPU oracle of every algorithm on the host cores (no GPU)")
     ap.add_argument("--allgatherv", action="store_true",
                     help="variable block sizes on the Sparbit schedule, one JSON line per size mix")
     args = ap.parse_args()
+    if args.cpu_sweep:
+        return run_cpu_sweep(args)
     if args.allgatherv:
         return run_allgatherv(args)
     if args.heatmap:
