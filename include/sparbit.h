@@ -210,6 +210,19 @@ int sparbit_plan_step_info(const sparbit_plan_t* plan, int step, int* distance, 
  */
 int sparbit_plan_messages(const sparbit_plan_t* plan, int phase, sparbit_msg* out, size_t cap, size_t* n);
 
+/*
+ * Host-side check of what the kernels will execute, in place of a device race detector: every
+ * pass of the full collective (the fused first pass included) is expanded through the kernels'
+ * own index function and checked for (a) ranks and slots inside their buffers, (b) no location
+ * read before an earlier pass has filled it, (c) inside a pass, no location written twice and
+ * none both read and written, (d) every receive slot written exactly once over the collective.
+ * The paper's Section III-B states (c) and (d) as the purpose of withholding blocks ("double
+ * writing the same block ... is not desirable").  Returns SPARBIT_OK, or SPARBIT_ERR_ARG with the
+ * offending phase in *bad_phase (may be NULL; last phase + 1 = the final count), SPARBIT_ERR_LIMIT
+ * for P > 8192 (the check needs P*P bytes of host memory), SPARBIT_ERR_NOMEM.  Host-only.
+ */
+int sparbit_plan_validate(const sparbit_plan_t* plan, int* bad_phase);
+
 /* Bytes of workspace the plan needs: 0, or P*P*m for Bruck. */
 size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* plan);
 

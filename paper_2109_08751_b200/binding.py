@@ -44,6 +44,7 @@ SYMBOLS = {
     "sparbit_plan_last_phase": (_i, [_vp]),
     "sparbit_plan_step_info": (_i, [_vp, _i, _pi, _pi, _pi]),
     "sparbit_plan_messages": (_i, [_vp, _i, _vp, _sz, ctypes.POINTER(_sz)]),
+    "sparbit_plan_validate": (_i, [_vp, _pi]),
     "sparbit_plan_workspace_bytes": (_sz, [_vp]),
     "sparbit_plan_set_workspace": (_i, [_vp, _vp, _sz]),
     "sparbit_plan_set_copy_path": (_i, [_vp, _i]),
@@ -161,6 +162,13 @@ class Plan:
             _check(lib.sparbit_plan_messages(self._h, phase, out.ctypes.data, n.value, ctypes.byref(n)),
                    "sparbit_plan_messages")
         return out
+
+    def validate(self) -> None:
+        """Host-side race and bounds check of the descriptors (raises with the offending phase)."""
+        bad = ctypes.c_int()
+        code = lib.sparbit_plan_validate(self._h, ctypes.byref(bad))
+        if code != OK:
+            raise SparbitError(code, f"sparbit_plan_validate (phase {bad.value})")
 
     @property
     def workspace_bytes(self) -> int:

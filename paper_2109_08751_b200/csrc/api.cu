@@ -941,6 +941,75 @@ int sparbit_plan_set_barrier_test(sparbit_plan_t* p, int extra_arrivals, uint64_
     return SPARBIT_OK;
 }
 
+// Host-side race and bounds check of the descriptors as the kernels will execute them: every
+// pass of the full collective (fused first pass included) is expanded through locate_copy; a
+// location is (space, rank, slot) and `valid` says whether it already holds its block.
+int sparbit_plan_validate(const sparbit_plan_t* p, int* bad_phase) {
+    if (!p) return SPARBIT_ERR_ARG;
+    if (bad_phase) *bad_phase = -2;
+    const Schedule& s = p->sched;
+    const uint32_t P = s.P;
+    if (P > 8192) return SPARBIT_ERR_LIMIT;
+    try {
+        const size_t PP = (size_t)P * P;
+        // per space (RECV, WORK): 0 = empty, 1 = valid, 2 = written in this pass, 3 = read in this pass
+        std::vector<uint8_t> state[2] = {std::vector<uint8_t>(PP, 0), std::vector<uint8_t>(PP, 0)};
+        std::vector<uint32_t> writes(PP, 0);
+        ExecSeq seq;
+        seq.s = &s;
+        seq.first = -1;
+        seq.last = s.last_phase();
+        seq.fused = s.last_phase() >= 0 && s.has_fused_first;
+        auto fail = [&](int pass) {
+            if (bad_phase) *bad_phase = pass;
+            return SPARBIT_ERR_ARG;
+        };
+        for (int i = 0; i < seq.count(); i++) {
+            const PhaseDesc& d = seq.item(i);
+            const int pass = seq.fused ? i : i - 1;  // phase number (the fused pass reports 0)
+            std::vector<size_t> touched_w, touched_r;
+            for (uint32_t r = 0; r < P; r++)
+                for (uint32_t j = 0; j < d.copies; j++) {
+                    const CopyLoc c = locate_copy(d, P, r, j);
+                    if (c.dst_rank >= P || c.src_rank >= P) return fail(pass);
+                    for (uint32_t k = 0; k < d.run; k++) {
+                        const uint32_t ss = c.src_slot + k, ds = c.dst_slot + k;
+                        if (ds >= P || d.dst_space == SPACE_SEND) return fail(pass);
+                        if (d.src_space == SPACE_SEND) {
+                            if (c.src_slot != 0 || d.run != 1) return fail(pass);  // one block per rank
+                        } else {
+                            if (ss >= P) return fail(pass);
+                            uint8_t& st = state[d.src_space - 1][(size_t)c.src_rank * P + ss];
+                            if (st != 1 && st != 3) return fail(pass);  // read before it is valid, or while written
+                            if (st == 1) touched_r.push_back((size_t)c.src_rank * P + ss);
+                            st = 3;
+                        }
+                        const int ndst = d.dup_self ? 2 : 1;
+                        for (int t = 0; t < ndst; t++) {
+                            const uint32_t dr = t == 0 ? c.dst_rank : r;
+                            if (t == 1 && dr == c.dst_rank) continue;  // one rank: both destinations coincide
+                            const size_t at = (size_t)dr * P + ds;
+                            uint8_t& st = state[d.dst_space - 1][at];
+                            if (st != 0) return fail(pass);  // written twice, or written while read / valid
+                            st = 2;
+                            touched_w.push_back(at);
+                            if (d.dst_space == SPACE_RECV) writes[at]++;
+                        }
+                    }
+                }
+            // the pass boundary: what was written becomes valid, what was read stays valid
+            if (d.src_space != SPACE_SEND)
+                for (size_t at : touched_r) state[d.src_space - 1][at] = 1;
+            for (size_t at : touched_w) state[d.dst_space - 1][at] = 1;
+        }
+        for (size_t at = 0; at < PP; at++)
+            if (state[0][at] != 1 || writes[at] != 1) return fail(s.last_phase() + 1);
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    return SPARBIT_OK;
+}
+
 const char* sparbit_strerror(int code) {
     switch (code) {
         case SPARBIT_OK: return "success";

@@ -146,3 +146,20 @@ def test_environment_overrides_only_the_automatic_choice(monkeypatch):
     assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_GRAPH                  # not offered there
     monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_descriptors_are_race_free_and_in_bounds(algo):
+    """The library's own host-side check of what the kernels execute (fused first pass included)."""
+    for P in list(range(1, 70)) + [100, 127, 128, 253, 256, 1000]:
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
+            continue
+        if algo == sp.ALGO_RING and P > 128:
+            continue
+        sp.Plan(P, 16, algo).validate()
+    sp.Plan.create_v([16, 0, 32, 48, 8, 8, 0]).validate()
+    with pytest.raises(sp.SparbitError) as e:
+        sp.Plan(10000, 16).validate()
+    assert e.value.code == sp.ERR_LIMIT
