@@ -47,9 +47,11 @@
  *   - the identity of the block carried into receive slot b is b, every receive slot is written
  *     exactly once, and every rank receives exactly P-1 blocks from other ranks.
  *
- * Parity status: pinned (see the CPU tests: plain definition of the result, the paper's P = 5
- * walk-through, the P = 21 decomposition, an independent binomial-tree construction, closed
- * forms, brute force over P = 1..64).
+ * Parity status: pinned (see the CPU tests: plain definition of the result for all five
+ * algorithms, the paper's P = 5 walk-through, the P = 21 decomposition, an independent
+ * binomial-tree construction, closed forms, the partner rule and block counts of the neighbor
+ * exchange, brute force over P = 1..64; for the variable-size runs the plain definition with
+ * byte-granular sizes including empty blocks, and equality with the fixed-size run).
  */
 #include <pthread.h>
 #include <stdarg.h>
