@@ -157,7 +157,8 @@ int sparbit_plan_destroy(sparbit_plan_t* plan);
  * MPI_Allgather(sendbuf, m, MPI_BYTE, recvbuf, m, MPI_BYTE, comm) for a communicator of P ranks.
  *   sendbuf  device, P*m bytes, read only          recvbuf  device, P*P*m bytes, fully overwritten
  *   stream   a cudaStream_t passed as void* (NULL = the legacy default stream)
- * Asynchronous: work is enqueued on `stream` and the call returns.  Any alignment of the
+ * Asynchronous: work is enqueued on `stream` and the call returns (in MPI terms this is the
+ * non-blocking form; synchronising the stream, or sparbit_plan_status, is the wait).  Any alignment of the
  * pointers and any m >= 1 give the right answer; 16-byte aligned buffers with m % 16 == 0 get
  * the fast paths.  Errors (nothing is launched): ERR_ARG (null plan; null buffer with P*m > 0),
  * ERR_ALIAS (ranges overlap), ERR_WORKSPACE (Bruck without workspace), ERR_CUDA.
