@@ -564,8 +564,16 @@ def run_heatmap(args):
              "rd": sp.ALGO_RECURSIVE_DOUBLING, "bruck": sp.ALGO_BRUCK}
     stream = torch.cuda.Stream(device=dev)
     free_bytes = torch.cuda.mem_get_info(dev)[0]
-    for P in (5, 8, 13, 16, 32, 61, 64, 128, 253, 256):
-        for m in (1, 8, 64, 512, 4096, 32768, 262144, 1048576):
+    if args.heatmap == "paper":
+        # the paper's grid (Section IV-A): 1 B .. 1 MiB by powers of two; process counts 8..256 in
+        # steps of 8 and 5..253 in steps of 8 (one less than a multiple of 8, plus the odd offsets)
+        grid_P = sorted(list(range(8, 257, 8)) + list(range(5, 254, 8)))
+        grid_m = [1 << k for k in range(21)]
+    else:
+        grid_P = (5, 8, 13, 16, 32, 61, 64, 128, 253, 256)
+        grid_m = (1, 8, 64, 512, 4096, 32768, 262144, 1048576)
+    for P in grid_P:
+        for m in grid_m:
             if P * P * m * 2.2 + 2 * P * m > free_bytes:
                 continue
             sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
@@ -620,8 +628,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
-    ap.add_argument("--heatmap", action="store_true",
-                    help="best algorithm per (P, m) cell, one JSON line per cell")
+    ap.add_argument("--heatmap", nargs="?", const="coarse", default=None, choices=["coarse", "paper"],
+                    help="best algorithm per (P, m) cell, one JSON line per cell; 'paper' = the paper's "
+                         "grid of 64 process counts x 21 block sizes (about a quarter of an hour)")
     ap.add_argument("--cpu-sweep", action="store_true",
                     help="time the CPU oracle of every algorithm on the host cores (no GPU)")
     ap.add_argument("--allgatherv", action="store_true",
