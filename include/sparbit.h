@@ -56,7 +56,8 @@ enum {
     SPARBIT_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sparbit_last_cuda_error() */
     SPARBIT_ERR_TIMEOUT = 7,     /* the device-side grid barrier gave up waiting */
     SPARBIT_ERR_NOMEM = 8,       /* host allocation failed */
-    SPARBIT_ERR_LIMIT = 9        /* larger than the fixed scratch of sparbit_allgather_noalloc */
+    SPARBIT_ERR_LIMIT = 9        /* beyond a fixed limit of the entry point: the scratch of
+                                    sparbit_allgather_noalloc, P of sparbit_plan_create_v / _validate */
 };
 
 /* Algorithms (paper, Section II-A and Section III).  Only Sparbit is the product's hot path; the
@@ -143,8 +144,9 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
  * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Runs on the
  * vector copy engine with the graph or stream executor: exec must be AUTO, GRAPH or STREAM
  * (PERSISTENT, CLUSTER: ERR_UNSUPPORTED).  Bruck is refused (ERR_UNSUPPORTED: its rotated
- * workspace assumes equal blocks).  Other errors as for sparbit_plan_create; P is limited to
- * 65536 here.  Host-only.
+ * workspace assumes equal blocks).  P is limited to 8192 here (ERR_LIMIT beyond: the plan keeps
+ * one task-list entry per 4 KiB of every copy).  Other errors as for sparbit_plan_create.
+ * Host-only.
  */
 int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, sparbit_plan_t** out);
 

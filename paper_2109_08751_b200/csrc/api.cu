@@ -713,7 +713,7 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     if (!out) return SPARBIT_ERR_ARG;
     *out = nullptr;
     if (!block_bytes || P < 1) return SPARBIT_ERR_ARG;
-    if (P > (1 << 16)) return SPARBIT_ERR_OVERFLOW;
+    if (P > 8192) return SPARBIT_ERR_LIMIT;  // the task lists are built copy by copy: P*(P-1) entries at least
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
     if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // rotated workspace: fixed sizes only
     if (exec != SPARBIT_EXEC_AUTO && exec != SPARBIT_EXEC_GRAPH && exec != SPARBIT_EXEC_STREAM) {
@@ -1022,7 +1022,7 @@ const char* sparbit_strerror(int code) {
         case SPARBIT_ERR_CUDA: return "CUDA runtime error";
         case SPARBIT_ERR_TIMEOUT: return "device barrier timed out";
         case SPARBIT_ERR_NOMEM: return "out of host memory";
-        case SPARBIT_ERR_LIMIT: return "larger than the fixed scratch of sparbit_allgather_noalloc";
+        case SPARBIT_ERR_LIMIT: return "beyond a fixed limit of this entry point (scratch size or rank count)";
         default: return "unknown error";
     }
 }

@@ -91,6 +91,8 @@ def test_create_v_errors_and_introspection():
     assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_PERSISTENT, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_CLUSTER, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     assert lib.sparbit_plan_create_v(3, counts, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    many = (ctypes.c_size_t * 8193)(*([16] * 8193))
+    assert lib.sparbit_plan_create_v(8193, many, 0, 0, ctypes.byref(out)) == sp.ERR_LIMIT
     big = (ctypes.c_size_t * 2)(1 << 61, 1 << 61)
     assert lib.sparbit_plan_create_v(2, big, 0, 0, ctypes.byref(out)) == sp.ERR_OVERFLOW
     plan = sp.Plan.create_v([16, 0, 32, 48, 8])

@@ -65,4 +65,4 @@ def test_noalloc_refuses_what_does_not_fit_its_scratch():
     assert lib.sparbit_allgather_noalloc(0, 16, sp.ALGO_SPARBIT, 4096, 1 << 20, None) == sp.ERR_ARG
     assert lib.sparbit_allgather_noalloc(8, 16, sp.ALGO_SPARBIT, 4096, 4100, None) == sp.ERR_ALIAS
     assert lib.sparbit_allgather_noalloc(8, 0, sp.ALGO_SPARBIT, None, None, None) == sp.OK
-    assert "scratch" in lib.sparbit_strerror(sp.ERR_LIMIT).decode()
+    assert "limit" in lib.sparbit_strerror(sp.ERR_LIMIT).decode()
