@@ -324,6 +324,15 @@ def run_ours(args):
     # two P), launched exactly as inside the collective and timed with events on the same stream
     launches_per_step = (k1 - k0) / args.steps
     one_kernel = launches_per_step <= 1
+    per_pass_us = None
+    if one_kernel and plan.exec_mode == sp.EXEC_PERSISTENT:
+        # one more, traced, launch: the persistent kernel's own time stamps, pass by pass
+        plan.set_trace(True)
+        plan.allgather(sends[0], recv, stream)
+        assert plan.status() == sp.OK
+        stamps = plan.get_trace().astype(np.int64)
+        per_pass_us = [round(float(x) / 1e3, 1) for x in np.diff(stamps)]
+        plan.set_trace(False)
     if one_kernel:
         dom_ms = float(np.mean(per_ms))
         dom_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
@@ -356,6 +365,7 @@ def run_ours(args):
             "kernel": f"{sp.EXEC_NAMES[plan.exec_mode]} executor, {sp.COPY_NAMES[plan.copy_path]} engine: "
                       f"{dom_name} ({launches_per_step:g} launch(es) per collective)",
             "algorithmic_bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
+            "per_pass_us": per_pass_us,
             "whole_path": {"algorithmic_bytes": path_bytes, "us": avg_ms * 1e3,
                            "achieved": path_bytes / (avg_ms * 1e-3) / 1e9,
                            "frac": path_bytes / (avg_ms * 1e-3) / 1e9 / peak},

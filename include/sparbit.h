@@ -254,6 +254,18 @@ int sparbit_plan_launch_counts(const sparbit_plan_t* plan, uint64_t* kernel_laun
 int sparbit_plan_status(sparbit_plan_t* plan, int* device_status);
 
 /*
+ * Per-pass time stamps of the PERSISTENT executor (off by default; the other executors are timed
+ * from outside, kernel by kernel).  With tracing on, CTA 0 stores the GPU's nanosecond timer at
+ * kernel start and each time it leaves a pass (for all passes but the last: after the grid
+ * barrier that ends it), so entry k+1 minus entry k is pass k as that CTA saw it, Waitall
+ * included.  sparbit_plan_get_trace synchronises the plan's last stream and copies the stamps of
+ * the last persistent launch: min(cap, *n) entries, *n = passes + 1 (0 if nothing was traced).
+ * The first traced call allocates the stamp buffer (not inside a stream capture).
+ */
+int sparbit_plan_set_trace(sparbit_plan_t* plan, int on);
+int sparbit_plan_get_trace(sparbit_plan_t* plan, uint64_t* ns, size_t cap, size_t* n);
+
+/*
  * Test hook for the bounded wait of the grid barrier: the next persistent launches expect
  * `extra_arrivals` more arrivals than there are CTAs and give up after `timeout_ns`
  * nanoseconds (0 restores the defaults: no extra arrivals, 2 s).  With extra_arrivals > 0 the

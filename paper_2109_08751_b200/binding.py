@@ -52,6 +52,8 @@ SYMBOLS = {
     "sparbit_plan_copy_path": (_i, [_vp]),
     "sparbit_plan_launch_counts": (_i, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
     "sparbit_plan_status": (_i, [_vp, _pi]),
+    "sparbit_plan_set_trace": (_i, [_vp, _i]),
+    "sparbit_plan_get_trace": (_i, [_vp, ctypes.POINTER(_u64), _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_set_barrier_test": (_i, [_vp, _i, _u64]),
     "sparbit_allgather_noalloc": (_i, [_i, _sz, _i, _vp, _vp, _vp]),
     "sparbit_strerror": (ctypes.c_char_p, [_i]),
@@ -202,6 +204,19 @@ class Plan:
         if code not in (OK, ERR_TIMEOUT):
             raise SparbitError(code, "sparbit_plan_status")
         return code
+
+    def set_trace(self, on: bool) -> None:
+        _check(lib.sparbit_plan_set_trace(self._h, int(bool(on))), "sparbit_plan_set_trace")
+
+    def get_trace(self) -> np.ndarray:
+        """Time stamps (ns) of the last persistent launch: kernel start, then the end of every pass."""
+        n = _sz()
+        _check(lib.sparbit_plan_get_trace(self._h, None, 0, ctypes.byref(n)), "sparbit_plan_get_trace")
+        out = np.zeros(n.value, dtype=np.uint64)
+        if n.value:
+            _check(lib.sparbit_plan_get_trace(self._h, out.ctypes.data_as(ctypes.POINTER(_u64)), n.value,
+                                              ctypes.byref(n)), "sparbit_plan_get_trace")
+        return out
 
     def set_barrier_test(self, extra_arrivals: int, timeout_ns: int) -> None:
         _check(lib.sparbit_plan_set_barrier_test(self._h, extra_arrivals, timeout_ns),

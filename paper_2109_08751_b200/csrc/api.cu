@@ -105,6 +105,11 @@ struct sparbit_plan_s {
     void* stage_recv = nullptr;
     void* stage_work = nullptr;
 
+    // per-pass time stamps of the persistent executor (off by default)
+    bool trace_on = false;
+    unsigned long long* d_trace = nullptr;
+    size_t trace_cap = 0, trace_len = 0;
+
     cudaStream_t last_stream = nullptr;
     bool launched = false;
     uint64_t kernel_launches = 0, graph_launches = 0;
@@ -590,6 +595,19 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     ctl.base = p->bar_base;
     ctl.expected = (unsigned)grid + (unsigned)p->extra_arrivals;
     ctl.timeout_ns = p->timeout_ns;
+    ctl.trace = nullptr;
+    if (p->trace_on) {
+        const size_t need_entries = (size_t)seq.count() + 1;
+        if (need_entries > p->trace_cap) {  // (re)allocate; the first traced call is not capturable
+            cudaFree(p->d_trace);
+            p->d_trace = nullptr;
+            p->trace_cap = 0;
+            CU(cudaMalloc((void**)&p->d_trace, need_entries * sizeof(unsigned long long)));
+            p->trace_cap = need_entries;
+        }
+        ctl.trace = p->d_trace;
+        p->trace_len = need_entries;
+    }
     int first_idx = (int)seq.table_index(0), last_idx = (int)seq.table_index(seq.count() - 1);
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
@@ -808,6 +826,7 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
         cudaFree(p->d_descs);
         cudaFree(p->d_voff);
         cudaFree(p->d_vtasks);
+        cudaFree(p->d_trace);
         cudaFree(p->d_ctl);
         cudaFree(p->stage_send);
         cudaFree(p->stage_recv);
@@ -931,6 +950,24 @@ int sparbit_plan_status(sparbit_plan_t* p, int* device_status) {
         p->bar_base = 0;
         return SPARBIT_ERR_TIMEOUT;
     }
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_set_trace(sparbit_plan_t* p, int on) {
+    if (!p) return SPARBIT_ERR_ARG;
+    p->trace_on = on != 0;
+    if (!p->trace_on) p->trace_len = 0;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_get_trace(sparbit_plan_t* p, uint64_t* ns, size_t cap, size_t* n) {
+    if (!p || !n || (cap > 0 && !ns)) return SPARBIT_ERR_ARG;
+    *n = p->trace_len;
+    if (p->trace_len == 0 || cap == 0) return SPARBIT_OK;
+    CU(cudaStreamSynchronize(p->last_stream));
+    static_assert(sizeof(uint64_t) == sizeof(unsigned long long), "time stamps are 64-bit");
+    const size_t k = p->trace_len < cap ? p->trace_len : cap;
+    CU(cudaMemcpy(ns, p->d_trace, k * sizeof(uint64_t), cudaMemcpyDeviceToHost));
     return SPARBIT_OK;
 }
 
@@ -1159,6 +1196,7 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     ctl.base = 0;
     ctl.expected = (unsigned)grid;
     ctl.timeout_ns = kDefaultTimeoutNs;
+    ctl.trace = nullptr;
     int first_idx = first + 1, last_idx = last + 1;
     const PhaseDesc* descs = d_descs;
     void* args[] = {&g, &descs, &first_idx, &last_idx, &ctl};

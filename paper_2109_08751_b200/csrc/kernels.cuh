@@ -38,6 +38,8 @@ struct BarrierCtl {
     unsigned  base;           // counter value when this launch starts
     unsigned  expected;       // arrivals that complete one barrier (grid size, + test extra)
     unsigned long long timeout_ns;
+    unsigned long long* trace;  // optional: CTA 0 stores %globaltimer at kernel start and after
+                                // every pass it leaves (passes + 1 entries); null = off
 };
 
 // Tunables (overridable at compile time for experiments).
@@ -532,6 +534,8 @@ __global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kern
     const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * wpb;
     unsigned epoch = 0;
+    const bool tracer = ctl.trace != nullptr && blockIdx.x == 0 && threadIdx.x == 0;
+    if (tracer) ctl.trace[0] = globaltimer_ns();
     fetch_desc(&sd[0], &descs[first]);
     __syncthreads();
     for (int ph = first; ph <= last; ph++) {
@@ -539,6 +543,7 @@ __global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kern
         if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
         vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
         if (ph != last && !grid_barrier<false>(ctl, epoch, &flag)) return;
+        if (tracer) ctl.trace[ph - first + 1] = globaltimer_ns();
     }
 }
 
@@ -555,6 +560,8 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
     BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
     if (driver) init_pipe(pp);
     unsigned epoch = 0;
+    const bool tracer = ctl.trace != nullptr && blockIdx.x == 0 && threadIdx.x == 0;
+    if (tracer) ctl.trace[0] = globaltimer_ns();
     fetch_desc(&sd[0], &descs[first]);
     __syncthreads();
     for (int ph = first; ph <= last; ph++) {
@@ -564,6 +571,7 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
             bulk_phase(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
                        ctl.timeout_ns);
         if (ph != last && !grid_barrier<true>(ctl, epoch, &flag)) return;
+        if (tracer) ctl.trace[ph - first + 1] = globaltimer_ns();
     }
 }
 

@@ -326,3 +326,28 @@ def test_graph_cache_recycles_entries(dev, copy):
     assert plan.status() == sp.OK
     want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
     assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+
+
+@pytest.mark.parametrize("copy", COPIES)
+def test_persistent_trace_gives_one_stamp_per_pass(dev, copy):
+    P, m = 64, 16384
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_PERSISTENT)
+    plan.set_copy_path(copy)
+    host_send = si.send_blocks(P, m, 21)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    assert len(plan.get_trace()) == 0
+    plan.set_trace(True)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    t = plan.get_trace().astype(np.int64)
+    assert len(t) == plan.num_steps + 1          # start + one per pass (own block fused with step 0)
+    d = np.diff(t)
+    assert (d > 0).all()
+    assert d[-1] > d[1]                           # the last pass moves 32x the bytes of the second
+    assert 10_000 < t[-1] - t[0] < 5_000_000      # tens of microseconds, not garbage
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+    plan.set_trace(False)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK and len(plan.get_trace()) == 0
