@@ -311,6 +311,16 @@ int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint
 int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* sendbuf, void* recvbuf,
                               void* stream);
 
+/*
+ * Test hook for the other bounded wait, the bulk engine's wait for a shared-memory stage to
+ * fill: the next launches expect `extra_tx_bytes` (a multiple of 16, at most 65536) more bytes
+ * per stage than are loaded, so no stage ever reports full; after `timeout_ns` nanoseconds
+ * (0 = the default 2 s) the waiting lane must set the time-out status and the kernel must return
+ * (every load it issued has long landed by then, so nothing is in flight).  0 bytes switches the
+ * hook off.  Shares the time limit with sparbit_plan_set_barrier_test.
+ */
+int sparbit_plan_set_mbarrier_test(sparbit_plan_t* plan, uint32_t extra_tx_bytes, uint64_t timeout_ns);
+
 const char* sparbit_strerror(int code);
 
 /* Text of the last CUDA error seen by this thread inside the library ("" if none). */

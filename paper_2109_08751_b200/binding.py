@@ -55,6 +55,7 @@ SYMBOLS = {
     "sparbit_plan_set_trace": (_i, [_vp, _i]),
     "sparbit_plan_get_trace": (_i, [_vp, ctypes.POINTER(_u64), _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_set_barrier_test": (_i, [_vp, _i, _u64]),
+    "sparbit_plan_set_mbarrier_test": (_i, [_vp, ctypes.c_uint32, _u64]),
     "sparbit_allgather_noalloc": (_i, [_i, _sz, _i, _vp, _vp, _vp]),
     "sparbit_strerror": (ctypes.c_char_p, [_i]),
     "sparbit_last_cuda_error": (ctypes.c_char_p, []),
@@ -217,6 +218,10 @@ class Plan:
             _check(lib.sparbit_plan_get_trace(self._h, out.ctypes.data_as(ctypes.POINTER(_u64)), n.value,
                                               ctypes.byref(n)), "sparbit_plan_get_trace")
         return out
+
+    def set_mbarrier_test(self, extra_tx_bytes: int, timeout_ns: int) -> None:
+        _check(lib.sparbit_plan_set_mbarrier_test(self._h, extra_tx_bytes, timeout_ns),
+               "sparbit_plan_set_mbarrier_test")
 
     def set_barrier_test(self, extra_arrivals: int, timeout_ns: int) -> None:
         _check(lib.sparbit_plan_set_barrier_test(self._h, extra_arrivals, timeout_ns),

@@ -39,8 +39,10 @@ struct GraphKey {
     int first = 0, last = -2;
     int path = 0, vec = 0;
     unsigned long long timeout_ns = 0;
+    unsigned extra_tx = 0;
     bool same_shape(const GraphKey& o) const {
-        return first == o.first && last == o.last && path == o.path && vec == o.vec && timeout_ns == o.timeout_ns;
+        return first == o.first && last == o.last && path == o.path && vec == o.vec && timeout_ns == o.timeout_ns &&
+               extra_tx == o.extra_tx;
     }
     bool same_buffers(const GraphKey& o) const { return send == o.send && recv == o.recv && work == o.work; }
 };
@@ -82,6 +84,7 @@ struct sparbit_plan_s {
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
+    unsigned mbar_extra_tx = 0;  // test hook of the bulk engine's bounded mbarrier wait
 
     // bulk engine geometry
     // measured on B200: about 32 KiB of loads in flight per SM is the sweet spot for a copy (more
@@ -423,9 +426,10 @@ struct PhaseArgs {
     uint32_t stage_bytes;
     unsigned* status;
     unsigned long long timeout_ns;
+    uint32_t extra_tx;
     const unsigned long long* list;  // variable block sizes: this pass's task list
     unsigned long long count;
-    void* ptrs[5];
+    void* ptrs[6];
     void fill(bool bulk, bool variable = false) {
         ptrs[0] = &g;
         ptrs[1] = &d;
@@ -436,6 +440,7 @@ struct PhaseArgs {
             ptrs[2] = &stage_bytes;
             ptrs[3] = &status;
             ptrs[4] = &timeout_ns;
+            ptrs[5] = &extra_tx;
         }
     }
 };
@@ -454,6 +459,7 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         a.stage_bytes = p->bulk_stage_bytes;
         a.status = p->d_ctl + 1;
         a.timeout_ns = p->timeout_ns;
+        a.extra_tx = p->mbar_extra_tx;
         a.list = nullptr;
         a.count = 0;
         if (p->variable) {
@@ -500,6 +506,7 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     key.path = rs.copy;
     key.vec = rs.vbytes;
     key.timeout_ns = p->timeout_ns;
+    key.extra_tx = p->mbar_extra_tx;
     sparbit_plan_s::GraphEntry* hit = nullptr;
     for (auto& e : p->gcache)
         if (e.key.same_shape(key) && e.key.same_buffers(key)) hit = &e;
@@ -595,6 +602,7 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     ctl.base = p->bar_base;
     ctl.expected = (unsigned)grid + (unsigned)p->extra_arrivals;
     ctl.timeout_ns = p->timeout_ns;
+    ctl.mbar_extra_tx = p->mbar_extra_tx;
     ctl.trace = nullptr;
     if (p->trace_on) {
         const size_t need_entries = (size_t)seq.count() + 1;
@@ -953,6 +961,13 @@ int sparbit_plan_status(sparbit_plan_t* p, int* device_status) {
     return SPARBIT_OK;
 }
 
+int sparbit_plan_set_mbarrier_test(sparbit_plan_t* p, uint32_t extra_tx_bytes, uint64_t timeout_ns) {
+    if (!p || (extra_tx_bytes & 15u) || extra_tx_bytes > 65536u) return SPARBIT_ERR_ARG;
+    p->mbar_extra_tx = extra_tx_bytes;
+    p->timeout_ns = timeout_ns ? timeout_ns : kDefaultTimeoutNs;
+    return SPARBIT_OK;
+}
+
 int sparbit_plan_set_trace(sparbit_plan_t* p, int on) {
     if (!p) return SPARBIT_ERR_ARG;
     p->trace_on = on != 0;
@@ -1196,6 +1211,7 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     ctl.base = 0;
     ctl.expected = (unsigned)grid;
     ctl.timeout_ns = kDefaultTimeoutNs;
+    ctl.mbar_extra_tx = 0;
     ctl.trace = nullptr;
     int first_idx = first + 1, last_idx = last + 1;
     const PhaseDesc* descs = d_descs;

@@ -38,6 +38,8 @@ struct BarrierCtl {
     unsigned  base;           // counter value when this launch starts
     unsigned  expected;       // arrivals that complete one barrier (grid size, + test extra)
     unsigned long long timeout_ns;
+    unsigned  mbar_extra_tx;  // test hook: bytes added to every expected transaction count, so
+                              // that no mbarrier of the bulk engine ever completes (0 = off)
     unsigned long long* trace;  // optional: CTA 0 stores %globaltimer at kernel start and after
                                 // every pass it leaves (passes + 1 entries); null = off
 };
@@ -325,7 +327,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 // (host-checked).  Returns false if a wait gave up.
 __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, uint32_t stage_bytes, uint32_t pipe_id,
                                            uint32_t n_pipes, BulkPipe& pp, unsigned* status,
-                                           unsigned long long timeout_ns) {
+                                           unsigned long long timeout_ns, uint32_t extra_tx = 0) {
     constexpr int S = kBulkStages;
     constexpr int L = kBulkLoadsAhead;
     const uint32_t P = g.P;
@@ -380,7 +382,7 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
                          "l"((unsigned long long)bytes)
                          : "memory");
             asm volatile("st.shared.u64 [%0], %1;" ::"r"(pp.meta + st * 32u + 16u), "l"(delta2) : "memory");
-            mbar_expect_tx(bar, bytes);
+            mbar_expect_tx(bar, bytes + extra_tx);
             bulk_load(pp.ring + st * stage_bytes, src, bytes, bar);
         }
         if (i >= (uint64_t)L) {
@@ -499,7 +501,7 @@ __device__ __forceinline__ void init_pipe(const BulkPipe& pp) {
 
 // one phase, bulk engine
 __global__ void __launch_bounds__(256) phase_bulk_kernel(Geom g, PhaseDesc d, uint32_t stage_bytes, unsigned* status,
-                                                         unsigned long long timeout_ns) {
+                                                         unsigned long long timeout_ns, uint32_t extra_tx) {
     extern __shared__ __align__(128) unsigned char smem[];
     // the bulk kernel leaves room on the SM for its successor (4 warps, 66 KB), and measures
     // best when the successor is let in at once and sets up its rings during this phase
@@ -510,7 +512,8 @@ __global__ void __launch_bounds__(256) phase_bulk_kernel(Geom g, PhaseDesc d, ui
         BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
         init_pipe(pp);
         chain_wait();
-        bulk_phase(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, status, timeout_ns);
+        bulk_phase(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, status, timeout_ns,
+                   extra_tx);
     }
 }
 
@@ -569,7 +572,7 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
         if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
         if (driver)
             bulk_phase(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
-                       ctl.timeout_ns);
+                       ctl.timeout_ns, ctl.mbar_extra_tx);
         if (ph != last && !grid_barrier<true>(ctl, epoch, &flag)) return;
         if (tracer) ctl.trace[ph - first + 1] = globaltimer_ns();
     }

@@ -351,3 +351,24 @@ def test_persistent_trace_gives_one_stamp_per_pass(dev, copy):
     plan.set_trace(False)
     plan.allgather(send, recv)
     assert plan.status() == sp.OK and len(plan.get_trace()) == 0
+
+
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_STREAM])
+def test_bulk_stage_wait_gives_up_instead_of_hanging(dev, exec_mode):
+    """The bulk engine's wait for a stage to fill is bounded too: with more bytes expected than
+    are ever loaded it must time out, report it through the status word, and leave the plan usable."""
+    P, m = 8, 4096
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    plan.set_copy_path(sp.COPY_BULK)
+    host_send = si.send_blocks(P, m, 2)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.set_mbarrier_test(16, 5_000_000)   # 5 ms
+    plan.allgather(send, recv)
+    assert plan.status() == sp.ERR_TIMEOUT
+    plan.set_mbarrier_test(0, 0)
+    recv.fill_(si.SENTINEL)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
