@@ -30,6 +30,12 @@ int cuda_fail(cudaError_t e, const char* what) {
 
 constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s
 constexpr int kVecBlock = 512;
+// Dynamic shared memory a per-pass vector kernel with a FULL grid (two CTAs per SM) asks for
+// without using it: it caps the kernel at two CTAs per SM whatever its register count, so that a
+// chained successor cannot squeeze a third CTA onto some SMs while the others get one (measured at
+// P = 1000, m = 1 KiB: 348 us without the cap, 339 us with it).  Small grids do not ask for it:
+// there the early residency of the successor is what keeps a pass at 2.6 us.
+constexpr size_t kVecOccupancySmem = 100 * 1024;
 constexpr int kClusterBlock = 1024;
 
 struct GraphKey {
@@ -154,6 +160,9 @@ size_t bulk_smem_bytes(const sparbit_plan_s* p) {
     return (size_t)p->bulk_warps * kBulkStages * (p->bulk_stage_bytes + 8 + 32);
 }
 
+const void* pick_phase_vec(int vbytes);
+const void* pick_phase_vec_var(int vbytes);
+
 int ensure_device(sparbit_plan_s* p) {
     if (p->dev_ready) {
         // a plan belongs to the device of its first launch
@@ -192,6 +201,12 @@ int ensure_device(sparbit_plan_s* p) {
     }
     CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
+    for (int vb = 1; vb <= 16; vb *= 2) {
+        CU(cudaFuncSetAttribute(pick_phase_vec(vb), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)kVecOccupancySmem));
+        CU(cudaFuncSetAttribute(pick_phase_vec_var(vb), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)kVecOccupancySmem));
+    }
     CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                             (int)bulk_smem_bytes(p)));
     CU(cudaFuncSetAttribute(persistent_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -392,7 +407,7 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         pl.fn = pick_phase_vec_var(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
-        pl.smem = 0;
+        pl.smem = ctas == cap ? kVecOccupancySmem : 0;
         return SPARBIT_OK;
     }
     if (rs.copy == SPARBIT_COPY_BULK) {
@@ -415,7 +430,7 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         pl.fn = pick_phase_vec(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
-        pl.smem = 0;
+        pl.smem = ctas == cap ? kVecOccupancySmem : 0;
     }
     return SPARBIT_OK;
 }

@@ -75,9 +75,10 @@ struct CopyLoc {
     uint32_t src_rank, dst_rank, src_slot, dst_slot;
 };
 
-SPB_HD uint32_t wrap_slot(int64_t v, uint32_t P) {
-    if (v < 0) v += P;
-    if (v >= (int64_t)P) v -= P;
+// All slot arithmetic fits 32 bits: P <= 2^24, bases are below 2P and |j * step| < P.
+SPB_HD uint32_t wrap_slot(int32_t v, uint32_t P) {
+    if (v < 0) v += (int32_t)P;
+    if (v >= (int32_t)P) v -= (int32_t)P;
     return (uint32_t)v;
 }
 
@@ -93,12 +94,12 @@ SPB_HD CopyLoc locate_copy(const PhaseDesc& d, uint32_t P, uint32_t r, uint32_t 
     c.dst_rank = t >= P ? t - P : t;
     const uint32_t rr = r & d.rank_mask;
     const bool odd = (r & 1u) != 0;
-    int64_t s = (int64_t)d.src_rcoef * rr + (odd ? d.src_off_odd : d.src_off);
-    if (s >= (int64_t)P) s -= P;
-    c.src_slot = wrap_slot(s + (int64_t)j * d.src_step, P);
-    int64_t u = (int64_t)d.dst_rcoef * rr + (odd ? d.dst_off_odd : d.dst_off);
-    if (u >= (int64_t)P) u -= P;
-    c.dst_slot = wrap_slot(u + (int64_t)j * d.dst_step, P);
+    uint32_t s = (d.src_rcoef ? rr : 0u) + (odd ? d.src_off_odd : d.src_off);
+    if (s >= P) s -= P;
+    c.src_slot = wrap_slot((int32_t)s + (int32_t)j * d.src_step, P);
+    uint32_t u = (d.dst_rcoef ? rr : 0u) + (odd ? d.dst_off_odd : d.dst_off);
+    if (u >= P) u -= P;
+    c.dst_slot = wrap_slot((int32_t)u + (int32_t)j * d.dst_step, P);
     return c;
 }
 
