@@ -161,7 +161,6 @@ size_t bulk_smem_bytes(const sparbit_plan_s* p) {
 }
 
 const void* pick_phase_vec(int vbytes);
-const void* pick_phase_vec_var(int vbytes);
 
 int ensure_device(sparbit_plan_s* p) {
     if (p->dev_ready) {
@@ -203,8 +202,6 @@ int ensure_device(sparbit_plan_s* p) {
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
     for (int vb = 1; vb <= 16; vb *= 2) {
         CU(cudaFuncSetAttribute(pick_phase_vec(vb), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)kVecOccupancySmem));
-        CU(cudaFuncSetAttribute(pick_phase_vec_var(vb), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)kVecOccupancySmem));
     }
     CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -407,7 +404,8 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         pl.fn = pick_phase_vec_var(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
-        pl.smem = ctas == cap ? kVecOccupancySmem : 0;
+        pl.smem = 0;  // no occupancy cap here: this kernel reads its task list and the size table
+                      // through L1, which a large shared-memory carve-out would shrink (measured)
         return SPARBIT_OK;
     }
     if (rs.copy == SPARBIT_COPY_BULK) {
