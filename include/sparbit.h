@@ -85,7 +85,8 @@ enum {
 
 /* Which copy engine a phase uses. */
 enum {
-    SPARBIT_COPY_AUTO = 0,   /* BULK for 16-byte aligned buffers and m >= 32 KiB, else VECTOR */
+    SPARBIT_COPY_AUTO = 0,   /* BULK for 16-byte aligned buffers, m >= 8 KiB and about 1 GB or more
+                                moved by the collective (2*P*(P-1)*m >= 10^9), else VECTOR */
     SPARBIT_COPY_VECTOR = 1, /* warp-cooperative ld/st.global, 16/8/4/2/1-byte vectors */
     SPARBIT_COPY_BULK = 2    /* cp.async.bulk global->shared->global ring (needs 16-byte
                                 alignment of buffers and m); falls back to VECTOR otherwise */

@@ -317,11 +317,16 @@ Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv) {
     const uint64_t m = p->sched.m;
     const bool bulk_possible = r.vbytes == 16;
     int copy = p->copy_req;
-    // measured on B200 (P = 256 sweep): with about 32 KiB of loads in flight per SM both engines
-    // reach the copy peak for blocks >= 32 KiB, the bulk engine a little ahead; below that the
-    // per-operation cost of a bulk copy shows and the vector engine wins
-    if (copy == SPARBIT_COPY_AUTO)
-        copy = (bulk_possible && m >= (32u << 10)) ? SPARBIT_COPY_BULK : SPARBIT_COPY_VECTOR;
+    // measured on B200 (P = 61 .. 509, m = 4 KiB .. 256 KiB): with about 32 KiB of loads in flight per
+    // SM both engines reach the copy peak; the bulk engine is 1-4 % ahead once blocks are >= 8 KiB
+    // and the collective is in the bandwidth regime (about 1 GB moved or more); below that its
+    // per-pass set-up (ring and mbarrier initialisation) and per-operation cost show and the
+    // vector engine wins
+    if (copy == SPARBIT_COPY_AUTO) {
+        const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
+        copy = (bulk_possible && m >= (8u << 10) && moved >= (unsigned __int128)1000000000) ? SPARBIT_COPY_BULK
+                                                                                            : SPARBIT_COPY_VECTOR;
+    }
     if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
     if (p->variable) copy = SPARBIT_COPY_VECTOR;  // variable block sizes run on the vector engine
     r.copy = copy;
