@@ -38,14 +38,16 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 7700.0  # HBM3e of the HGX B200 (8000 on DGX); context only, not the roofline's peak
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, measured with
-# one-pass ncu captures of this benchmark at full size (bytes; absent = not captured)
-NCU_TRAFFIC_BYTES = {
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from ncu captures
+# of this benchmark's own kernels: bytes, and the summary under profiles/ that holds the capture's
+# command and figures (a configuration that is not listed was not captured: traffic = null)
+NCU_TRAFFIC = {
     # persistent_bulk_kernel, whole collective: 4.16 GB read + 4.25 GB written
-    "sparbit:P256:m65536:persistent:bulk": 8.41e9,
+    "sparbit:P256:m65536:persistent:bulk": (8.41e9, "profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md"),
     # phase_bulk_kernel, last phase: 2.15 GB read + 2.10 GB written
-    "sparbit:P256:m65536:graph:bulk": 4.25e9,
+    "sparbit:P256:m65536:graph:bulk": (4.25e9, "profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md"),
 }
+MIN_TIMED_MS = 250.0   # the timed rounds together last at least this long, whatever --steps is
 
 
 def effective_bytes(P: int, m: int) -> int:
@@ -136,6 +138,15 @@ def whole_job_value(world: int, P: int, m: int, ms_per_step: float) -> float:
     return world * effective_bytes(P, m) / (ms_per_step * 1e-3) / 1e9
 
 
+def workload_config(algo: str, P: int, m: int, world: int) -> dict:
+    """The part of the JSON line that names the workload; the same for both arms."""
+    return {"workload": f"{algo} allgather, P={P} virtual ranks, m={m} B blocks",
+            "P": P, "block_bytes": m, "algo": algo,
+            "l2": "inputs larger than L2 (no flush needed)" if P * P * m > (256 << 20)
+                  else "working set may sit in L2 (latency regime, reported as such)",
+            "parallelism": "replicas only" if world > 1 else "1 GPU"}
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -210,9 +221,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": f"sparbit allgather, P={P} virtual ranks, m={m} B blocks"
-                               + (f" (sampled at m={ms} B)" if ms != m else ""),
-                   "P": P, "block_bytes": ms, "algo": "sparbit"},
+        "config": workload_config("sparbit", P, m, world), "sampled_block_bytes": ms,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "checked": ok,
@@ -266,25 +275,40 @@ def run_ours(args):
         stream.synchronize()
         assert plan.status() == sp.OK
 
+        # rounds: each round is exactly --steps collectives between a barrier + synchronize on
+        # both sides; enough rounds that the timed work lasts MIN_TIMED_MS, so that neither one
+        # noisy neighbour nor a handful of clock samples decides the number
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for it in range(args.steps):
+            plan.allgather(sends[it & 1], recv, stream)
+        e1.record(stream)
+        stream.synchronize()
+        est_ms = max_over_ranks(e0.elapsed_time(e1), dev, use_dist)   # one untimed round sizes the run
+        rounds = int(min(200, max(1, -(-MIN_TIMED_MS // max(est_ms, 1e-3)))))
+
         sampler = ClockSampler(local)
         if rank == 0:
             sampler.start()
             time.sleep(0.25)
         k0, g0 = plan.launch_counts()
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-        barrier()
+        round_ms, per_ms = [], []
         t_wall0 = time.time()
-        ev[0].record(stream)
-        for it in range(args.steps):
-            plan.allgather(sends[it & 1], recv, stream)
-            ev[it + 1].record(stream)
-        stream.synchronize()
-        barrier()
+        for _ in range(rounds):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            barrier()
+            ev[0].record(stream)
+            for it in range(args.steps):
+                plan.allgather(sends[it & 1], recv, stream)
+                ev[it + 1].record(stream)
+            stream.synchronize()
+            barrier()
+            round_ms.append(max_over_ranks(ev[0].elapsed_time(ev[-1]), dev, use_dist))
+            per_ms += [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
         t_wall1 = time.time()
         k1, g1 = plan.launch_counts()
     assert plan.status() == sp.OK
-    total_ms = ev[0].elapsed_time(ev[-1])
-    per_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
     # the last collective's result, checked against the result's definition on the device
@@ -292,8 +316,7 @@ def run_ours(args):
     view = recv.view(P, P * m)
     checked = all(bool(torch.equal(view[r], last_send)) for r in (0, P // 3, P - 1))
 
-    max_total_ms = max_over_ranks(total_ms, dev, use_dist)
-    ms_per_step = max_total_ms / args.steps
+    ms_per_step = float(np.median(round_ms)) / args.steps   # the median round, slowest rank
     value = whole_job_value(world, P, m, ms_per_step)
 
     # end to end through the host-buffer entry point (pinned host memory; H2D + D2H inside)
@@ -322,7 +345,7 @@ def run_ours(args):
     # the dominant kernel on its own, for the roofline entry: the whole collective when it is one
     # kernel (persistent, cluster), else the last schedule step (half of all bytes for a power of
     # two P), launched exactly as inside the collective and timed with events on the same stream
-    launches_per_step = (k1 - k0) / args.steps
+    launches_per_step = (k1 - k0) / (args.steps * rounds)
     one_kernel = launches_per_step <= 1
     per_pass_us = None
     if one_kernel and plan.exec_mode == sp.EXEC_PERSISTENT:
@@ -361,7 +384,8 @@ def run_ours(args):
         key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[plan.exec_mode]}:{sp.COPY_NAMES[plan.copy_path]}"
         roofline = {
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": peak_src,
+            "traffic": NCU_TRAFFIC.get(key, (None, None))[0],
+            "traffic_source": NCU_TRAFFIC.get(key, (None, None))[1], "peak_source": peak_src,
             "kernel": f"{sp.EXEC_NAMES[plan.exec_mode]} executor, {sp.COPY_NAMES[plan.copy_path]} engine: "
                       f"{dom_name} ({launches_per_step:g} launch(es) per collective)",
             "algorithmic_bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
@@ -375,19 +399,18 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-            "config": {"workload": f"{args.algo} allgather, P={P} virtual ranks, m={m} B blocks "
-                                   f"({P * P * m / 2**30:.3g} GiB of receive buffers per GPU)",
-                       "P": P, "block_bytes": m, "algo": args.algo,
-                       "exec": sp.EXEC_NAMES[plan.exec_mode], "copy": sp.COPY_NAMES[plan.copy_path],
-                       "l2": "inputs larger than L2 (no flush needed)" if P * P * m > (256 << 20)
-                             else "working set may sit in L2 (latency regime, reported as such)",
-                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "config": workload_config(args.algo, P, m, world),
+            "executor": {"exec": sp.EXEC_NAMES[plan.exec_mode], "copy": sp.COPY_NAMES[plan.copy_path],
+                         "recv_GiB_per_gpu": round(P * P * m / 2**30, 3)},
+            "rounds": rounds, "timed_ms": float(sum(round_ms)),
+            "ms_per_step_rounds": {"min": min(round_ms) / args.steps, "median": ms_per_step,
+                                   "max": max(round_ms) / args.steps},
             "us_per_collective": {"min": min(per_ms) * 1e3, "avg": avg_ms * 1e3, "max": max(per_ms) * 1e3},
             "pct_of_hbm_peak": 100.0 * value / world / peak,
             "pct_of_nominal_hbm": 100.0 * value / world / NOMINAL_HBM_GBS,
             "GBps_from_min_time": world * effective_bytes(P, m) / (min(per_ms) * 1e-3) / 1e9,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
-            "gpu_launches": int(k1 - k0), "graph_launches": int(g1 - g0),
+            "gpu_launches": int((k1 - k0) // rounds), "graph_launches": int((g1 - g0) // rounds),
             "clocks": clocks, "checked": bool(checked),
         }
         print(json.dumps(line), flush=True)
@@ -458,7 +481,14 @@ def run_sweep(args):
              "cluster": sp.EXEC_CLUSTER}
     copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
     stream = torch.cuda.Stream(device=dev)
+    cores = min(os.cpu_count() or 1, 16)
     for P, m, names in points:
+        # the CPU oracle on the same point (Sparbit, all host threads up to 16, best of 2), where
+        # its buffers stay at or below 1 GiB
+        oracle_ms = None
+        if P * P * m <= (1 << 30):
+            t, ok = time_oracle(P, m, steps=2, warmup=0, threads=cores, seed=args.seed)
+            oracle_ms = round(min(t) * 1e3, 3) if ok else None
         sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
         recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
         work = None
@@ -497,6 +527,9 @@ def run_sweep(args):
                         "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
                         "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
                         "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
+                        "pct_nominal_hbm": round(100 * effective_bytes(P, m) / avg / 1e3 / NOMINAL_HBM_GBS, 1),
+                        "oracle_ms": oracle_ms if name == "sparbit" else None,
+                        "oracle_cores": cores if name == "sparbit" and oracle_ms is not None else None,
                         "checked": ok}), flush=True)
                     plan.destroy()
         del sends, recv, work
@@ -557,6 +590,29 @@ def run_allgatherv(args):
         plan.destroy()
         del sends, recv
         torch.cuda.empty_cache()
+    return 0
+
+
+def run_mapping_study(args):
+    """Section III-C in numbers, for G devices instead of machines (host only, no GPU): how many
+    blocks of every Sparbit step leave their device under the sequential and the cyclic mapping of
+    ranks to devices.  One JSON line per (P, G, mapping); multiply blocks by m for bytes."""
+    import paper_2109_08751_b200 as sp
+    for P in (256, 1000):
+        plan = sp.Plan(P, 1)
+        for G in (2, 4, 8):
+            for name, mp in (("sequential", sp.MAP_SEQUENTIAL), ("cyclic", sp.MAP_CYCLIC)):
+                steps = []
+                for st in range(plan.num_steps):
+                    d, n, _ = plan.step_info(st)
+                    b = plan.partition(G, mp, st)
+                    steps.append({"distance": d, "blocks": int(b.sum()), "cross": int(b.sum() - np.trace(b)),
+                                  "busiest_link": int((b - np.diag(np.diag(b))).max())})
+                total = sum(x["blocks"] for x in steps)
+                cross = sum(x["cross"] for x in steps)
+                print(json.dumps({"P": P, "G": G, "mapping": name, "total_blocks": total, "cross_blocks": cross,
+                                  "cross_pct": round(100.0 * cross / total, 2), "steps": steps}), flush=True)
+        plan.destroy()
     return 0
 
 
@@ -643,11 +699,16 @@ def main():
                          "grid of 64 process counts x 21 block sizes (about a quarter of an hour)")
     ap.add_argument("--cpu-sweep", action="store_true",
                     help="time the CPU oracle of every algorithm on the host cores (no GPU)")
+    ap.add_argument("--mapping-study", action="store_true",
+                    help="blocks per Sparbit step that cross devices under the sequential and cyclic "
+                         "rank-to-device mappings (host only), one JSON line per (P, G, mapping)")
     ap.add_argument("--allgatherv", action="store_true",
                     help="variable block sizes on the Sparbit schedule, one JSON line per size mix")
     args = ap.parse_args()
     if args.cpu_sweep:
         return run_cpu_sweep(args)
+    if args.mapping_study:
+        return run_mapping_study(args)
     if args.allgatherv:
         return run_allgatherv(args)
     if args.heatmap:

@@ -220,12 +220,46 @@ int sparbit_plan_messages(const sparbit_plan_t* plan, int phase, sparbit_msg* ou
  * own index function and checked for (a) ranks and slots inside their buffers, (b) no location
  * read before an earlier pass has filled it, (c) inside a pass, no location written twice and
  * none both read and written, (d) every receive slot written exactly once over the collective.
- * The paper's Section III-B states (c) and (d) as the purpose of withholding blocks ("double
- * writing the same block ... is not desirable").  Returns SPARBIT_OK, or SPARBIT_ERR_ARG with the
+ * Section III-B withholds blocks for exactly this purpose: so that no slot is written twice.
+ * Returns SPARBIT_OK, or SPARBIT_ERR_ARG with the
  * offending phase in *bad_phase (may be NULL; last phase + 1 = the final count), SPARBIT_ERR_LIMIT
  * for P > 8192 (the check needs P*P bytes of host memory), SPARBIT_ERR_NOMEM.  Host-only.
  */
 int sparbit_plan_validate(const sparbit_plan_t* plan, int* bad_phase);
+
+/* ---- placement of the ranks on several devices (host-only, no CUDA call) --------------------
+ *
+ * Section III-C of the paper discusses how the mapping of processes to machines decides how much
+ * of each step's traffic crosses the network: with the sequential mapping neighbouring ranks
+ * share a machine, so Sparbit's late steps (small distance, most of the data) stay inside it;
+ * with the cyclic mapping they are the ones that leave it.  These calls state the same thing for
+ * G devices: they split the messages of a phase into the copies a device performs inside its own
+ * memory and the blocks it has to hand to each other device.  They only describe the split; this
+ * library executes collectives on one device.
+ */
+enum {
+    SPARBIT_MAP_SEQUENTIAL = 0, /* device g holds ranks [floor(g*P/G), floor((g+1)*P/G)) */
+    SPARBIT_MAP_CYCLIC = 1      /* rank r sits on device r mod G */
+};
+
+/* The device that holds `rank` when P ranks are placed on G devices; -1 on a bad argument. */
+int sparbit_rank_device(int P, int G, int mapping, int rank);
+
+/*
+ * Counts the single-block messages of one phase (-1 .. last phase) by sending and receiving
+ * device: blocks[s * G + d] = blocks that ranks on device s send to ranks on device d in that
+ * phase (s == d: copies that stay local).  blocks must hold G*G entries; multiply by m for
+ * bytes.  1 <= G <= 4096.  Errors: ERR_ARG, ERR_NOMEM.
+ */
+int sparbit_plan_partition(const sparbit_plan_t* plan, int G, int mapping, int phase, uint64_t* blocks);
+
+/*
+ * The messages of one phase that go from device src_device to device dst_device (equal: the
+ * local copy list of that device), same record and conventions as sparbit_plan_messages.
+ * Over all G*G pairs every message of the phase appears exactly once.
+ */
+int sparbit_plan_partition_messages(const sparbit_plan_t* plan, int G, int mapping, int phase, int src_device,
+                                    int dst_device, sparbit_msg* out, size_t cap, size_t* n);
 
 /* Bytes of workspace the plan needs: 0, or P*P*m for Bruck. */
 size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* plan);

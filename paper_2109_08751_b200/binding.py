@@ -19,6 +19,7 @@ ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK, ALGO_NEIGHBOR_EXCH
 EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_CLUSTER = range(5)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
 SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
+MAP_SEQUENTIAL, MAP_CYCLIC = range(2)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
               ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}
@@ -45,6 +46,9 @@ SYMBOLS = {
     "sparbit_plan_step_info": (_i, [_vp, _i, _pi, _pi, _pi]),
     "sparbit_plan_messages": (_i, [_vp, _i, _vp, _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_validate": (_i, [_vp, _pi]),
+    "sparbit_rank_device": (_i, [_i, _i, _i, _i]),
+    "sparbit_plan_partition": (_i, [_vp, _i, _i, _i, ctypes.POINTER(_u64)]),
+    "sparbit_plan_partition_messages": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_workspace_bytes": (_sz, [_vp]),
     "sparbit_plan_set_workspace": (_i, [_vp, _vp, _sz]),
     "sparbit_plan_set_copy_path": (_i, [_vp, _i]),
@@ -164,6 +168,24 @@ class Plan:
         if n.value:
             _check(lib.sparbit_plan_messages(self._h, phase, out.ctypes.data, n.value, ctypes.byref(n)),
                    "sparbit_plan_messages")
+        return out
+
+    def partition(self, G: int, mapping: int, phase: int) -> np.ndarray:
+        """blocks[s, d] = blocks ranks on device s send to ranks on device d in `phase`."""
+        out = np.zeros((G, G), dtype=np.uint64)
+        _check(lib.sparbit_plan_partition(self._h, G, mapping, phase,
+                                          out.ctypes.data_as(ctypes.POINTER(_u64))), "sparbit_plan_partition")
+        return out
+
+    def partition_messages(self, G: int, mapping: int, phase: int, src_device: int, dst_device: int) -> np.ndarray:
+        n = _sz()
+        _check(lib.sparbit_plan_partition_messages(self._h, G, mapping, phase, src_device, dst_device, None, 0,
+                                                   ctypes.byref(n)), "sparbit_plan_partition_messages")
+        out = np.zeros(n.value, dtype=MSG_DTYPE)
+        if n.value:
+            _check(lib.sparbit_plan_partition_messages(self._h, G, mapping, phase, src_device, dst_device,
+                                                       out.ctypes.data, n.value, ctypes.byref(n)),
+                   "sparbit_plan_partition_messages")
         return out
 
     def validate(self) -> None:

@@ -186,19 +186,21 @@ int ensure_device(sparbit_plan_s* p) {
         table.push_back(p->sched.fused_first);
         table.insert(table.end(), p->sched.phases.begin() + 2, p->sched.phases.end());
     }
+    // a set-up that failed half way is run again by the next launch: what it already allocated is
+    // kept and filled again, never allocated twice
     const size_t n = table.size();
-    CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
+    if (!p->d_descs) CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
     CU(cudaMemcpy(p->d_descs, table.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
     if (p->variable) {
-        CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
+        if (!p->d_voff) CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
         CU(cudaMemcpy(p->d_voff, p->voff.data(), p->voff.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
         const size_t nt = p->vtasks.size() ? p->vtasks.size() : 1;
-        CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(unsigned long long)));
+        if (!p->d_vtasks) CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(unsigned long long)));
         if (p->vtasks.size())
             CU(cudaMemcpy(p->d_vtasks, p->vtasks.data(), p->vtasks.size() * sizeof(unsigned long long),
                           cudaMemcpyHostToDevice));
     }
-    CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
+    if (!p->d_ctl) CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
     for (int vb = 1; vb <= 16; vb *= 2) {
         CU(cudaFuncSetAttribute(pick_phase_vec(vb), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -882,6 +884,9 @@ int sparbit_allgather_host(sparbit_plan_t* p, const void* host_send, void* host_
     if (send_bytes == 0) return SPARBIT_OK;
     if (!host_send || !host_recv) return SPARBIT_ERR_ARG;
     if (ranges_overlap(host_send, send_bytes, host_recv, recv_bytes)) return SPARBIT_ERR_ALIAS;
+    // bind the plan to the current device (or refuse another one) before anything is allocated
+    int rc0 = ensure_device(p);
+    if (rc0) return rc0;
     if (!p->stage_send) CU(cudaMalloc(&p->stage_send, send_bytes));
     if (!p->stage_recv) CU(cudaMalloc(&p->stage_recv, recv_bytes));
     if (s.algo == ALGO_BRUCK && !p->work) {
@@ -920,6 +925,43 @@ int sparbit_plan_messages(const sparbit_plan_t* p, int phase, sparbit_msg* out, 
         expand_phase(p->sched, phase, v);
         const size_t k = v.size() < cap ? v.size() : cap;
         memcpy(out, v.data(), k * sizeof(Msg));
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    return SPARBIT_OK;
+}
+
+int sparbit_rank_device(int P, int G, int mapping, int rank) {
+    if (P < 1 || G < 1 || rank < 0 || rank >= P) return -1;
+    if (mapping != SPARBIT_MAP_SEQUENTIAL && mapping != SPARBIT_MAP_CYCLIC) return -1;
+    return (int)rank_device((uint32_t)P, (uint32_t)G, mapping, (uint32_t)rank);
+}
+
+int sparbit_plan_partition(const sparbit_plan_t* p, int G, int mapping, int phase, uint64_t* blocks) {
+    if (!p || !blocks || G < 1 || G > 4096 || phase < -1 || phase > p->sched.last_phase()) return SPARBIT_ERR_ARG;
+    if (mapping != SPARBIT_MAP_SEQUENTIAL && mapping != SPARBIT_MAP_CYCLIC) return SPARBIT_ERR_ARG;
+    try {
+        std::vector<uint64_t> v;
+        partition_counts(p->sched, phase, (uint32_t)G, mapping, v);
+        memcpy(blocks, v.data(), v.size() * sizeof(uint64_t));
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_partition_messages(const sparbit_plan_t* p, int G, int mapping, int phase, int src_device,
+                                    int dst_device, sparbit_msg* out, size_t cap, size_t* n) {
+    if (!p || !n || G < 1 || G > 4096 || phase < -1 || phase > p->sched.last_phase()) return SPARBIT_ERR_ARG;
+    if (mapping != SPARBIT_MAP_SEQUENTIAL && mapping != SPARBIT_MAP_CYCLIC) return SPARBIT_ERR_ARG;
+    if (src_device < 0 || src_device >= G || dst_device < 0 || dst_device >= G) return SPARBIT_ERR_ARG;
+    if (cap > 0 && !out) return SPARBIT_ERR_ARG;
+    try {
+        std::vector<Msg> v;
+        partition_messages(p->sched, phase, (uint32_t)G, mapping, (uint32_t)src_device, (uint32_t)dst_device, v);
+        *n = v.size();
+        const size_t k = v.size() < cap ? v.size() : cap;
+        if (k) memcpy(out, v.data(), k * sizeof(Msg));
     } catch (const std::bad_alloc&) {
         return SPARBIT_ERR_NOMEM;
     }

@@ -9,8 +9,8 @@
 //           sizes.
 //   bulk    cp.async.bulk global -> shared -> global through a ring of shared-memory stages, one
 //           elected lane per warp driving its own ring; completion of loads through mbarriers,
-//           of stores through bulk async-groups.  No cluster multicast anywhere: every block has
-//           one destination (two in the fused first pass, issued as two stores).
+//           of stores through bulk async-groups.  Every load fills one CTA's own shared memory and
+//           every block has one destination (two in the fused first pass, issued as two stores).
 //
 // and four ways to sequence passes: one kernel per pass, chained by programmatic dependent launch
 // (plain stream launches or a CUDA graph); one persistent cooperative kernel with a bounded-wait

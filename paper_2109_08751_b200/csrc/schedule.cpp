@@ -281,4 +281,27 @@ void expand_phase(const Schedule& s, int phase, std::vector<Msg>& out) {
         }
 }
 
+void partition_counts(const Schedule& s, int phase, uint32_t G, int mapping, std::vector<uint64_t>& blocks) {
+    const PhaseDesc& d = s.phase(phase);
+    blocks.assign((size_t)G * G, 0);
+    for (uint32_t r = 0; r < s.P; r++) {
+        const uint32_t from = rank_device(s.P, G, mapping, r);
+        for (uint32_t j = 0; j < d.copies; j++) {
+            const CopyLoc c = locate_copy(d, s.P, r, j);
+            blocks[(size_t)from * G + rank_device(s.P, G, mapping, c.dst_rank)] += d.run;
+        }
+    }
+}
+
+void partition_messages(const Schedule& s, int phase, uint32_t G, int mapping, uint32_t src_dev, uint32_t dst_dev,
+                        std::vector<Msg>& out) {
+    std::vector<Msg> all;
+    expand_phase(s, phase, all);
+    out.clear();
+    for (const Msg& msg : all)
+        if (rank_device(s.P, G, mapping, (uint32_t)msg.src_rank) == src_dev &&
+            rank_device(s.P, G, mapping, (uint32_t)msg.dst_rank) == dst_dev)
+            out.push_back(msg);
+}
+
 }  // namespace spb

@@ -49,4 +49,23 @@ void expand_phase(const Schedule& s, int phase, std::vector<Msg>& out);
 // Number of single-block messages of one phase.
 uint64_t phase_message_count(const Schedule& s, int phase);
 
+// Placement of the P ranks on G devices (Section III-C).  Sequential keeps neighbouring ranks
+// together: device g holds the ranks [floor(g*P/G), floor((g+1)*P/G)).  Cyclic deals them out
+// round robin: rank r sits on device r mod G.
+enum Mapping { MAP_SEQUENTIAL = 0, MAP_CYCLIC = 1 };
+
+inline uint32_t rank_device(uint32_t P, uint32_t G, int mapping, uint32_t r) {
+    if (mapping == MAP_CYCLIC) return r % G;
+    return (uint32_t)((((uint64_t)r + 1) * G - 1) / P);
+}
+
+// Splits the single-block messages of one phase by (device of the sender, device of the
+// receiver).  blocks gets G*G counts, row = sending device; the diagonal is what stays local.
+void partition_counts(const Schedule& s, int phase, uint32_t G, int mapping, std::vector<uint64_t>& blocks);
+
+// The messages of one phase that go from device src_dev to device dst_dev (src_dev == dst_dev:
+// the local copy list of that device), in the order expand_phase lists them.
+void partition_messages(const Schedule& s, int phase, uint32_t G, int mapping, uint32_t src_dev, uint32_t dst_dev,
+                        std::vector<Msg>& out);
+
 }  // namespace spb

@@ -81,6 +81,92 @@ def test_config5_sweep(dev, m, algo):
     full_compare(dev, 256, m, algo, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 5, iters=1)
 
 
+@pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_NEIGHBOR_EXCHANGE])
+def test_config5_comparators_at_64k(dev, algo):
+    """The comparators at the headline block size, whole receive space against the oracle."""
+    full_compare(dev, 256, 64 * 1024, algo, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 5, iters=1)
+
+
+def sampled_compare(dev, plan, ref, P, offsets, host_send, recv, samples=192, seed=12345):
+    """Sampled (rank, slot) outputs through the oracle's message lists, then the whole state
+    against the property that holds at any size: every receive buffer is the concatenation of
+    the send blocks.  offsets[b] .. offsets[b+1] is block b inside a receive buffer."""
+    T = int(offsets[P])
+    send = torch.from_numpy(host_send).to(dev)
+    for k in si.sample_indices(samples, P * P, seed=seed):
+        r, b = divmod(int(k), P)
+        path = ref.trace(r, b)
+        origin = int(path[0]["src_rank"])
+        lo, hi = int(offsets[b]), int(offsets[b + 1])
+        got = recv[r * T + lo:r * T + hi].cpu().numpy()
+        assert np.array_equal(got, host_send[int(offsets[origin]):int(offsets[origin + 1])]), (r, b)
+    view = recv.view(P, T)
+    for r in range(P):
+        assert torch.equal(view[r], send), r
+
+
+def test_config5_bruck_at_64k_sampled(dev):
+    """Bruck at the headline block size: the oracle would need 8 GiB of host memory for its two
+    spaces, so sampled outputs are traced through its message lists (rotation included)."""
+    P, m = 256, 64 * 1024
+    plan = sp.Plan(P, m, sp.ALGO_BRUCK, sp.EXEC_AUTO)
+    ref = oracle.Plan(oracle.BRUCK, P)
+    host_send = si.send_blocks(P, m, si.BASE_SEED + 5).reshape(-1)
+    send = torch.from_numpy(host_send).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    work = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.set_workspace(work, P * P * m)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    sampled_compare(dev, plan, ref, P, np.arange(P + 1, dtype=np.int64) * m, host_send, recv)
+    plan.destroy()
+
+
+# Receive spaces beyond 4 GiB: byte offsets that do not fit 32 bits, on every engine and executor
+# (at the headline point P*P*m is exactly 2^32, so no offset there needs the 33rd bit).
+BIG_P, BIG_M = 272, 64 * 1024   # 4.85 GB of receive buffers, not a power of two, 9 steps
+
+
+@pytest.mark.parametrize("exec_mode,copy", [(sp.EXEC_GRAPH, sp.COPY_VECTOR), (sp.EXEC_PERSISTENT, sp.COPY_VECTOR),
+                                            (sp.EXEC_PERSISTENT, sp.COPY_BULK), (sp.EXEC_STREAM, sp.COPY_BULK)])
+def test_offsets_beyond_4gib(dev, exec_mode, copy):
+    P, m = BIG_P, BIG_M
+    assert P * P * m > 1 << 32
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    plan.set_copy_path(copy)
+    ref = oracle.Plan(oracle.SPARBIT, P)
+    host_send = si.send_blocks(P, m, si.BASE_SEED + 6).reshape(-1)
+    send = torch.from_numpy(host_send).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    assert plan.copy_path == copy
+    for k in si.sample_indices(8, P * P, seed=99):   # hop counts: one per set bit of the distance
+        r, b = divmod(int(k), P)
+        assert len(ref.trace(r, b)) - 1 == bin((r - b) % P).count("1")
+    sampled_compare(dev, plan, ref, P, np.arange(P + 1, dtype=np.int64) * m, host_send, recv)
+    plan.destroy()
+
+
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_GRAPH, sp.EXEC_PERSISTENT])
+def test_allgatherv_offsets_beyond_4gib(dev, exec_mode):
+    """Blocks of different sizes whose receive space P*T exceeds 4 GiB."""
+    P = BIG_P
+    counts = si.block_counts(P, 77, kind="mixed", unit=16, scale=BIG_M // 16 * 9 // 13)
+    offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    T = int(offsets[P])
+    assert P * T > 1 << 32
+    plan = sp.Plan.create_v(counts, sp.ALGO_SPARBIT, exec_mode)
+    ref = oracle.Plan(oracle.SPARBIT, P)
+    host_send = si.send_blocks_v(counts, si.BASE_SEED + 7)
+    send = torch.from_numpy(host_send).to(dev)
+    recv = torch.full((P * T,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    sampled_compare(dev, plan, ref, P, offsets, host_send, recv)
+    plan.destroy()
+
+
 @pytest.mark.parametrize("exec_mode,copy", [(sp.EXEC_AUTO, sp.COPY_AUTO), (sp.EXEC_GRAPH, sp.COPY_BULK),
                                             (sp.EXEC_PERSISTENT, sp.COPY_VECTOR)])
 def test_config5_headline_point_p256_m64k(dev, exec_mode, copy):

@@ -408,3 +408,45 @@ def test_partial_runs_compose():
 def test_zero_byte_blocks_are_a_no_op():
     recv, _ = oracle.allgather(oracle.SPARBIT, 8, 0, np.empty((8, 0), np.uint8))
     assert recv.shape == (8, 0)
+
+
+# ------------------------------------------------------------------ tracing a slot back to its origin
+@pytest.mark.parametrize("algo", ALGOS)
+def test_trace_leads_back_to_the_owner_of_the_slot(algo):
+    """Plan.trace follows the messages that fill (rank, slot) back to a send buffer.  Whatever
+    the algorithm, the walk must end at the send block of rank `slot` (Section II: slot j holds
+    rank j's block), start with the own-block copy of that rank, and be connected hop to hop."""
+    for P in ALL_P:
+        if not defined_for(algo, P):
+            continue
+        pl = plan(algo, P)
+        for r in range(P):
+            for b in range(P):
+                path = pl.trace(r, b)
+                assert int(path[0]["src_space"]) == oracle.SPACE_SEND
+                assert int(path[0]["src_rank"]) == b, (algo, P, r, b)
+                assert (int(path[-1]["dst_space"]), int(path[-1]["dst_rank"]), int(path[-1]["dst_slot"])) \
+                    == (oracle.SPACE_RECV, r, b)
+                for a, c in zip(path, path[1:]):
+                    assert (int(a["dst_space"]), int(a["dst_rank"]), int(a["dst_slot"])) \
+                        == (int(c["src_space"]), int(c["src_rank"]), int(c["src_slot"]))
+                    assert int(a["phase"]) < int(c["phase"])
+
+
+@pytest.mark.parametrize("P", ALL_P + [100, 272])
+def test_sparbit_trace_has_one_hop_per_set_bit_of_the_distance(P):
+    """Sections III-A/B: block b reaches rank b + k through the binomial tree rooted at b, i.e. by
+    adding the set bits of k from the most significant down - popcount(k) messages after the
+    own-block copy, at strictly decreasing distances that sum to k."""
+    pl = plan(oracle.SPARBIT, P)
+    pairs = [(r, b) for r in range(P) for b in range(P)] if P <= 64 else \
+        [divmod(int(k), P) for k in si.sample_indices(400, P * P, seed=P)]
+    for r, b in pairs:
+        k = (r - b) % P
+        path = pl.trace(r, b)
+        hops = path[1:]
+        assert len(hops) == bin(k).count("1"), (P, r, b)
+        dists = [(int(h["dst_rank"]) - int(h["src_rank"])) % P for h in hops]
+        assert dists == sorted(dists, reverse=True) and len(set(dists)) == len(dists)
+        assert sum(dists) == k and all(d & (d - 1) == 0 for d in dists)
+        assert all(int(h["src_slot"]) == b and int(h["dst_slot"]) == b for h in hops)
