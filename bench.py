@@ -249,7 +249,7 @@ def run_ours(args):
     algo = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
             "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}[args.algo]
     exec_mode = {"auto": sp.EXEC_AUTO, "persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH,
-                 "stream": sp.EXEC_STREAM, "cluster": sp.EXEC_CLUSTER}[args.exec]
+                 "stream": sp.EXEC_STREAM, "flow": sp.EXEC_FLOW}[args.exec]
     copy = {"auto": sp.COPY_AUTO, "vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}[args.copy]
 
     plan = sp.Plan(P, m, algo, exec_mode)
@@ -343,7 +343,7 @@ def run_ours(args):
         del hs, hr
 
     # the dominant kernel on its own, for the roofline entry: the whole collective when it is one
-    # kernel (persistent, cluster), else the last schedule step (half of all bytes for a power of
+    # kernel (persistent, flow), else the last schedule step (half of all bytes for a power of
     # two P), launched exactly as inside the collective and timed with events on the same stream
     launches_per_step = (k1 - k0) / (args.steps * rounds)
     one_kernel = launches_per_step <= 1
@@ -478,7 +478,7 @@ def run_sweep(args):
     algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
              "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}
     execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
-             "cluster": sp.EXEC_CLUSTER}
+             "flow": sp.EXEC_FLOW}
     copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
     stream = torch.cuda.Stream(device=dev)
     cores = min(os.cpu_count() or 1, 16)
@@ -495,14 +495,15 @@ def run_sweep(args):
         for name in names:
             if name == "bruck" and work is None:
                 work = torch.empty(P * P * m, dtype=torch.uint8, device=dev)
-            for ename, e in execs.items():
-                if ename == "cluster" and effective_bytes(P, m) > (64 << 20):
-                    continue
+            combos = [("auto", sp.EXEC_AUTO, "auto", sp.COPY_AUTO)]
+            if not args.sweep_auto_only:
+                combos += [(en, e, cn, c) for en, e in execs.items() for cn, c in copies.items()]
+            for ename, e, cname, c in combos:
                 if ename == "stream" and name in ("ring", "ne") and m >= 32768:
                     continue  # same kernels as the graph chain; skipped to bound the sweep
-                for cname, c in copies.items():
-                    if cname == "bulk" and (m % 16 or ename == "cluster"):
-                        continue
+                if cname == "bulk" and (m % 16 or ename == "flow"):
+                    continue
+                if True:
                     plan = sp.Plan(P, m, algos[name], e)
                     plan.set_copy_path(c)
                     if name == "bruck":
@@ -512,6 +513,7 @@ def run_sweep(args):
                             plan.allgather(sends[it & 1], recv, stream)
                         stream.synchronize()
                         ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
+                        k_before = plan.launch_counts()[0]
                         ev[0].record(stream)
                         for it in range(50):
                             plan.allgather(sends[it & 1], recv, stream)
@@ -523,6 +525,8 @@ def run_sweep(args):
                     avg = float(np.mean(us))
                     print(json.dumps({
                         "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
+                        "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
+                        "launches_per_collective": (plan.launch_counts()[0] - k_before) / 50,
                         "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
                         "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
                         "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
@@ -687,13 +691,15 @@ def main():
     ap.add_argument("--P", type=int, default=P_DEFAULT)
     ap.add_argument("--m", type=int, default=M_DEFAULT)
     ap.add_argument("--algo", choices=["sparbit", "ring", "ne", "rd", "bruck"], default="sparbit")
-    ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "cluster"], default="auto")
+    ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "flow"], default="auto")
     ap.add_argument("--copy", choices=["auto", "vector", "bulk"], default="auto")
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
+    ap.add_argument("--sweep-auto-only", action="store_true",
+                    help="with --sweep: only the executor and engine the library picks by itself")
     ap.add_argument("--heatmap", nargs="?", const="coarse", default=None, choices=["coarse", "paper"],
                     help="best algorithm per (P, m) cell, one JSON line per cell; 'paper' = the paper's "
                          "grid of 64 process counts x 21 block sizes (about a quarter of an hour)")

@@ -74,13 +74,19 @@ enum {
  * as ONE pass (the own block is read once from sendbuf and written both to its own slot and to
  * the first peer's): same state after phase 0, one pass less. */
 enum {
-    SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: the graph chain, at every size */
+    SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: FLOW for collectives that move 1 to
+                                    6 GB (SPARBIT_TUNE_FLOW_*), the graph chain otherwise */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
                                     re-parameterise the least recently used graph) */
     SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
-    SPARBIT_EXEC_CLUSTER = 4     /* one thread-block cluster, hardware cluster barrier per pass */
+    SPARBIT_EXEC_FLOW = 4        /* one cooperative kernel without grid barriers: Algorithm 1's
+                                    Waitall is kept per rank (counters of what each rank has
+                                    received), so a pass starts where its senders are ready while
+                                    the pass before is still finishing elsewhere.  Whole
+                                    collectives of fixed-size blocks of at least 32 vectors on the
+                                    vector engine; other calls run as GRAPH */
 };
 
 /* Which copy engine a phase uses. */
@@ -126,7 +132,7 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
  * unknown enum), ERR_OVERFLOW (P*P*block_bytes does not fit in 63 bits, or P > 2^24),
  * ERR_UNSUPPORTED (recursive doubling with P not a power of two, neighbor exchange with odd P:
  * Section II-A defines them for those P only), ERR_NOMEM.  Host-only.
- * Environment: when exec is AUTO, SPARBIT_EXEC=persistent|graph|stream|cluster replaces the
+ * Environment: when exec is AUTO, SPARBIT_EXEC=persistent|graph|stream|flow replaces the
  * automatic choice; SPARBIT_COPY=vector|bulk presets the copy engine (sparbit_plan_set_copy_path
  * still overrides it).  Other values are ignored.
  */
@@ -142,12 +148,13 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
  *   sendbuf   T bytes       rank r's block at byte offset off[r]
  *   recvbuf   P * T bytes   rank r's buffer at r * T, block j at + off[j]
  * The plan is then used with sparbit_allgather, sparbit_allgather_steps and
- * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Runs on the
- * vector copy engine with the graph or stream executor: exec must be AUTO, GRAPH or STREAM
- * (PERSISTENT, CLUSTER: ERR_UNSUPPORTED).  Bruck is refused (ERR_UNSUPPORTED: its rotated
- * workspace assumes equal blocks).  P is limited to 8192 here (ERR_LIMIT beyond: the plan keeps
- * one task-list entry per 4 KiB of every copy).  Other errors as for sparbit_plan_create.
- * Host-only.
+ * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Both copy
+ * engines (the bulk engine when all counts and the buffers are multiples of 16 bytes; COPY_AUTO
+ * applies its thresholds to the average block) and the GRAPH, STREAM and PERSISTENT executors;
+ * FLOW is refused (ERR_UNSUPPORTED: its work units assume equal blocks), and so is Bruck (its
+ * rotated workspace assumes equal blocks).  P is limited to 8192 here and P * T to 2^48 bytes
+ * (ERR_LIMIT, ERR_OVERFLOW beyond: the plan keeps one 16-byte task record per 4 KiB of every
+ * copy, with 48-bit offsets).  Other errors as for sparbit_plan_create.  Host-only.
  */
 int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, sparbit_plan_t** out);
 
@@ -271,6 +278,23 @@ int sparbit_plan_set_workspace(sparbit_plan_t* plan, void* dev, size_t bytes);
 /* Forces the copy engine (SPARBIT_COPY_*).  BULK silently runs as VECTOR for a call whose
  * buffers or m are not 16-byte aligned. */
 int sparbit_plan_set_copy_path(sparbit_plan_t* plan, int copy_path);
+
+/*
+ * Thresholds behind the automatic choices, per plan.  Defaults come from sweeps on B200; a value
+ * set here holds for all later calls on the plan (cached graphs are rebuilt).
+ */
+enum {
+    SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES = 0, /* COPY_AUTO: smallest m that gets the bulk engine (8 KiB) */
+    SPARBIT_TUNE_BULK_MIN_MOVED_BYTES = 1, /* COPY_AUTO: and only if 2*P*(P-1)*m reaches this (10^9) */
+    SPARBIT_TUNE_FLOW_UNITS_PER_WARP = 2,  /* EXEC_FLOW: a pass is cut into units of 1..4 warp spans
+                                              so that every warp gets at least about this many (1) */
+    SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS = 3,  /* EXEC_FLOW: largest unit, in warp spans of 1 KiB (8) */
+    SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (10^9) */
+    SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES = 5, /* ... and below this (6*10^9); GRAPH otherwise */
+    SPARBIT_TUNE_COUNT_ = 6
+};
+int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
+int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);
 
 /* What the plan resolved to: executor (SPARBIT_EXEC_*, never AUTO) and the copy engine the last
  * launch used (SPARBIT_COPY_*; AUTO before the first launch). */

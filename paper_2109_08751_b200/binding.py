@@ -16,15 +16,17 @@ OK = 0
 ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT = \
     range(1, 10)
 ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK, ALGO_NEIGHBOR_EXCHANGE = range(5)
-EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_CLUSTER = range(5)
+EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_FLOW = range(5)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
 SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
 MAP_SEQUENTIAL, MAP_CYCLIC = range(2)
+(TUNE_BULK_MIN_BLOCK_BYTES, TUNE_BULK_MIN_MOVED_BYTES, TUNE_FLOW_UNITS_PER_WARP, TUNE_FLOW_MAX_UNIT_SPANS,
+ TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES) = range(6)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
               ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}
 EXEC_NAMES = {EXEC_AUTO: "auto", EXEC_PERSISTENT: "persistent", EXEC_GRAPH: "graph", EXEC_STREAM: "stream",
-              EXEC_CLUSTER: "cluster"}
+              EXEC_FLOW: "flow"}
 COPY_NAMES = {COPY_AUTO: "auto", COPY_VECTOR: "vector", COPY_BULK: "bulk"}
 
 MSG_DTYPE = np.dtype([("phase", "<i4"), ("src_rank", "<i4"), ("dst_rank", "<i4"), ("src_space", "<i4"),
@@ -52,6 +54,8 @@ SYMBOLS = {
     "sparbit_plan_workspace_bytes": (_sz, [_vp]),
     "sparbit_plan_set_workspace": (_i, [_vp, _vp, _sz]),
     "sparbit_plan_set_copy_path": (_i, [_vp, _i]),
+    "sparbit_plan_set_tunable": (_i, [_vp, _i, _u64]),
+    "sparbit_plan_get_tunable": (_i, [_vp, _i, ctypes.POINTER(_u64)]),
     "sparbit_plan_exec_mode": (_i, [_vp]),
     "sparbit_plan_copy_path": (_i, [_vp]),
     "sparbit_plan_launch_counts": (_i, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
@@ -202,6 +206,14 @@ class Plan:
     def set_workspace(self, dev, nbytes: int) -> None:
         _check(lib.sparbit_plan_set_workspace(self._h, _ptr(dev), nbytes), "sparbit_plan_set_workspace")
         self._workspace = dev  # keep the owner alive
+
+    def set_tunable(self, key: int, value: int) -> None:
+        _check(lib.sparbit_plan_set_tunable(self._h, key, value), "sparbit_plan_set_tunable")
+
+    def get_tunable(self, key: int) -> int:
+        v = _u64()
+        _check(lib.sparbit_plan_get_tunable(self._h, key, ctypes.byref(v)), "sparbit_plan_get_tunable")
+        return int(v.value)
 
     def set_copy_path(self, path: int) -> None:
         _check(lib.sparbit_plan_set_copy_path(self._h, path), "sparbit_plan_set_copy_path")

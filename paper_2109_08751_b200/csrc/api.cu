@@ -36,7 +36,6 @@ constexpr int kVecBlock = 512;
 // P = 1000, m = 1 KiB: 348 us without the cap, 339 us with it).  Small grids do not ask for it:
 // there the early residency of the successor is what keeps a pass at 2.6 us.
 constexpr size_t kVecOccupancySmem = 100 * 1024;
-constexpr int kClusterBlock = 1024;
 
 struct GraphKey {
     const void* send = nullptr;
@@ -60,6 +59,7 @@ struct sparbit_plan_s {
     int exec_req = SPARBIT_EXEC_AUTO;
     int copy_req = SPARBIT_COPY_AUTO;
     int copy_last = SPARBIT_COPY_AUTO;
+    int exec_last = SPARBIT_EXEC_AUTO;
     void* work = nullptr;
     size_t work_bytes = 0;
 
@@ -70,9 +70,10 @@ struct sparbit_plan_s {
     uint64_t* d_voff = nullptr;
     // task lists of the variable-size kernels, one per descriptor of the device table order
     // (phases in order, then the fused first pass): entries, and where each list starts
-    std::vector<unsigned long long> vtasks;
+    std::vector<VarTask> vtasks;
     std::vector<size_t> vtask_lo, vtask_hi;  // per device-table index: [lo, hi) inside vtasks
-    unsigned long long* d_vtasks = nullptr;
+    VarTask* d_vtasks = nullptr;
+    VarRange* d_vranges = nullptr;           // the same ranges on the device (persistent executor)
 
     size_t send_bytes() const { return variable ? (size_t)voff.back() : (size_t)sched.P * sched.m; }
     size_t recv_bytes() const { return (size_t)sched.P * send_bytes(); }
@@ -84,9 +85,11 @@ struct sparbit_plan_s {
     int sm_count = 0;
     int coop = 0;
     int max_smem_optin = 0;
-    int cluster_ok = 0;
     PhaseDesc* d_descs = nullptr;
     unsigned* d_ctl = nullptr;  // [0] barrier counter, [1] status word
+    unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
+    unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
+    int flow_vbytes = 0;             // vector width those launches ran with
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -97,6 +100,16 @@ struct sparbit_plan_s {
     // lowers the achieved HBM bandwidth): 4 rings x 2 loads x 4 KiB
     uint32_t bulk_warps = 4;
     uint32_t bulk_stage_bytes = 4096;
+
+    // thresholds of the automatic choices (sparbit_plan_set_tunable); defaults from measured sweeps
+    uint64_t tune[SPARBIT_TUNE_COUNT_] = {
+        8u << 10,     // BULK_MIN_BLOCK_BYTES
+        1000000000u,  // BULK_MIN_MOVED_BYTES
+        1,            // FLOW_UNITS_PER_WARP
+        8,            // FLOW_MAX_UNIT_SPANS
+        1000000000u,  // FLOW_MIN_MOVED_BYTES
+        6000000000ull,  // FLOW_MAX_MOVED_BYTES
+    };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
     // that callers alternating between buffer sets never re-instantiate
@@ -127,7 +140,7 @@ struct sparbit_plan_s {
 namespace {
 
 // SPARBIT_EXEC / SPARBIT_COPY in the environment override what AUTO would pick (not an explicit
-// request): persistent|graph|stream|cluster and vector|bulk.  Anything else is ignored.
+// request): persistent|graph|stream|flow and vector|bulk.  Anything else is ignored.
 int env_choice(const char* name, const char* const* words, const int* values, int n, int fallback) {
     const char* v = getenv(name);
     if (!v) return fallback;
@@ -136,8 +149,8 @@ int env_choice(const char* name, const char* const* words, const int* values, in
     return fallback;
 }
 int env_exec(int fallback) {
-    static const char* const w[] = {"persistent", "graph", "stream", "cluster"};
-    static const int x[] = {SPARBIT_EXEC_PERSISTENT, SPARBIT_EXEC_GRAPH, SPARBIT_EXEC_STREAM, SPARBIT_EXEC_CLUSTER};
+    static const char* const w[] = {"persistent", "graph", "stream", "flow"};
+    static const int x[] = {SPARBIT_EXEC_PERSISTENT, SPARBIT_EXEC_GRAPH, SPARBIT_EXEC_STREAM, SPARBIT_EXEC_FLOW};
     return env_choice("SPARBIT_EXEC", w, x, 4, fallback);
 }
 int env_copy(int fallback) {
@@ -157,7 +170,7 @@ int map_sched_err(int e) {
 }
 
 size_t bulk_smem_bytes(const sparbit_plan_s* p) {
-    return (size_t)p->bulk_warps * kBulkStages * (p->bulk_stage_bytes + 8 + 32);
+    return (size_t)p->bulk_warps * (kBulkStages * (p->bulk_stage_bytes + 8 + 32) + kTaskQueue * 16);
 }
 
 const void* pick_phase_vec(int vbytes);
@@ -174,9 +187,6 @@ int ensure_device(sparbit_plan_s* p) {
     CU(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device));
     CU(cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device));
     CU(cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device));
-    int cc_major = 0;
-    CU(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, p->device));
-    p->cluster_ok = cc_major >= 9;
     // shrink the bulk ring if this device offers less shared memory than planned
     while (bulk_smem_bytes(p) > (size_t)p->max_smem_optin && p->bulk_stage_bytes > 1024) p->bulk_stage_bytes -= 1024;
     // descriptor table: the phases in order, then (if the schedule has one) the same sequence with
@@ -195,10 +205,16 @@ int ensure_device(sparbit_plan_s* p) {
         if (!p->d_voff) CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
         CU(cudaMemcpy(p->d_voff, p->voff.data(), p->voff.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
         const size_t nt = p->vtasks.size() ? p->vtasks.size() : 1;
-        if (!p->d_vtasks) CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(unsigned long long)));
+        if (!p->d_vtasks) CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(VarTask)));
         if (p->vtasks.size())
-            CU(cudaMemcpy(p->d_vtasks, p->vtasks.data(), p->vtasks.size() * sizeof(unsigned long long),
-                          cudaMemcpyHostToDevice));
+            CU(cudaMemcpy(p->d_vtasks, p->vtasks.data(), p->vtasks.size() * sizeof(VarTask), cudaMemcpyHostToDevice));
+        std::vector<VarRange> ranges(p->vtask_lo.size());
+        for (size_t i = 0; i < ranges.size(); i++) {
+            ranges[i].lo = p->vtask_lo[i];
+            ranges[i].count = p->vtask_hi[i] - p->vtask_lo[i];
+        }
+        if (!p->d_vranges) CU(cudaMalloc((void**)&p->d_vranges, ranges.size() * sizeof(VarRange)));
+        CU(cudaMemcpy(p->d_vranges, ranges.data(), ranges.size() * sizeof(VarRange), cudaMemcpyHostToDevice));
     }
     if (!p->d_ctl) CU(cudaMalloc((void**)&p->d_ctl, 2 * sizeof(unsigned)));
     CU(cudaMemset(p->d_ctl, 0, 2 * sizeof(unsigned)));
@@ -208,7 +224,11 @@ int ensure_device(sparbit_plan_s* p) {
     }
     CU(cudaFuncSetAttribute(phase_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                             (int)bulk_smem_bytes(p)));
-    CU(cudaFuncSetAttribute(persistent_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    CU(cudaFuncSetAttribute(persistent_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            (int)bulk_smem_bytes(p)));
+    CU(cudaFuncSetAttribute(persistent_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            (int)bulk_smem_bytes(p)));
+    CU(cudaFuncSetAttribute(phase_bulk_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                             (int)bulk_smem_bytes(p)));
     p->dev_ready = true;
     return SPARBIT_OK;
@@ -231,16 +251,16 @@ int pick_vector_bytes(const sparbit_plan_s* p, const void* send, const void* rec
 }
 
 // warp tasks of one phase on the vector engine (mirrors vec_phase)
-uint64_t vec_tasks(const PhaseDesc& d, uint32_t P, int vbytes) {
+uint64_t vec_tasks(const PhaseDesc& d, uint32_t P, int vbytes, int unroll = kVecUnroll) {
     const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
     const uint64_t n_copies = (uint64_t)P * d.copies;
     if (n_copies >> 32) return ~0ull;  // the kernels index copies with 32 bits
     if (vpc >= 32) {
-        const uint64_t span = 32ull * kVecUnroll;
+        const uint64_t span = 32ull * unroll;
         return n_copies * ((vpc + span - 1) / span);
     }
     if (vpc == 0) return 0;
-    const uint64_t per_task = (32 / vpc) * kVecUnroll;
+    const uint64_t per_task = (32 / vpc) * unroll;
     return (n_copies + per_task - 1) / per_task;
 }
 
@@ -251,7 +271,9 @@ uint64_t bulk_tasks(const PhaseDesc& d, uint32_t P, uint32_t stage_bytes) {
 template <typename V>
 const void* phase_vec_fn() { return (const void*)phase_vec_kernel<V>; }
 template <typename V>
-const void* persistent_vec_fn() { return (const void*)persistent_vec_kernel<V>; }
+const void* persistent_vec_fn(bool list) {
+    return list ? (const void*)persistent_vec_kernel<V, true> : (const void*)persistent_vec_kernel<V, false>;
+}
 
 const void* pick_phase_vec(int vbytes) {
     switch (vbytes) {
@@ -273,74 +295,25 @@ const void* pick_phase_vec_var(int vbytes) {
         default: return phase_vec_var_fn<unsigned char>();
     }
 }
-const void* pick_persistent_vec(int vbytes) {
+const void* pick_persistent_vec(int vbytes, bool list = false) {
     switch (vbytes) {
-        case 16: return persistent_vec_fn<uint4>();
-        case 8: return persistent_vec_fn<uint2>();
-        case 4: return persistent_vec_fn<unsigned>();
-        case 2: return persistent_vec_fn<unsigned short>();
-        default: return persistent_vec_fn<unsigned char>();
+        case 16: return persistent_vec_fn<uint4>(list);
+        case 8: return persistent_vec_fn<uint2>(list);
+        case 4: return persistent_vec_fn<unsigned>(list);
+        case 2: return persistent_vec_fn<unsigned short>(list);
+        default: return persistent_vec_fn<unsigned char>(list);
     }
 }
 template <typename V>
-const void* cluster_vec_fn() { return (const void*)cluster_vec_kernel<V>; }
-const void* pick_cluster_vec(int vbytes) {
+const void* flow_vec_fn() { return (const void*)flow_vec_kernel<V, kVecUnroll>; }
+const void* pick_flow_vec(int vbytes) {
     switch (vbytes) {
-        case 16: return cluster_vec_fn<uint4>();
-        case 8: return cluster_vec_fn<uint2>();
-        case 4: return cluster_vec_fn<unsigned>();
-        case 2: return cluster_vec_fn<unsigned short>();
-        default: return cluster_vec_fn<unsigned char>();
+        case 16: return flow_vec_fn<uint4>();
+        case 8: return flow_vec_fn<uint2>();
+        case 4: return flow_vec_fn<unsigned>();
+        case 2: return flow_vec_fn<unsigned short>();
+        default: return flow_vec_fn<unsigned char>();
     }
-}
-
-// Executor for SPARBIT_EXEC_AUTO, from the measured P = 256 and P = 1000 sweeps on B200: the
-// CUDA-graph chain of per-phase kernels (programmatic dependent launch between phases, grids sized
-// per phase) is the fastest or within noise at every block size - about 2.7 us per phase in the
-// latency regime against 3.7 us for the grid barrier of the persistent kernel, and 1-2 % ahead
-// at 64 KiB blocks.  The persistent kernel stays available (SPARBIT_EXEC_PERSISTENT) and is what
-// sparbit_allgather_noalloc runs.
-int auto_exec(const Schedule& s, bool coop, bool cluster_ok) {
-    (void)s;
-    (void)coop;
-    (void)cluster_ok;
-    return SPARBIT_EXEC_GRAPH;
-}
-
-struct Resolved {
-    int exec;    // SPARBIT_EXEC_* (never AUTO)
-    int copy;    // SPARBIT_COPY_VECTOR or _BULK
-    int vbytes;  // vector width for the vector engine
-};
-
-Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv) {
-    Resolved r;
-    r.vbytes = pick_vector_bytes(p, send, recv);
-    const uint64_t m = p->sched.m;
-    const bool bulk_possible = r.vbytes == 16;
-    int copy = p->copy_req;
-    // measured on B200 (P = 61 .. 509, m = 4 KiB .. 256 KiB): with about 32 KiB of loads in flight per
-    // SM both engines reach the copy peak; the bulk engine is 1-4 % ahead once blocks are >= 8 KiB
-    // and the collective is in the bandwidth regime (about 1 GB moved or more); below that its
-    // per-pass set-up (ring and mbarrier initialisation) and per-operation cost show and the
-    // vector engine wins
-    if (copy == SPARBIT_COPY_AUTO) {
-        const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
-        copy = (bulk_possible && m >= (8u << 10) && moved >= (unsigned __int128)1000000000) ? SPARBIT_COPY_BULK
-                                                                                            : SPARBIT_COPY_VECTOR;
-    }
-    if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
-    if (p->variable) copy = SPARBIT_COPY_VECTOR;  // variable block sizes run on the vector engine
-    r.copy = copy;
-    int exec = p->exec_req;
-    if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p->sched, p->coop != 0, p->cluster_ok != 0);
-    if (exec == SPARBIT_EXEC_PERSISTENT && !p->coop) exec = SPARBIT_EXEC_GRAPH;
-    if (exec == SPARBIT_EXEC_CLUSTER) {
-        if (!p->cluster_ok) exec = SPARBIT_EXEC_GRAPH;
-        r.copy = SPARBIT_COPY_VECTOR;  // the cluster executor has the vector engine only
-    }
-    r.exec = exec;
-    return r;
 }
 
 Geom make_geom(const sparbit_plan_s* p, const void* send, void* recv) {
@@ -392,6 +365,98 @@ ExecSeq make_seq(const sparbit_plan_s* p, int first, int last) {
     return q;
 }
 
+struct Resolved {
+    int exec;    // SPARBIT_EXEC_* (never AUTO)
+    int copy;    // SPARBIT_COPY_VECTOR or _BULK
+    int vbytes;  // vector width for the vector engine
+};
+
+bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, bool assume_coop = false) {
+    if (p->variable || !(p->coop || assume_coop)) return false;
+    if (first != -1 || last != p->sched.last_phase()) return false;
+    const ExecSeq seq = make_seq(p, first, last);
+    if (seq.count() < 1 || seq.count() > kFlowMaxPasses) return false;
+    for (int i = 0; i < seq.count(); i++) {
+        const PhaseDesc& d = seq.item(i);
+        const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
+        if (vpc < 32) return false;
+        const uint64_t spc = (vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll);
+        if (((uint64_t)p->sched.P * d.copies * spc) >> 31) return false;
+    }
+    return true;
+}
+
+// Executor for SPARBIT_EXEC_AUTO, from measurements on B200.
+//  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
+//    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
+//    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
+//    - are most of it), so there the host's cost decides: one graph launch (2.6 us) instead of one
+//    launch per pass (4 us each).  The graph chain it is.
+//  - From about 1 GB moved (150 us and more) the flow executor is 1-4 % ahead of the chain: the
+//    start-up and drain of every pass overlap with its neighbours (P = 1000, m = 1 KiB: 323 us
+//    against 334; P = 512, m = 4 KiB: 334 against 347; P = 128, m = 64 KiB: 333 against 338).
+//  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
+//    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
+//    which is the only one the flow executor has.
+int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
+    if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
+        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
+        return SPARBIT_EXEC_FLOW;
+    return SPARBIT_EXEC_GRAPH;
+}
+
+int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
+    const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
+    if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
+        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
+        flow_possible(p, vbytes, -1, p->sched.last_phase(), true))
+        return SPARBIT_EXEC_FLOW;
+    return SPARBIT_EXEC_GRAPH;
+}
+
+Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv, int first, int last) {
+    Resolved r;
+    r.vbytes = pick_vector_bytes(p, send, recv);
+    const uint64_t m = p->sched.m;
+    const bool bulk_possible = r.vbytes == 16;
+    int copy = p->copy_req;
+    // measured on B200 (P = 61 .. 509, m = 4 KiB .. 256 KiB): with about 32 KiB of loads in flight per
+    // SM both engines reach the copy peak; the bulk engine is 1-4 % ahead once blocks are >= 8 KiB
+    // and the collective is in the bandwidth regime (about 1 GB moved or more); below that its
+    // per-pass set-up (ring and mbarrier initialisation) and per-operation cost show and the
+    // vector engine wins
+    if (copy == SPARBIT_COPY_AUTO) {
+        const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
+        copy = (bulk_possible && m >= p->tune[SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES] &&
+                moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_BULK_MIN_MOVED_BYTES])
+                   ? SPARBIT_COPY_BULK
+                   : SPARBIT_COPY_VECTOR;
+    }
+    if (p->variable && p->copy_req == SPARBIT_COPY_AUTO) {
+        // the same rule on the average block size, with 2*(P-1)*T bytes moved
+        const uint64_t T = p->voff.back();
+        const unsigned __int128 moved = (unsigned __int128)2 * (p->sched.P - 1) * T;
+        copy = (bulk_possible && T / p->sched.P >= p->tune[SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES] &&
+                moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_BULK_MIN_MOVED_BYTES])
+                   ? SPARBIT_COPY_BULK
+                   : SPARBIT_COPY_VECTOR;
+    }
+    if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
+    r.copy = copy;
+    int exec = p->exec_req;
+    if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p, r.vbytes, first, last);
+    if (exec == SPARBIT_EXEC_PERSISTENT && !p->coop) exec = SPARBIT_EXEC_GRAPH;
+    if (exec == SPARBIT_EXEC_FLOW) {
+        // the flow executor runs whole collectives of fixed-size blocks on the vector engine, every
+        // copy at least one warp row long; anything else goes to the graph chain
+        if (flow_possible(p, r.vbytes, first, last)) r.copy = SPARBIT_COPY_VECTOR;
+        else exec = SPARBIT_EXEC_GRAPH;
+    }
+    r.exec = exec;
+    return r;
+}
+
 // launch geometry of one phase as its own kernel
 struct PhaseLaunch {
     const void* fn;
@@ -402,6 +467,16 @@ struct PhaseLaunch {
 int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d, PhaseLaunch& pl,
                       uint64_t var_tasks = 0) {
     const uint32_t P = p->sched.P;
+    if (p->variable && rs.copy == SPARBIT_COPY_BULK) {
+        uint64_t ctas = (var_tasks + p->bulk_warps - 1) / p->bulk_warps;
+        if (ctas > (uint64_t)p->sm_count) ctas = p->sm_count;
+        if (ctas < 1) ctas = 1;
+        pl.fn = (const void*)phase_bulk_list_kernel;
+        pl.grid = dim3((unsigned)ctas);
+        pl.block = dim3(p->bulk_warps * 32);
+        pl.smem = bulk_smem_bytes(p);
+        return SPARBIT_OK;
+    }
     if (p->variable) {
         const uint64_t wpb = kVecBlock / 32;
         uint64_t ctas = (var_tasks + wpb - 1) / wpb;
@@ -447,20 +522,22 @@ struct PhaseArgs {
     unsigned* status;
     unsigned long long timeout_ns;
     uint32_t extra_tx;
-    const unsigned long long* list;  // variable block sizes: this pass's task list
+    const VarTask* list;  // variable block sizes: this pass's task list
     unsigned long long count;
-    void* ptrs[6];
+    void* ptrs[8];
     void fill(bool bulk, bool variable = false) {
         ptrs[0] = &g;
         ptrs[1] = &d;
-        if (variable) {
-            ptrs[2] = &list;
-            ptrs[3] = &count;
-        } else if (bulk) {
+        if (bulk) {
             ptrs[2] = &stage_bytes;
             ptrs[3] = &status;
             ptrs[4] = &timeout_ns;
             ptrs[5] = &extra_tx;
+            ptrs[6] = &list;   // the list form of the bulk kernel only
+            ptrs[7] = &count;
+        } else if (variable) {
+            ptrs[2] = &list;
+            ptrs[3] = &count;
         }
     }
 };
@@ -473,6 +550,14 @@ struct PhaseArgs {
 int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const ExecSeq seq = make_seq(p, first, last);
     for (int i = 0; i < seq.count(); i++) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
         PhaseArgs a;
         a.g = g;
         a.d = seq.item(i);
@@ -491,17 +576,9 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         PhaseLaunch pl;
         int rc = plan_phase_launch(p, rs, a.d, pl, a.count);
         if (rc) return rc;
-        cudaLaunchConfig_t cfg;
-        memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = pl.grid;
         cfg.blockDim = pl.block;
         cfg.dynamicSmemBytes = pl.smem;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
         CU(cudaLaunchKernelExC(&cfg, pl.fn, a.ptrs));
         p->kernel_launches++;
     }
@@ -592,19 +669,25 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     dim3 block;
     size_t smem = 0;
     int per_sm = 0;
+    // tasks of pass i: listed (variable block sizes) or counted from the descriptor
+    auto list_tasks = [&](int i) {
+        const size_t ti = seq.table_index(i);
+        return (uint64_t)(p->vtask_hi[ti] - p->vtask_lo[ti]);
+    };
     if (rs.copy == SPARBIT_COPY_BULK) {
-        fn = (const void*)persistent_bulk_kernel;
+        fn = p->variable ? (const void*)persistent_bulk_kernel<true> : (const void*)persistent_bulk_kernel<false>;
         block = dim3(p->bulk_warps * 32);
         smem = bulk_smem_bytes(p);
         for (int i = 0; i < seq.count(); i++) {
-            uint64_t t = (bulk_tasks(seq.item(i), P, p->bulk_stage_bytes) + p->bulk_warps - 1) / p->bulk_warps;
+            const uint64_t tasks = p->variable ? list_tasks(i) : bulk_tasks(seq.item(i), P, p->bulk_stage_bytes);
+            uint64_t t = (tasks + p->bulk_warps - 1) / p->bulk_warps;
             if (t > need) need = t;
         }
     } else {
-        fn = pick_persistent_vec(rs.vbytes);
+        fn = pick_persistent_vec(rs.vbytes, p->variable);
         block = dim3(kVecBlock);
         for (int i = 0; i < seq.count(); i++) {
-            const uint64_t tasks = vec_tasks(seq.item(i), P, rs.vbytes);
+            const uint64_t tasks = p->variable ? list_tasks(i) : vec_tasks(seq.item(i), P, rs.vbytes);
             if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
             uint64_t t = (tasks + kVecBlock / 32 - 1) / (kVecBlock / 32);
             if (t > need) need = t;
@@ -640,8 +723,10 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
     uint32_t stage = p->bulk_stage_bytes;
-    void* args_vec[] = {&gg, &descs, &first_idx, &last_idx, &ctl};
-    void* args_bulk[] = {&gg, &descs, &first_idx, &last_idx, &stage, &ctl};
+    const VarTask* vtasks = p->d_vtasks;   // null unless the plan has variable block sizes
+    const VarRange* vranges = p->d_vranges;
+    void* args_vec[] = {&gg, &descs, &first_idx, &last_idx, &ctl, &vtasks, &vranges};
+    void* args_bulk[] = {&gg, &descs, &first_idx, &last_idx, &stage, &ctl, &vtasks, &vranges};
     CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), block,
                                    rs.copy == SPARBIT_COPY_BULK ? args_bulk : args_vec, smem, st));
     p->bar_base += (unsigned)(last_idx - first_idx) * ctl.expected;  // one barrier between consecutive passes
@@ -649,48 +734,87 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     return SPARBIT_OK;
 }
 
-int launch_cluster(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+// The whole collective as one cooperative kernel without grid barriers (flow_vec_kernel).
+int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
-    uint64_t need = 1;
-    for (int i = 0; i < seq.count(); i++) {
-        const uint64_t tasks = vec_tasks(seq.item(i), P, rs.vbytes);
-        if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
-        uint64_t t = (tasks + kClusterBlock / 32 - 1) / (kClusterBlock / 32);
-        if (t > need) need = t;
+    const int n = seq.count();
+    if (!p->d_flow_cnt) {
+        CU(cudaMalloc((void**)&p->d_flow_cnt, (size_t)P * kFlowMaxPasses * sizeof(unsigned)));
+        p->flow_epoch = 0;
+        p->flow_vbytes = 0;
     }
-    const void* fn = pick_cluster_vec(rs.vbytes);
-    // 16 CTAs (the non-portable maximum) when the device can place such a cluster, else 8
-    unsigned ctas = 16;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
-        (void)cudaGetLastError();
-        ctas = 8;
+    if (p->flow_vbytes != rs.vbytes || p->flow_epoch == 0) {
+        // counters count units, and a unit's size follows the vector width: start over
+        CU(cudaMemsetAsync(p->d_flow_cnt, 0, (size_t)P * kFlowMaxPasses * sizeof(unsigned), st));
+        p->flow_epoch = 0;
+        p->flow_vbytes = rs.vbytes;
     }
-    for (;;) {
-        while (ctas > 1 && ctas / 2 >= need) ctas /= 2;
-        memset(&cfg, 0, sizeof cfg);
-        cfg.gridDim = dim3(ctas);
-        cfg.blockDim = dim3(kClusterBlock);
-        cfg.dynamicSmemBytes = 0;
-        cfg.stream = st;
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = ctas;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int fit = 0;
-        if (ctas <= 8 || (cudaOccupancyMaxActiveClusters(&fit, fn, &cfg) == cudaSuccess && fit >= 1)) break;
-        (void)cudaGetLastError();
-        ctas = 8;
-        need = ~0ull;  // keep 8
+    p->flow_epoch++;
+    FlowArgs fa;
+    memset(&fa, 0, sizeof fa);
+    fa.n = (uint32_t)n;
+    fa.cnt = p->d_flow_cnt;
+    fa.status = p->d_ctl + 1;
+    fa.timeout_ns = p->timeout_ns;
+    const void* fn = pick_flow_vec(rs.vbytes);
+    int per_sm = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kVecBlock, 0));
+    if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "flow kernel does not fit on an SM");
+    if (per_sm > 2) per_sm = 2;
+    const uint64_t max_warps = (uint64_t)per_sm * p->sm_count * (kVecBlock / 32);
+    uint64_t most_units = 1;
+    uint32_t rot = 0;
+    for (int i = 0; i < n; i++) {
+        const PhaseDesc& d = seq.item(i);
+        FlowPass& fp = fa.pass[i];
+        const uint64_t vpc = d.copy_bytes / (uint64_t)rs.vbytes;
+        fp.spc = (uint32_t)((vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll));
+        const uint64_t spans = (uint64_t)d.copies * fp.spc;  // per source rank
+        // Unit size: a small pass is cut into single spans, so that as many warps as possible share
+        // it and a hop (copy, release, the next pass's poll) stays short; a pass that keeps every
+        // warp busy takes units of up to FLOW_MAX_UNIT_SPANS spans, which spreads
+        // the poll and the release over more bytes.
+        uint64_t us = (uint64_t)P * spans / (max_warps * p->tune[SPARBIT_TUNE_FLOW_UNITS_PER_WARP]);
+        if (us < 1) us = 1;
+        if (us > p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS]) us = p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS];
+        if (us > spans) us = spans;
+        fp.us = (uint32_t)us;
+        fp.upr = (uint32_t)((spans + fp.us - 1) / fp.us);
+        fp.rot = rot;
+        // units that write into one rank's buffer in this pass: those of its one sender, and in the
+        // fused first pass its own as well
+        const uint32_t per_rank = fp.upr * (d.dup_self ? 2u : 1u);
+        fp.target = p->flow_epoch * per_rank + (p->extra_arrivals ? 1u : 0u);  // test hook: never reached
+        fp.dep_mask = 0;
+        for (int k = 0; k < i; k++)
+            if (seq.item(k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
+        if ((uint64_t)P * fp.upr > most_units) most_units = (uint64_t)P * fp.upr;
+        fp.eager = (uint64_t)P * fp.upr <= max_warps ? 1u : 0u;
+        // the next pass starts its enumeration where this pass's first receivers are
+        if (d.peer_xor == 0 && d.peer_pre == 0) rot = (rot + d.peer_add) % P;
     }
-    int first_idx = (int)seq.table_index(0), last_idx = (int)seq.table_index(seq.count() - 1);
+    uint64_t grid = (uint64_t)per_sm * p->sm_count;
+    const uint64_t need = (most_units + kVecBlock / 32 - 1) / (kVecBlock / 32);
+    if (grid > need) grid = need;
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
-    void* args[] = {&gg, &descs, &first_idx, &last_idx};
+    int first_idx = (int)seq.table_index(0);
+    void* args[] = {&gg, &descs, &first_idx, &fa};
+    // cooperative (all CTAs resident: the waits inside depend on it) and, like the per-pass kernels,
+    // launched ahead behind its predecessor in the stream
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kVecBlock);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     CU(cudaLaunchKernelExC(&cfg, fn, args));
     p->kernel_launches++;
     return SPARBIT_OK;
@@ -711,17 +835,18 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
         return SPARBIT_ERR_ALIAS;
     int rc = ensure_device(p);
     if (rc) return rc;
-    const Resolved rs = resolve(p, send, recv);
+    const Resolved rs = resolve(p, send, recv, first, last);
     const Geom g = make_geom(p, send, recv);
     cudaStream_t st = (cudaStream_t)stream;
     switch (rs.exec) {
         case SPARBIT_EXEC_PERSISTENT: rc = launch_persistent(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_GRAPH: rc = launch_graph(p, rs, g, first, last, st); break;
-        case SPARBIT_EXEC_CLUSTER: rc = launch_cluster(p, rs, g, first, last, st); break;
+        case SPARBIT_EXEC_FLOW: rc = launch_flow(p, rs, g, first, last, st); break;
         default: rc = launch_stream(p, rs, g, first, last, st); break;
     }
     if (rc == SPARBIT_OK) {
         p->copy_last = rs.copy;
+        p->exec_last = rs.exec;
         p->last_stream = st;
         p->launched = true;
     }
@@ -736,7 +861,7 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
     if (!out) return SPARBIT_ERR_ARG;
     *out = nullptr;
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
-    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_CLUSTER) return SPARBIT_ERR_ARG;
+    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_FLOW) return SPARBIT_ERR_ARG;
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
     int rc;
@@ -762,10 +887,8 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     if (P > 8192) return SPARBIT_ERR_LIMIT;  // the task lists are built copy by copy: P*(P-1) entries at least
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
     if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // rotated workspace: fixed sizes only
-    if (exec != SPARBIT_EXEC_AUTO && exec != SPARBIT_EXEC_GRAPH && exec != SPARBIT_EXEC_STREAM) {
-        if (exec == SPARBIT_EXEC_PERSISTENT || exec == SPARBIT_EXEC_CLUSTER) return SPARBIT_ERR_UNSUPPORTED;
-        return SPARBIT_ERR_ARG;
-    }
+    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_FLOW) return SPARBIT_ERR_ARG;
+    if (exec == SPARBIT_EXEC_FLOW) return SPARBIT_ERR_UNSUPPORTED;  // its units assume equal blocks
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
     int rc;
@@ -799,16 +922,29 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
             if (p->sched.has_fused_first) set_max(p->sched.fused_first);
             p->sched.m = 0;
             // task lists, indexed like the device descriptor table: every phase, the fused first
-            // pass, and (as in that table) phases 1.. once more after it
+            // pass, and (as in that table) phases 1.. once more after it.  A task is a segment of at
+            // most kVarSegmentBytes of one copy, with its source and destination byte offsets.
+            const uint64_t T = p->voff.back();
+            if (((unsigned __int128)T * (unsigned)P) >> 48) rc = SPARBIT_ERR_OVERFLOW;  // offsets are 48-bit fields
             auto add_list = [&](const PhaseDesc& d) {
                 p->vtask_lo.push_back(p->vtasks.size());
                 for (uint32_t r = 0; r < p->sched.P; r++)
                     for (uint32_t j = 0; j < d.copies; j++) {
                         const CopyLoc c = locate_copy(d, p->sched.P, r, j);
                         const uint64_t b = p->voff[c.dst_slot + d.run] - p->voff[c.dst_slot];
-                        const uint64_t q = (uint64_t)r * d.copies + j;
-                        for (uint64_t sg = 0; sg * kVarSegmentBytes < b; sg++)
-                            p->vtasks.push_back((unsigned long long)((q << 32) | sg));
+                        // send blocks sit at voff[rank]; every receive buffer holds all blocks
+                        const uint64_t soff = d.src_space == SPACE_SEND
+                                                  ? p->voff[c.src_rank]
+                                                  : (uint64_t)c.src_rank * T + p->voff[c.src_slot];
+                        const uint64_t doff = (uint64_t)c.dst_rank * T + p->voff[c.dst_slot];
+                        const int delta = (int)r - (int)c.dst_rank;  // |delta| < P <= 8192
+                        for (uint64_t at = 0; at < b; at += kVarSegmentBytes) {
+                            const uint64_t n = b - at < kVarSegmentBytes ? b - at : kVarSegmentBytes;
+                            VarTask t;
+                            t.a = (soff + at) | ((n - 1) << 48);
+                            t.b = (doff + at) | ((unsigned long long)(unsigned short)(short)delta << 48);
+                            p->vtasks.push_back(t);
+                        }
                     }
                 p->vtask_hi.push_back(p->vtasks.size());
             };
@@ -820,7 +956,7 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
                     p->vtask_hi.push_back(p->vtask_hi[i]);
                 }
             }
-            if (p->vtasks.size() >> 28) rc = SPARBIT_ERR_OVERFLOW;  // 2 GiB of task entries: refuse
+            if (p->vtasks.size() >> 27) rc = SPARBIT_ERR_OVERFLOW;  // 2 GiB of task entries: refuse
         }
     } catch (const std::bad_alloc&) {
         rc = SPARBIT_ERR_NOMEM;
@@ -830,10 +966,11 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
         return rc;
     }
     p->exec_req = exec;
-    if (exec == SPARBIT_EXEC_AUTO) {  // variable-size plans take graph or stream only
+    if (exec == SPARBIT_EXEC_AUTO) {  // variable-size plans have no flow executor
         const int e = env_exec(SPARBIT_EXEC_AUTO);
-        if (e == SPARBIT_EXEC_GRAPH || e == SPARBIT_EXEC_STREAM) p->exec_req = e;
+        if (e != SPARBIT_EXEC_FLOW) p->exec_req = e;
     }
+    p->copy_req = env_copy(SPARBIT_COPY_AUTO);
     *out = p;
     return SPARBIT_OK;
 }
@@ -854,8 +991,10 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
         cudaFree(p->d_descs);
         cudaFree(p->d_voff);
         cudaFree(p->d_vtasks);
+        cudaFree(p->d_vranges);
         cudaFree(p->d_trace);
         cudaFree(p->d_ctl);
+        cudaFree(p->d_flow_cnt);
         cudaFree(p->stage_send);
         cudaFree(p->stage_recv);
         cudaFree(p->stage_work);
@@ -988,11 +1127,34 @@ int sparbit_plan_set_copy_path(sparbit_plan_t* p, int copy_path) {
     return SPARBIT_OK;
 }
 
+int sparbit_plan_set_tunable(sparbit_plan_t* p, int key, uint64_t value) {
+    if (!p || key < 0 || key >= SPARBIT_TUNE_COUNT_) return SPARBIT_ERR_ARG;
+    if (p->tune[key] == value) return SPARBIT_OK;
+    if (p->launched) {
+        // cached graphs were cut into launches with the old value
+        if (cudaStreamSynchronize(p->last_stream) != cudaSuccess) return SPARBIT_ERR_CUDA;
+        drop_graph(p);
+    }
+    p->tune[key] = value;
+    return SPARBIT_OK;
+}
+
+int sparbit_plan_get_tunable(const sparbit_plan_t* p, int key, uint64_t* value) {
+    if (!p || !value || key < 0 || key >= SPARBIT_TUNE_COUNT_) return SPARBIT_ERR_ARG;
+    *value = p->tune[key];
+    return SPARBIT_OK;
+}
+
 int sparbit_plan_exec_mode(const sparbit_plan_t* p) {
     if (!p) return -1;
+    if (p->exec_last != SPARBIT_EXEC_AUTO) return p->exec_last;  // what the last launch ran on
     if (p->exec_req != SPARBIT_EXEC_AUTO) return p->exec_req;
-    // before the first launch the device is not known yet: assume a B200 (both features present)
-    return auto_exec(p->sched, p->dev_ready ? p->coop != 0 : true, p->dev_ready ? p->cluster_ok != 0 : true);
+    // before the first launch neither the buffers nor the device are known: assume 16-byte aligned
+    // buffers on a B200
+    uintptr_t bits = p->variable ? p->voff_bits : (uintptr_t)p->sched.m;
+    int v = 16;
+    while (v > 1 && (bits & (uintptr_t)(v - 1))) v >>= 1;
+    return auto_exec_before_launch(p, v);
 }
 
 int sparbit_plan_copy_path(const sparbit_plan_t* p) { return p ? p->copy_last : -1; }
@@ -1016,6 +1178,7 @@ int sparbit_plan_status(sparbit_plan_t* p, int* device_status) {
         // a failed launch leaves the arrival counter in an unknown state: start over
         CU(cudaMemset(p->d_ctl, 0, sizeof ctl));
         p->bar_base = 0;
+        p->flow_epoch = 0;  // the next flow launch clears its counters
         return SPARBIT_ERR_TIMEOUT;
     }
     return SPARBIT_OK;

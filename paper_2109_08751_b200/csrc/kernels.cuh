@@ -14,7 +14,8 @@
 //
 // and four ways to sequence passes: one kernel per pass, chained by programmatic dependent launch
 // (plain stream launches or a CUDA graph); one persistent cooperative kernel with a bounded-wait
-// grid barrier after every pass; or one thread-block cluster with the hardware cluster barrier.
+// grid barrier after every pass; or one cooperative kernel in which every rank's Waitall is a set
+// of per-rank counters instead of a barrier (flow).
 //
 // Loads never use the non-coherent path or L1: data written in one pass is read by other SMs in
 // the next one, possibly inside the same launch.
@@ -154,10 +155,9 @@ __device__ __forceinline__ void st_cg<unsigned char>(unsigned char* p, unsigned 
 
 // One phase on the vector engine.  warp_id / n_warps enumerate all warps taking part.
 // Requires P * copies * ceil(vectors_per_copy / (32*U)) < 2^32 (checked on the host).
-template <typename V>
+template <typename V, int U = kVecUnroll>
 __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uint32_t warp_id, uint32_t n_warps,
                                           uint32_t lane) {
-    constexpr int U = kVecUnroll;
     const uint32_t P = g.P;
     const uint64_t vpc64 = d.copy_bytes / sizeof(V);  // vectors per copy
     const uint32_t n_copies = P * d.copies;            // copies in the phase (< 2^32, host-checked)
@@ -236,43 +236,48 @@ __device__ __forceinline__ void vec_phase(const Geom& g, const PhaseDesc& d, uin
     }
 }
 
-// One phase with blocks of DIFFERENT sizes (allgatherv).  The host lists the phase's work as
-// tasks of at most kVarSegmentBytes: entry = copy index (r * copies + j) in the high half, segment
-// number inside that copy in the low half; empty blocks have no entry.  Every task is then about
-// the same size, so handing task t to warp t mod n_warps balances the warps whatever the mix of
-// block sizes is.  A copy's size and position come from g.voff (prefix sums of the byte counts):
-// block b is voff[b+1]-voff[b] bytes, at voff[b] in the send buffer and in every receive buffer.
+// One phase with blocks of DIFFERENT sizes (allgatherv).  The host lists the phase's work as tasks
+// of at most kVarSegmentBytes, each a self-contained record: where the bytes are read (offset
+// inside the phase's source space), where they go (offset inside its destination space), how
+// many, and - for the fused first pass - how many ranks away the second destination is.  Empty
+// blocks have no entry.  Every task is about the same size, so handing task t to warp
+// t mod n_warps balances the warps whatever the mix of block sizes is, and a task needs no
+// index arithmetic and no size table on the device.
 constexpr uint32_t kVarSegmentBytes = 4096;
 
+struct VarTask {
+    unsigned long long a;  // bits 0..47 source byte offset, bits 48..63 byte count - 1
+    unsigned long long b;  // bits 0..47 destination byte offset, bits 48..63 (signed) rank distance
+                           // of the second destination in a dup_self phase
+};
+static_assert(sizeof(VarTask) == 16, "a task is read with one 16-byte load");
+constexpr unsigned long long kVarOffsetMask = (1ull << 48) - 1;
+
+__device__ __forceinline__ VarTask ld_task(const VarTask* p) {
+    const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2*>(p));
+    VarTask t;
+    t.a = v.x;
+    t.b = v.y;
+    return t;
+}
+
 template <typename V>
-__device__ __forceinline__ void vec_list_phase(const Geom& g, const PhaseDesc& d,
-                                               const unsigned long long* __restrict__ list, uint64_t count,
-                                               uint32_t warp_id, uint32_t n_warps, uint32_t lane) {
+__device__ __forceinline__ void vec_list_phase(const Geom& g, const PhaseDesc& d, const VarTask* __restrict__ list,
+                                               uint64_t count, uint32_t warp_id, uint32_t n_warps, uint32_t lane) {
     constexpr int U = kVecUnroll;
     constexpr uint32_t span = 32u * U;  // vectors per warp iteration
-    const uint32_t P = g.P;
     const char* sbase = space_base(g, d.src_space);
     char* dbase = space_base(g, d.dst_space);
-    const uint64_t spitch = space_pitch(g, d.src_space);
-    const uint64_t dpitch = space_pitch(g, d.dst_space);
+    const long long dpitch = (long long)space_pitch(g, d.dst_space);
+    if (warp_id >= count) return;
+    VarTask next = ld_task(list + warp_id);
     for (uint64_t t = warp_id; t < count; t += n_warps) {
-        const unsigned long long e = __ldg(list + t);
-        const uint32_t q = (uint32_t)(e >> 32);
-        const uint32_t sg = (uint32_t)e;
-        const uint32_t r = q / d.copies;
-        const uint32_t j = q - r * d.copies;
-        const CopyLoc c = locate_copy(d, P, r, j);
-        const uint64_t lo = __ldg(g.voff + c.dst_slot);
-        const uint64_t hi = __ldg(g.voff + c.dst_slot + d.run);
-        const uint64_t soff = d.src_space == SPACE_SEND ? __ldg(g.voff + c.src_rank)
-                                                        : (uint64_t)c.src_rank * spitch + __ldg(g.voff + c.src_slot);
-        const uint64_t begin = (uint64_t)sg * kVarSegmentBytes;  // this task's bytes of the copy
-        uint64_t end = begin + kVarSegmentBytes;
-        if (end > hi - lo) end = hi - lo;
-        const V* src = reinterpret_cast<const V*>(sbase + soff + begin);
-        V* dst = reinterpret_cast<V*>(dbase + (uint64_t)c.dst_rank * dpitch + lo + begin);
-        V* dst2 = reinterpret_cast<V*>(dbase + (uint64_t)r * dpitch + lo + begin);
-        const uint32_t vectors = (uint32_t)((end - begin) / sizeof(V));
+        const VarTask e = next;
+        if (t + n_warps < count) next = ld_task(list + t + n_warps);  // in flight while this task is copied
+        const V* src = reinterpret_cast<const V*>(sbase + (e.a & kVarOffsetMask));
+        V* dst = reinterpret_cast<V*>(dbase + (e.b & kVarOffsetMask));
+        V* dst2 = reinterpret_cast<V*>(reinterpret_cast<char*>(dst) + (long long)(short)(e.b >> 48) * dpitch);
+        const uint32_t vectors = ((uint32_t)(e.a >> 48) + 1u) / (uint32_t)sizeof(V);
 #pragma unroll 1
         for (uint32_t first = 0; first < vectors; first += span) {
             V regs[U];
@@ -300,8 +305,11 @@ struct BulkPipe {
     uint32_t ring;      // shared address of this warp's first stage
     uint32_t bars;      // shared address of this warp's first mbarrier (kBulkStages of them)
     uint32_t meta;      // shared address of per-stage {dst pointer, bytes, second-dst delta, pad} records (32 B: v2.u64 accesses need 16-byte alignment)
+    uint32_t taskq;     // shared address of this ring's queue of prefetched task-list entries (kTaskQueue x 16 B)
     uint32_t it;        // stages used so far by this ring (carried across phases)
 };
+constexpr int kTaskQueue = 8;   // entries of the queue
+constexpr int kTaskAhead = 6;   // list entries in flight ahead of the task being issued
 
 // Bounded wait on one mbarrier phase.  Returns false (after setting the status word) on time-out
 // or when another CTA already reported a failure.
@@ -325,17 +333,37 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 // One phase on the bulk engine, driven by ONE thread (the elected lane of a warp).  pipe_id /
 // n_pipes enumerate all rings taking part.  All addresses and sizes are multiples of 16 bytes
 // (host-checked).  Returns false if a wait gave up.
+//
+// With a task list (blocks of different sizes) a task is one list entry (at most one stage, host-
+// checked) instead of a chunk of a copy located through the descriptor; the entry of the task
+// after the one being issued is fetched one step ahead.
+template <bool kList = false>
 __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, uint32_t stage_bytes, uint32_t pipe_id,
                                            uint32_t n_pipes, BulkPipe& pp, unsigned* status,
-                                           unsigned long long timeout_ns, uint32_t extra_tx = 0) {
+                                           unsigned long long timeout_ns, uint32_t extra_tx = 0,
+                                           const VarTask* __restrict__ list = nullptr, uint64_t count = 0) {
     constexpr int S = kBulkStages;
     constexpr int L = kBulkLoadsAhead;
     const uint32_t P = g.P;
-    const uint64_t cpc = (d.copy_bytes + stage_bytes - 1) / stage_bytes;  // chunks per copy
-    const uint64_t tasks = (uint64_t)P * d.copies * cpc;
+    const uint64_t cpc = kList ? 1 : (d.copy_bytes + stage_bytes - 1) / stage_bytes;  // chunks per copy
+    const uint64_t tasks = kList ? count : (uint64_t)P * d.copies * cpc;
     if (pipe_id >= tasks) return true;
     // equal chunks (rounded up to 128 B) instead of full stages plus a short tail
-    const uint32_t chunk = (uint32_t)((((d.copy_bytes + cpc - 1) / cpc) + 127u) & ~127ull);
+    const uint32_t chunk = kList ? 0u : (uint32_t)((((d.copy_bytes + cpc - 1) / cpc) + 127u) & ~127ull);
+    // A list entry costs a memory round trip and the ring issues a task every third of one, so the
+    // entries of the next kTaskAhead tasks are kept in flight, copied asynchronously into a small
+    // shared-memory queue (one async group per entry, empty past the end of the list).
+    auto fetch_entry = [&](uint64_t k) {
+        if (k < tasks) {
+            const uint64_t n = (k - pipe_id) / n_pipes;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(pp.taskq + (uint32_t)(n % kTaskQueue) * 16u),
+                         "l"(list + k)
+                         : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (kList)
+        for (int k = 0; k < kTaskAhead; k++) fetch_entry(pipe_id + (uint64_t)k * n_pipes);
     fence_proxy_async_all();  // what other CTAs wrote before the barrier -> visible to bulk loads
     const uint64_t mine = (tasks - pipe_id + n_pipes - 1) / n_pipes;      // tasks of this ring
     const bool small = (tasks >> 32) == 0;
@@ -353,29 +381,45 @@ __device__ __forceinline__ bool bulk_phase(const Geom& g, const PhaseDesc& d, ui
             // memory: stores are committed one group per task, L tasks behind the loads
             bulk_wait_read<S - L - 1>();
             const uint64_t w = pipe_id + i * n_pipes;
-            uint64_t q, ch;
-            uint32_t r, j;
-            if (small) {  // everything fits 32 bits: four cheap divisions instead of four long ones
-                const uint32_t w32 = (uint32_t)w, cpc32 = (uint32_t)cpc;
-                const uint32_t q32 = w32 / cpc32;
-                ch = w32 - q32 * cpc32;
-                r = q32 / d.copies;
-                j = q32 - r * d.copies;
-                q = q32;
+            const char* src;
+            char* dst;
+            uint32_t bytes;
+            long long delta2;  // second destination of a dup_self phase, as a byte delta from the first
+            if constexpr (kList) {
+                fetch_entry(w + (uint64_t)kTaskAhead * n_pipes);
+                asm volatile("cp.async.wait_group %0;" ::"n"(kTaskAhead) : "memory");  // entry i has landed
+                VarTask e;
+                asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(e.a), "=l"(e.b)
+                             : "r"(pp.taskq + (uint32_t)(i % kTaskQueue) * 16u)
+                             : "memory");
+                src = sbase + (e.a & kVarOffsetMask);
+                dst = dbase + (e.b & kVarOffsetMask);
+                bytes = (uint32_t)(e.a >> 48) + 1u;
+                delta2 = (long long)(short)(e.b >> 48) * (long long)dpitch;
             } else {
-                q = w / cpc;
-                ch = w - q * cpc;
-                r = (uint32_t)(q / d.copies);
-                j = (uint32_t)(q - (uint64_t)r * d.copies);
+                uint64_t q, ch;
+                uint32_t r, j;
+                if (small) {  // everything fits 32 bits: four cheap divisions instead of four long ones
+                    const uint32_t w32 = (uint32_t)w, cpc32 = (uint32_t)cpc;
+                    const uint32_t q32 = w32 / cpc32;
+                    ch = w32 - q32 * cpc32;
+                    r = q32 / d.copies;
+                    j = q32 - r * d.copies;
+                    q = q32;
+                } else {
+                    q = w / cpc;
+                    ch = w - q * cpc;
+                    r = (uint32_t)(q / d.copies);
+                    j = (uint32_t)(q - (uint64_t)r * d.copies);
+                }
+                const CopyLoc c = locate_copy(d, P, r, j);
+                const uint64_t off = ch * chunk;
+                const uint64_t left = d.copy_bytes - off;
+                bytes = left < chunk ? (uint32_t)left : chunk;
+                src = sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m) + off;
+                dst = dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m) + off;
+                delta2 = ((long long)r - (long long)c.dst_rank) * (long long)dpitch;
             }
-            const CopyLoc c = locate_copy(d, P, r, j);
-            const uint64_t off = ch * chunk;
-            const uint64_t left = d.copy_bytes - off;
-            const uint32_t bytes = left < chunk ? (uint32_t)left : chunk;
-            const char* src = sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m) + off;
-            char* dst = dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m) + off;
-            // second destination of a dup_self phase, as a byte delta from the first
-            const long long delta2 = ((long long)r - (long long)c.dst_rank) * (long long)dpitch;
             const uint32_t bar = pp.bars + st * 8u;
             // remember where this stage goes
             asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(pp.meta + st * 32u), "l"(dst),
@@ -473,7 +517,7 @@ __global__ void __launch_bounds__(512, 2) phase_vec_kernel(Geom g, PhaseDesc d) 
 
 // one phase, vector engine, variable block sizes (task list built by the host)
 template <typename V>
-__global__ void __launch_bounds__(512, 2) phase_vec_list_kernel(Geom g, PhaseDesc d, const unsigned long long* list,
+__global__ void __launch_bounds__(512, 2) phase_vec_list_kernel(Geom g, PhaseDesc d, const VarTask* list,
                                                                 unsigned long long count) {
     chain_wait();
     const uint32_t wpb = blockDim.x >> 5;
@@ -490,6 +534,7 @@ __device__ __forceinline__ BulkPipe make_pipe(unsigned char* smem, uint32_t stag
     pp.ring = base + warp * kBulkStages * stage_bytes;
     pp.bars = base + rings + warp * kBulkStages * 8u;
     pp.meta = base + rings + warps * kBulkStages * 8u + warp * kBulkStages * 32u;
+    pp.taskq = base + rings + warps * kBulkStages * 40u + warp * kTaskQueue * 16u;
     pp.it = 0;
     return pp;
 }
@@ -517,6 +562,30 @@ __global__ void __launch_bounds__(256) phase_bulk_kernel(Geom g, PhaseDesc d, ui
     }
 }
 
+// one phase, bulk engine, variable block sizes (same task list as the vector form)
+__global__ void __launch_bounds__(256) phase_bulk_list_kernel(Geom g, PhaseDesc d, uint32_t stage_bytes,
+                                                              unsigned* status, unsigned long long timeout_ns,
+                                                              uint32_t extra_tx, const VarTask* list,
+                                                              unsigned long long count) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    chain_trigger();
+    const uint32_t warps = blockDim.x >> 5;
+    const uint32_t warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31u) == 0) {
+        BulkPipe pp = make_pipe(smem, stage_bytes, warps, warp);
+        init_pipe(pp);
+        chain_wait();
+        bulk_phase<true>(g, d, stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, status, timeout_ns,
+                         extra_tx, list, count);
+    }
+}
+
+// Where the task list of each entry of the device descriptor table starts, and how long it is
+// (variable block sizes; the persistent kernels walk the table).
+struct VarRange {
+    unsigned long long lo, count;
+};
+
 // Descriptors of a multi-phase kernel live in shared memory, double-buffered: the next phase's
 // descriptor is fetched while the current phase runs, so no phase starts with a global load on
 // its critical path, and the copy loops need no registers to hold it.
@@ -527,9 +596,11 @@ __device__ __forceinline__ void fetch_desc(PhaseDesc* dst, const PhaseDesc* __re
 }
 
 // phases first..last (indices into descs), vector engine, grid barrier between phases
-template <typename V>
+template <typename V, bool kList = false>
 __global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs,
-                                                                int first, int last, BarrierCtl ctl) {
+                                                                int first, int last, BarrierCtl ctl,
+                                                                const VarTask* __restrict__ tasks = nullptr,
+                                                                const VarRange* __restrict__ ranges = nullptr) {
     __shared__ int flag;
     __shared__ PhaseDesc sd[2];
     if (ld_relaxed_gpu(ctl.status) != DEV_OK) return;  // an earlier failure was not cleared yet
@@ -544,15 +615,23 @@ __global__ void __launch_bounds__(512, SPB_PERSIST_MIN_CTAS) persistent_vec_kern
     for (int ph = first; ph <= last; ph++) {
         const int cur = (ph - first) & 1;
         if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
-        vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
+        if (kList) {
+            const VarRange vr = ranges[ph];
+            vec_list_phase<V>(g, sd[cur], tasks + vr.lo, vr.count, warp_id, n_warps, threadIdx.x & 31u);
+        } else {
+            vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
+        }
         if (ph != last && !grid_barrier<false>(ctl, epoch, &flag)) return;
         if (tracer) ctl.trace[ph - first + 1] = globaltimer_ns();
     }
 }
 
 // phases first..last, bulk engine, grid barrier between phases
+template <bool kList = false>
 __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
-                                                              int last, uint32_t stage_bytes, BarrierCtl ctl) {
+                                                              int last, uint32_t stage_bytes, BarrierCtl ctl,
+                                                              const VarTask* __restrict__ tasks = nullptr,
+                                                              const VarRange* __restrict__ ranges = nullptr) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int flag;
     __shared__ PhaseDesc sd[2];
@@ -570,36 +649,189 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
     for (int ph = first; ph <= last; ph++) {
         const int cur = (ph - first) & 1;
         if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
-        if (driver)
-            bulk_phase(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
-                       ctl.timeout_ns, ctl.mbar_extra_tx);
+        if (driver) {
+            if (kList) {
+                const VarRange vr = ranges[ph];
+                bulk_phase<true>(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp, ctl.status,
+                                 ctl.timeout_ns, ctl.mbar_extra_tx, tasks + vr.lo, vr.count);
+            } else {
+                bulk_phase<false>(g, sd[cur], stage_bytes, blockIdx.x * warps + warp, gridDim.x * warps, pp,
+                                  ctl.status, ctl.timeout_ns, ctl.mbar_extra_tx);
+            }
+        }
         if (ph != last && !grid_barrier<true>(ctl, epoch, &flag)) return;
         if (tracer) ctl.trace[ph - first + 1] = globaltimer_ns();
     }
 }
 
-// phases first..last, vector engine, ONE thread-block cluster as the whole grid: the hardware
-// cluster barrier (arrive.release / wait.acquire) separates phases.  For collectives so small
-// that a grid-wide barrier or a kernel boundary per phase would dominate.
-template <typename V>
-__global__ void __launch_bounds__(1024) cluster_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first,
-                                                           int last) {
-    __shared__ PhaseDesc sd[2];
-    const uint32_t wpb = blockDim.x >> 5;
-    const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
-    const uint32_t n_warps = gridDim.x * wpb;
-    fetch_desc(&sd[0], &descs[first]);
+// ------------------------------------------------------------------------------------------------
+// flow executor: the whole collective in one cooperative kernel WITHOUT grid-wide barriers
+// ------------------------------------------------------------------------------------------------
+// Algorithm 1 ends every step with MPI_Waitall, but what a rank sends in step i+1 depends only on
+// what THAT rank has received in the steps before.  So the Waitall is kept per rank instead of per
+// grid: a (rank, pass) counter counts the finished work units that wrote into that rank's buffer
+// in that pass, and a unit that reads rank r in pass i first waits until the counters of rank r
+// for every earlier pass that writes the space it reads have reached their final value.  Blocks
+// still travel exactly as the schedule says (each forwarded block is read from the sending
+// rank's receive buffer after that rank has received it); only the idle time at the pass
+// boundaries goes away, because warps that are done with pass i start on pass i+1 while others
+// are still busy.
+//
+// A unit is up to `us` consecutive warp spans (32*U vectors each) of the copies ONE rank sends
+// in one pass: one source rank, one destination rank, hence one dependency and one counter.
+// Units are numbered pass by pass and dealt to the warps round robin, every warp taking its units
+// in increasing order; the unit with the smallest number that is not finished never waits for a
+// later one, so the scheme cannot deadlock while all CTAs are resident (cooperative launch).
+// Within a pass the ranks are enumerated from `rot` on, chosen by the host so that a unit's
+// producers sit at about the same relative position of the pass before.
+//
+// Counters are never reset between collectives: the host passes, per pass, the value they reach
+// at the end of THIS launch (launch number times units per rank).
+constexpr int kFlowMaxPasses = 32;  // a rank's counters fill one 128-byte line
+
+struct FlowPass {
+    uint32_t upr;       // units per source rank
+    uint32_t us;        // spans per unit (the last unit of a rank may hold fewer)
+    uint32_t spc;       // spans per copy
+    uint32_t rot;       // position x of the pass handles source rank (x + rot) mod P
+    uint32_t target;    // counter value of a (rank, this pass) when all its units of this launch are done
+    uint32_t dep_mask;  // bit k: pass k (< this one) writes the space this pass reads
+    uint32_t eager;     // 1: no warp has a second unit in this pass - signal a unit as soon as it is stored
+    uint32_t pad_;
+};
+struct FlowArgs {
+    FlowPass pass[kFlowMaxPasses];
+    uint32_t n;
+    uint32_t pad_;
+    unsigned* cnt;      // [P][kFlowMaxPasses]
+    unsigned* status;
+    unsigned long long timeout_ns;
+};
+
+__device__ __forceinline__ void red_relaxed_gpu_add(unsigned* p, unsigned v) {
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+
+template <typename V, int U>
+__global__ void __launch_bounds__(512, 2) flow_vec_kernel(Geom g, const PhaseDesc* __restrict__ descs, int first_idx,
+                                                          const __grid_constant__ FlowArgs fa) {
+    __shared__ PhaseDesc sd[kFlowMaxPasses];
+    __shared__ uint32_t s_target[kFlowMaxPasses];
+    for (uint32_t k = threadIdx.x; k < fa.n * 16u; k += blockDim.x)
+        reinterpret_cast<uint32_t*>(sd)[k] = reinterpret_cast<const uint32_t*>(descs + first_idx)[k];
+    if (threadIdx.x < kFlowMaxPasses) s_target[threadIdx.x] = threadIdx.x < fa.n ? fa.pass[threadIdx.x].target : 0u;
     __syncthreads();
-    for (int ph = first; ph <= last; ph++) {
-        const int cur = (ph - first) & 1;
-        if (ph != last) fetch_desc(&sd[cur ^ 1], &descs[ph + 1]);
-        vec_phase<V>(g, sd[cur], warp_id, n_warps, threadIdx.x & 31u);
-        if (ph != last) {
-            // the cluster barrier also orders this CTA's shared-memory descriptor fetch
-            asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    chain_trigger();
+    chain_wait();  // the collective before this one in the stream is complete
+    if (ld_relaxed_gpu(fa.status) != DEV_OK) return;  // an earlier failure was not cleared yet
+    const uint32_t P = g.P;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t wpb = blockDim.x >> 5;
+    const uint32_t n_warps = gridDim.x * wpb;
+    const uint32_t warp_id = blockIdx.x * wpb + (threadIdx.x >> 5);
+    constexpr uint32_t span = 32u * U;
+
+    // completion of the unit before: signalled after the next unit's first loads are on their
+    // way (the fence then waits for stores that have long been issued), or before any wait
+    unsigned* pend0 = nullptr;
+    unsigned* pend1 = nullptr;
+    auto flush = [&]() {
+        if (pend0) {
+            __syncwarp();
+            if (lane == 0) {
+                fence_acq_rel_gpu();  // the unit's stores (all lanes, ordered by the warp barrier) first
+                red_relaxed_gpu_add(pend0, 1u);
+                if (pend1) red_relaxed_gpu_add(pend1, 1u);
+            }
+            pend0 = pend1 = nullptr;
         }
+    };
+
+    uint64_t g0 = 0;  // number of the pass's first unit
+    for (uint32_t i = 0; i < fa.n; i++) {
+        const FlowPass fp = fa.pass[i];
+        const PhaseDesc& d = sd[i];
+        const uint32_t units = P * fp.upr;  // < 2^32, host-checked
+        const uint32_t spans_per_rank = d.copies * fp.spc;
+        const uint64_t vpc64 = d.copy_bytes / sizeof(V);
+        const char* sbase = space_base(g, d.src_space);
+        char* dbase = space_base(g, d.dst_space);
+        const uint64_t spitch = space_pitch(g, d.src_space);
+        const uint64_t dpitch = space_pitch(g, d.dst_space);
+        const bool polls = lane < i && ((fp.dep_mask >> lane) & 1u);
+        uint32_t w = (warp_id + n_warps - (uint32_t)(g0 % n_warps)) % n_warps;
+        for (; w < units; w += n_warps) {
+            const uint32_t x = w / fp.upr;
+            const uint32_t k = w - x * fp.upr;
+            uint32_t r = x + fp.rot;
+            if (r >= P) r -= P;
+            // the Waitall of rank r: everything it receives before this pass has arrived
+            if (fp.dep_mask) {
+                const unsigned* line = fa.cnt + (size_t)r * kFlowMaxPasses;
+                bool ok = !polls || (int)(ld_acquire_gpu(line + lane) - s_target[lane]) >= 0;
+                if (!__all_sync(0xffffffffu, ok)) {
+                    flush();
+                    const unsigned long long t0 = globaltimer_ns();
+                    unsigned tries = 0;
+                    for (;;) {
+                        ok = !polls || (int)(ld_acquire_gpu(line + lane) - s_target[lane]) >= 0;
+                        if (__all_sync(0xffffffffu, ok)) break;
+                        if ((++tries & 15u) == 0) {
+                            bool give_up = false;
+                            if (lane == 0) {
+                                if (ld_relaxed_gpu(fa.status) != DEV_OK) give_up = true;
+                                else if (globaltimer_ns() - t0 > fa.timeout_ns) {
+                                    atomicCAS(fa.status, DEV_OK, DEV_BARRIER_TIMEOUT);
+                                    give_up = true;
+                                }
+                            }
+                            if (__any_sync(0xffffffffu, give_up)) return;
+                        }
+                    }
+                }
+                __syncwarp();  // what one lane acquired, all lanes may read
+            }
+            const uint32_t s0 = k * fp.us;
+            uint32_t s1 = s0 + fp.us;
+            if (s1 > spans_per_rank) s1 = spans_per_rank;
+            uint32_t j = s0 / fp.spc;
+            uint32_t sp = s0 - j * fp.spc;
+            uint32_t dst_rank = 0;
+            for (uint32_t s = s0; s < s1; s++) {
+                const CopyLoc c = locate_copy(d, P, r, j);
+                dst_rank = c.dst_rank;
+                const V* src = reinterpret_cast<const V*>(sbase + ((uint64_t)c.src_rank * spitch + (uint64_t)c.src_slot * g.m));
+                V* dst = reinterpret_cast<V*>(dbase + ((uint64_t)c.dst_rank * dpitch + (uint64_t)c.dst_slot * g.m));
+                V* dst2 = reinterpret_cast<V*>(dbase + ((uint64_t)r * dpitch + (uint64_t)c.dst_slot * g.m));
+                const uint64_t v0 = (uint64_t)sp * span + lane;
+                V regs[U];
+#pragma unroll
+                for (int q = 0; q < U; q++) {
+                    const uint64_t v = v0 + 32u * q;
+                    if (v < vpc64) regs[q] = ld_cg<V>(src + v);
+                }
+                if (s == s0) flush();
+#pragma unroll
+                for (int q = 0; q < U; q++) {
+                    const uint64_t v = v0 + 32u * q;
+                    if (v < vpc64) {
+                        st_cg<V>(dst + v, regs[q]);
+                        if (d.dup_self) st_cg<V>(dst2 + v, regs[q]);
+                    }
+                }
+                if (++sp == fp.spc) {
+                    sp = 0;
+                    j++;
+                }
+            }
+            pend0 = fa.cnt + (size_t)dst_rank * kFlowMaxPasses + i;
+            pend1 = d.dup_self && dst_rank != r ? fa.cnt + (size_t)r * kFlowMaxPasses + i : nullptr;
+            if (fp.eager) flush();
+        }
+        g0 += units;
     }
+    flush();
 }
 
 }  // namespace spb

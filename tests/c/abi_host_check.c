@@ -50,6 +50,12 @@ int main(void) {
     }
     CHECK(sparbit_plan_workspace_bytes(plan) == 0);
     CHECK(sparbit_plan_exec_mode(plan) == SPARBIT_EXEC_GRAPH);
+    {
+        uint64_t v = 0;
+        CHECK(sparbit_plan_get_tunable(plan, SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES, &v) == SPARBIT_OK && v == 8192);
+        CHECK(sparbit_plan_set_tunable(plan, SPARBIT_TUNE_COUNT_, 1) == SPARBIT_ERR_ARG);
+        CHECK(sparbit_rank_device(13, 2, SPARBIT_MAP_SEQUENTIAL, 6) == 1 && sparbit_rank_device(13, 2, SPARBIT_MAP_CYCLIC, 6) == 0);
+    }
     /* argument errors are found before anything touches a device */
     CHECK(sparbit_allgather(plan, NULL, NULL, NULL) == SPARBIT_ERR_ARG);
     CHECK(sparbit_allgather_steps(plan, (const void*)4096, (void*)(1 << 24), NULL, 3, 1) == SPARBIT_ERR_ARG);

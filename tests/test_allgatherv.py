@@ -88,8 +88,8 @@ def test_create_v_errors_and_introspection():
     assert lib.sparbit_plan_create_v(0, counts, 0, 0, ctypes.byref(out)) == sp.ERR_ARG
     assert lib.sparbit_plan_create_v(4, counts, 0, 0, None) == sp.ERR_ARG
     assert lib.sparbit_plan_create_v(4, counts, sp.ALGO_BRUCK, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
-    assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_PERSISTENT, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
-    assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_CLUSTER, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_FLOW, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create_v(4, counts, 0, 9, ctypes.byref(out)) == sp.ERR_ARG
     assert lib.sparbit_plan_create_v(3, counts, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     many = (ctypes.c_size_t * 8193)(*([16] * 8193))
     assert lib.sparbit_plan_create_v(8193, many, 0, 0, ctypes.byref(out)) == sp.ERR_LIMIT
@@ -117,9 +117,10 @@ def _gpu():
     return torch, torch.device("cuda:0")
 
 
-def run_v_case(P, counts, algo, exec_mode, seed, shift=0, iters=2):
+def run_v_case(P, counts, algo, exec_mode, seed, shift=0, iters=2, copy=sp.COPY_AUTO):
     torch, dev = _gpu()
     plan = sp.Plan.create_v(counts, algo, exec_mode)
+    plan.set_copy_path(copy)
     ref = oracle.Plan(algo, P)
     T = sum(counts)
     G = si.GUARD_BYTES
@@ -143,13 +144,18 @@ def run_v_case(P, counts, algo, exec_mode, seed, shift=0, iters=2):
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("algo", V_ALGOS)
-@pytest.mark.parametrize("exec_mode", [sp.EXEC_AUTO, sp.EXEC_STREAM])
-def test_gpu_v_parity_mixed_sizes(algo, exec_mode):
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_AUTO, sp.EXEC_STREAM, sp.EXEC_PERSISTENT])
+@pytest.mark.parametrize("copy", [sp.COPY_VECTOR, sp.COPY_BULK])
+def test_gpu_v_parity_mixed_sizes(algo, exec_mode, copy):
+    """Both copy engines and all three executors.  Byte counts that are not multiples of 16 send
+    a bulk request to the vector engine (the bulk engine moves 16-byte units), which is part of
+    what is checked."""
     for P in (1, 2, 5, 6, 8, 13, 16, 32, 50, 64):
         if not defined_for(algo, P):
             continue
         for unit, scale in ((16, 40), (1, 30), (4, 300), (16, 1200)):
-            run_v_case(P, si.block_counts(P, 40 + P + unit, unit=unit, scale=scale), algo, exec_mode, 77, iters=1)
+            run_v_case(P, si.block_counts(P, 40 + P + unit, unit=unit, scale=scale), algo, exec_mode, 77, iters=1,
+                       copy=copy)
 
 
 @pytest.mark.gpu
@@ -176,12 +182,15 @@ def test_gpu_v_equal_sizes_match_the_fixed_size_plan():
 
 
 @pytest.mark.gpu
-def test_gpu_v_state_after_every_phase():
+@pytest.mark.parametrize("exec_mode,copy", [(sp.EXEC_STREAM, sp.COPY_VECTOR), (sp.EXEC_STREAM, sp.COPY_BULK),
+                                            (sp.EXEC_PERSISTENT, sp.COPY_VECTOR), (sp.EXEC_PERSISTENT, sp.COPY_BULK)])
+def test_gpu_v_state_after_every_phase(exec_mode, copy):
     torch, dev = _gpu()
     P = 21
-    counts = si.block_counts(P, 5, unit=16, scale=20)
+    counts = si.block_counts(P, 5, unit=16, scale=400)   # up to 13 KiB: several segments per block
     T = sum(counts)
-    plan = sp.Plan.create_v(counts, sp.ALGO_SPARBIT, sp.EXEC_STREAM)
+    plan = sp.Plan.create_v(counts, sp.ALGO_SPARBIT, exec_mode)
+    plan.set_copy_path(copy)
     ref = oracle.Plan(oracle.SPARBIT, P)
     host_send = si.send_blocks_v(counts, 3)
     send = torch.from_numpy(host_send).to(dev)
@@ -192,6 +201,15 @@ def test_gpu_v_state_after_every_phase():
         assert plan.status() == sp.OK
         ref.run_v(counts, host_send, want, first=ph, last=ph)
         assert np.array_equal(recv.cpu().numpy(), want), ph
+    assert plan.copy_path == copy
+    # and two phases in one launch (the persistent kernel's grid barrier between them)
+    recv.fill_(si.SENTINEL)
+    want.fill(si.SENTINEL)
+    plan.allgather_steps(send, recv, -1, 1)
+    plan.allgather_steps(send, recv, 2, ref.num_steps - 1)
+    assert plan.status() == sp.OK
+    ref.run_v(counts, host_send, want)
+    assert np.array_equal(recv.cpu().numpy(), want)
 
 
 @pytest.mark.gpu
@@ -199,6 +217,8 @@ def test_gpu_v_large_blocks_and_host_entry_point():
     P = 64
     counts = si.block_counts(P, 11, unit=16, scale=2048)   # about 32 KiB on average, up to ~390 KiB
     run_v_case(P, counts, sp.ALGO_SPARBIT, sp.EXEC_AUTO, 5, iters=1)
+    run_v_case(P, counts, sp.ALGO_SPARBIT, sp.EXEC_PERSISTENT, 5, iters=2, copy=sp.COPY_BULK)
+    run_v_case(P, counts, sp.ALGO_SPARBIT, sp.EXEC_GRAPH, 5, iters=2, copy=sp.COPY_BULK)
     plan = sp.Plan.create_v(counts)
     T = sum(counts)
     host_send = si.send_blocks_v(counts, 6)

@@ -19,7 +19,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK, sp.ALGO_NEIGHBOR_EXCHANGE]
-EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_CLUSTER]
+EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_FLOW]
 COPIES = [sp.COPY_VECTOR, sp.COPY_BULK]
 G = si.GUARD_BYTES
 
@@ -162,10 +162,14 @@ def test_state_after_every_phase(dev, algo, P, exec_mode):
 
 
 # ---------------------------------------------------------------- brute force over P
-@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_CLUSTER])
-def test_every_p_up_to_64(dev, exec_mode):
+@pytest.mark.parametrize("exec_mode,m", [(sp.EXEC_PERSISTENT, 16), (sp.EXEC_FLOW, 512), (sp.EXEC_FLOW, 1040),
+                                         (sp.EXEC_FLOW, 16)])
+def test_every_p_up_to_64(dev, exec_mode, m):
+    """Every communicator size, on both single-kernel executors.  The flow executor takes blocks
+    of at least 32 vectors (512 B: one warp row; 1040 B: two ragged spans per block) and hands
+    smaller ones to the graph chain."""
     for P in range(1, 65):
-        run_case(dev, P, 16, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=1)
+        run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=2 if m != 16 else 1)
 
 
 @pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK,
@@ -181,7 +185,7 @@ def test_comparators_many_p(dev, algo):
 
 # ---------------------------------------------------------------- any block size, any alignment
 @pytest.mark.parametrize("m", [1, 2, 3, 6, 10, 20, 100, 1000, 4100, 16400])
-@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_CLUSTER])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_FLOW])
 def test_odd_block_sizes(dev, m, exec_mode):
     run_case(dev, 7, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 31 + m, iters=1)
 
@@ -245,6 +249,44 @@ def test_grid_barrier_gives_up_instead_of_hanging(dev, copy):
     assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
 
 
+def test_flow_wait_gives_up_instead_of_hanging(dev):
+    """The flow executor's per-rank waits are bounded too: with counter targets that are never
+    reached (the same host-set hook) every waiting warp must leave with the time-out status, and
+    the plan must work again afterwards, its counters cleared."""
+    P, m = 16, 4096
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_FLOW)
+    host_send = si.send_blocks(P, m, 1)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_FLOW
+    plan.set_barrier_test(1, 20_000_000)  # 20 ms
+    plan.allgather(send, recv)
+    assert plan.status() == sp.ERR_TIMEOUT
+    assert plan.status() == sp.OK
+    plan.set_barrier_test(0, 0)
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    for _ in range(2):
+        recv.fill_(si.SENTINEL)
+        plan.allgather(send, recv)
+        assert plan.status() == sp.OK
+        assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_flow_all_algorithms_changing_data(dev, algo):
+    """Every algorithm on the flow executor, several calls in a row on one plan (the counters
+    carry over from call to call) with new data and a fresh sentinel fill each time."""
+    for P, m in ((16, 2048), (12, 1024), (64, 512), (13, 4096), (1, 512), (2, 8192)):
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
+            continue
+        if algo == sp.ALGO_RING and P > 32:
+            continue   # more passes than the flow executor's counter line holds: runs as a graph
+        run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 77 + P, iters=3)
+
+
 # ---------------------------------------------------------------- host-buffer entry point, streams, bookkeeping
 @pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_BRUCK])
 def test_host_entry_point(dev, algo):
@@ -275,7 +317,7 @@ def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
     assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
     kernels, graphs = plan.launch_counts()
     phases = plan.num_steps  # the own-block copy and step 0 run as one fused pass
-    if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_CLUSTER):
+    if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_FLOW):
         assert (kernels, graphs) == (2, 0)
     elif exec_mode == sp.EXEC_GRAPH:
         assert (kernels, graphs) == (2 * phases, 2)

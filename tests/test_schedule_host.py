@@ -135,14 +135,31 @@ def test_strerror_covers_every_code():
 
 def test_exec_mode_resolution():
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH             # measured best at every size
-    assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH
+    assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH         # 8.6 GB moved: chain + bulk engine
+    assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
+    assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
+    assert sp.Plan(256, 4096).exec_mode == sp.EXEC_GRAPH          # 0.5 GB moved
+    assert sp.Plan(40000, 1).exec_mode == sp.EXEC_GRAPH           # blocks shorter than a warp row
     assert sp.Plan(256, 65536, exec_mode=sp.EXEC_PERSISTENT).exec_mode == sp.EXEC_PERSISTENT
+
+
+def test_engine_thresholds_are_plan_fields():
+    plan = sp.Plan(8, 64)
+    assert plan.get_tunable(sp.TUNE_BULK_MIN_BLOCK_BYTES) == 8192
+    assert plan.get_tunable(sp.TUNE_BULK_MIN_MOVED_BYTES) == 10 ** 9
+    plan.set_tunable(sp.TUNE_BULK_MIN_BLOCK_BYTES, 4096)
+    assert plan.get_tunable(sp.TUNE_BULK_MIN_BLOCK_BYTES) == 4096
+    with pytest.raises(sp.binding.SparbitError):
+        plan.set_tunable(99, 1)
 
 
 def test_environment_overrides_only_the_automatic_choice(monkeypatch):
     monkeypatch.setenv("SPARBIT_EXEC", "persistent")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_PERSISTENT
     assert sp.Plan(8, 64, exec_mode=sp.EXEC_STREAM).exec_mode == sp.EXEC_STREAM   # explicit wins
+    assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_PERSISTENT
+    monkeypatch.setenv("SPARBIT_EXEC", "flow")
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_FLOW
     assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_GRAPH                  # not offered there
     monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH
