@@ -286,7 +286,7 @@ def run_ours(args):
         e1.record(stream)
         stream.synchronize()
         est_ms = max_over_ranks(e0.elapsed_time(e1), dev, use_dist)   # one untimed round sizes the run
-        rounds = int(min(200, max(1, -(-MIN_TIMED_MS // max(est_ms, 1e-3)))))
+        rounds = int(min(200, max(1, -(-args.min_timed_ms // max(est_ms, 1e-3)))))
 
         sampler = ClockSampler(local)
         if rank == 0:
@@ -503,39 +503,38 @@ def run_sweep(args):
                     continue  # same kernels as the graph chain; skipped to bound the sweep
                 if cname == "bulk" and (m % 16 or ename == "flow"):
                     continue
-                if True:
-                    plan = sp.Plan(P, m, algos[name], e)
-                    plan.set_copy_path(c)
-                    if name == "bruck":
-                        plan.set_workspace(work, P * P * m)
-                    with torch.cuda.stream(stream):
-                        for it in range(5):
-                            plan.allgather(sends[it & 1], recv, stream)
-                        stream.synchronize()
-                        ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
-                        k_before = plan.launch_counts()[0]
-                        ev[0].record(stream)
-                        for it in range(50):
-                            plan.allgather(sends[it & 1], recv, stream)
-                            ev[it + 1].record(stream)
-                        stream.synchronize()
-                    assert plan.status() == sp.OK
-                    ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
-                    us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(50)]
-                    avg = float(np.mean(us))
-                    print(json.dumps({
-                        "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
-                        "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
-                        "launches_per_collective": (plan.launch_counts()[0] - k_before) / 50,
-                        "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
-                        "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
-                        "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
-                        "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
-                        "pct_nominal_hbm": round(100 * effective_bytes(P, m) / avg / 1e3 / NOMINAL_HBM_GBS, 1),
-                        "oracle_ms": oracle_ms if name == "sparbit" else None,
-                        "oracle_cores": cores if name == "sparbit" and oracle_ms is not None else None,
-                        "checked": ok}), flush=True)
-                    plan.destroy()
+                plan = sp.Plan(P, m, algos[name], e)
+                plan.set_copy_path(c)
+                if name == "bruck":
+                    plan.set_workspace(work, P * P * m)
+                with torch.cuda.stream(stream):
+                    for it in range(5):
+                        plan.allgather(sends[it & 1], recv, stream)
+                    stream.synchronize()
+                    ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
+                    k_before = plan.launch_counts()[0]
+                    ev[0].record(stream)
+                    for it in range(50):
+                        plan.allgather(sends[it & 1], recv, stream)
+                        ev[it + 1].record(stream)
+                    stream.synchronize()
+                assert plan.status() == sp.OK
+                ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
+                us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(50)]
+                avg = float(np.mean(us))
+                print(json.dumps({
+                    "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
+                    "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
+                    "launches_per_collective": (plan.launch_counts()[0] - k_before) / 50,
+                    "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
+                    "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
+                    "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
+                    "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
+                    "pct_nominal_hbm": round(100 * effective_bytes(P, m) / avg / 1e3 / NOMINAL_HBM_GBS, 1),
+                    "oracle_ms": oracle_ms if name == "sparbit" else None,
+                    "oracle_cores": cores if name == "sparbit" and oracle_ms is not None else None,
+                    "checked": ok}), flush=True)
+                plan.destroy()
         del sends, recv, work
         torch.cuda.empty_cache()
     return 0
@@ -694,6 +693,9 @@ def main():
     ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "flow"], default="auto")
     ap.add_argument("--copy", choices=["auto", "vector", "bulk"], default="auto")
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="rounds of --steps collectives are repeated until the timed work lasts this long "
+                         "(0 = one round, for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,

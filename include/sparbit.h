@@ -268,6 +268,18 @@ int sparbit_plan_partition(const sparbit_plan_t* plan, int G, int mapping, int p
 int sparbit_plan_partition_messages(const sparbit_plan_t* plan, int G, int mapping, int phase, int src_device,
                                     int dst_device, sparbit_msg* out, size_t cap, size_t* n);
 
+/*
+ * The same kind of check for the bookkeeping of the FLOW executor, which replaces the Waitall of
+ * Algorithm 1 by per-rank counters: for vector_bytes-wide vectors (1, 2, 4, 8 or 16) and
+ * resident_warps warps, the work units of every pass, decoded the way the kernel decodes them,
+ * must cover each rank's copies exactly once; the units that write into a rank's buffer must
+ * number what the counter of that (rank, pass) is compared with; and a pass must wait for every
+ * earlier pass that writes the space it reads.  SPARBIT_OK, SPARBIT_ERR_ARG with the offending
+ * pass in *bad_pass (may be NULL), SPARBIT_ERR_UNSUPPORTED if the plan cannot run on FLOW with
+ * that vector width, SPARBIT_ERR_LIMIT for more than 2^26 spans in a pass.  Host-only.
+ */
+int sparbit_plan_validate_flow(const sparbit_plan_t* plan, int vector_bytes, int resident_warps, int* bad_pass);
+
 /* Bytes of workspace the plan needs: 0, or P*P*m for Bruck. */
 size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* plan);
 
@@ -348,17 +360,18 @@ int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint
  * carries those 2 KiB until the process exits.  On the host it uses only short-lived ordinary
  * heap memory for the schedule.
  *
- * It runs the persistent executor with the vector copy engine (the same kernel
- * sparbit_allgather launches for EXEC_PERSISTENT / COPY_VECTOR), for algo = SPARBIT, RING or
- * RECURSIVE_DOUBLING; sendbuf / recvbuf / stream as for sparbit_allgather.  Unlike
- * sparbit_allgather it WAITS: the work is enqueued on `stream`, the stream is synchronised, and
- * the return value is final - SPARBIT_OK, or SPARBIT_ERR_TIMEOUT if the grid barrier gave up
- * (recvbuf is then incomplete).
+ * It runs the persistent executor with the vector copy engine (the same kernel and the same
+ * passes sparbit_allgather launches for EXEC_PERSISTENT / COPY_VECTOR, the fused first pass
+ * included), for algo = SPARBIT, RING, RECURSIVE_DOUBLING or NEIGHBOR_EXCHANGE; sendbuf / recvbuf /
+ * stream as for sparbit_allgather.  Unlike sparbit_allgather it WAITS: the work is enqueued on
+ * `stream`, then the call synchronises that stream, on every call, and the return value is
+ * final - SPARBIT_OK, or SPARBIT_ERR_TIMEOUT if the grid barrier gave up (recvbuf is then
+ * incomplete).
  *
- * Limit: the array holds 28 phase descriptors, i.e. any Sparbit or recursive-doubling
- * collective this library accepts (K + 1 <= 25 phases) and rings of at most 28 ranks.  Anything
- * larger is refused with SPARBIT_ERR_LIMIT before anything is enqueued.  Bruck needs a
- * P*P*m workspace and is refused with SPARBIT_ERR_UNSUPPORTED.
+ * Limit: the array holds 28 pass descriptors, i.e. any Sparbit or recursive-doubling collective
+ * this library accepts (at most 24 passes), rings of at most 29 ranks and neighbor exchanges of
+ * at most 56.  Anything larger is refused with SPARBIT_ERR_LIMIT before anything is enqueued.
+ * Bruck needs a P*P*m workspace and is refused with SPARBIT_ERR_UNSUPPORTED.
  *
  * The first call on each device looks up the array's device address (once per device, with that
  * device current); make that first call before any stream capture begins.  All calls on a

@@ -48,6 +48,7 @@ SYMBOLS = {
     "sparbit_plan_step_info": (_i, [_vp, _i, _pi, _pi, _pi]),
     "sparbit_plan_messages": (_i, [_vp, _i, _vp, _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_validate": (_i, [_vp, _pi]),
+    "sparbit_plan_validate_flow": (_i, [_vp, _i, _i, _pi]),
     "sparbit_rank_device": (_i, [_i, _i, _i, _i]),
     "sparbit_plan_partition": (_i, [_vp, _i, _i, _i, ctypes.POINTER(_u64)]),
     "sparbit_plan_partition_messages": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _sz, ctypes.POINTER(_sz)]),
@@ -198,6 +199,15 @@ class Plan:
         code = lib.sparbit_plan_validate(self._h, ctypes.byref(bad))
         if code != OK:
             raise SparbitError(code, f"sparbit_plan_validate (phase {bad.value})")
+
+    def validate_flow(self, vector_bytes: int = 16, resident_warps: int = 4736) -> int:
+        """Host-side check of the flow executor's units and counters; returns the library's code
+        (OK, or ERR_UNSUPPORTED when the plan cannot run on that executor) and raises on a fault."""
+        bad = ctypes.c_int()
+        code = lib.sparbit_plan_validate_flow(self._h, vector_bytes, resident_warps, ctypes.byref(bad))
+        if code not in (OK, ERR_UNSUPPORTED):
+            raise SparbitError(code, f"sparbit_plan_validate_flow (pass {bad.value})")
+        return code
 
     @property
     def workspace_bytes(self) -> int:

@@ -67,7 +67,6 @@ struct sparbit_plan_s {
     bool variable = false;
     std::vector<uint64_t> voff;
     uintptr_t voff_bits = 0;  // OR of all prefix sums: decides the vector width
-    uint64_t* d_voff = nullptr;
     // task lists of the variable-size kernels, one per descriptor of the device table order
     // (phases in order, then the fused first pass): entries, and where each list starts
     std::vector<VarTask> vtasks;
@@ -202,8 +201,6 @@ int ensure_device(sparbit_plan_s* p) {
     if (!p->d_descs) CU(cudaMalloc((void**)&p->d_descs, n * sizeof(PhaseDesc)));
     CU(cudaMemcpy(p->d_descs, table.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice));
     if (p->variable) {
-        if (!p->d_voff) CU(cudaMalloc((void**)&p->d_voff, p->voff.size() * sizeof(uint64_t)));
-        CU(cudaMemcpy(p->d_voff, p->voff.data(), p->voff.size() * sizeof(uint64_t), cudaMemcpyHostToDevice));
         const size_t nt = p->vtasks.size() ? p->vtasks.size() : 1;
         if (!p->d_vtasks) CU(cudaMalloc((void**)&p->d_vtasks, nt * sizeof(VarTask)));
         if (p->vtasks.size())
@@ -327,13 +324,11 @@ Geom make_geom(const sparbit_plan_s* p, const void* send, void* recv) {
     g.rank_pitch[SPACE_SEND] = g.m;
     g.rank_pitch[SPACE_RECV] = (uint64_t)g.P * g.m;
     g.rank_pitch[SPACE_WORK] = (uint64_t)g.P * g.m;
-    g.voff = nullptr;
     if (p->variable) {
         g.m = 0;
         g.rank_pitch[SPACE_SEND] = 0;                 // send blocks sit at voff[rank]
         g.rank_pitch[SPACE_RECV] = p->voff.back();    // every receive buffer holds all blocks
         g.rank_pitch[SPACE_WORK] = 0;
-        g.voff = p->d_voff;
     }
     return g;
 }
@@ -734,6 +729,49 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     return SPARBIT_OK;
 }
 
+// The flow executor's pass table (host only): how each pass is cut into units, where its rank
+// enumeration starts, which earlier passes a unit has to wait for, and the counter value that
+// says "all units of this launch that write into this rank in this pass are done".  Returns the
+// unit count of the largest pass.
+uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint64_t max_warps, unsigned epoch,
+                         bool never_reached, FlowArgs& fa) {
+    const uint32_t P = p->sched.P;
+    const int n = seq.count();
+    fa.n = (uint32_t)n;
+    uint64_t most_units = 1;
+    uint32_t rot = 0;
+    for (int i = 0; i < n; i++) {
+        const PhaseDesc& d = seq.item(i);
+        FlowPass& fp = fa.pass[i];
+        const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
+        fp.spc = (uint32_t)((vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll));
+        const uint64_t spans = (uint64_t)d.copies * fp.spc;  // per source rank
+        // Unit size: a small pass is cut into single spans, so that as many warps as possible share
+        // it and a hop (copy, release, the next pass's poll) stays short; a pass that keeps every
+        // warp busy takes units of up to FLOW_MAX_UNIT_SPANS spans, which spreads
+        // the poll and the release over more bytes.
+        uint64_t us = (uint64_t)P * spans / (max_warps * p->tune[SPARBIT_TUNE_FLOW_UNITS_PER_WARP]);
+        if (us < 1) us = 1;
+        if (us > p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS]) us = p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS];
+        if (us > spans) us = spans;
+        fp.us = (uint32_t)us;
+        fp.upr = (uint32_t)((spans + fp.us - 1) / fp.us);
+        fp.rot = rot;
+        // units that write into one rank's buffer in this pass: those of its one sender, and in the
+        // fused first pass its own as well
+        const uint32_t per_rank = fp.upr * (d.dup_self ? 2u : 1u);
+        fp.target = epoch * per_rank + (never_reached ? 1u : 0u);  // test hook: a target that is never reached
+        fp.dep_mask = 0;
+        for (int k = 0; k < i; k++)
+            if (seq.item(k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
+        if ((uint64_t)P * fp.upr > most_units) most_units = (uint64_t)P * fp.upr;
+        fp.eager = (uint64_t)P * fp.upr <= max_warps ? 1u : 0u;
+        // the next pass starts its enumeration where this pass's first receivers are
+        if (d.peer_xor == 0 && d.peer_pre == 0) rot = (rot + d.peer_add) % P;
+    }
+    return most_units;
+}
+
 // The whole collective as one cooperative kernel without grid barriers (flow_vec_kernel).
 int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
@@ -763,37 +801,7 @@ int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first,
     if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "flow kernel does not fit on an SM");
     if (per_sm > 2) per_sm = 2;
     const uint64_t max_warps = (uint64_t)per_sm * p->sm_count * (kVecBlock / 32);
-    uint64_t most_units = 1;
-    uint32_t rot = 0;
-    for (int i = 0; i < n; i++) {
-        const PhaseDesc& d = seq.item(i);
-        FlowPass& fp = fa.pass[i];
-        const uint64_t vpc = d.copy_bytes / (uint64_t)rs.vbytes;
-        fp.spc = (uint32_t)((vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll));
-        const uint64_t spans = (uint64_t)d.copies * fp.spc;  // per source rank
-        // Unit size: a small pass is cut into single spans, so that as many warps as possible share
-        // it and a hop (copy, release, the next pass's poll) stays short; a pass that keeps every
-        // warp busy takes units of up to FLOW_MAX_UNIT_SPANS spans, which spreads
-        // the poll and the release over more bytes.
-        uint64_t us = (uint64_t)P * spans / (max_warps * p->tune[SPARBIT_TUNE_FLOW_UNITS_PER_WARP]);
-        if (us < 1) us = 1;
-        if (us > p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS]) us = p->tune[SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS];
-        if (us > spans) us = spans;
-        fp.us = (uint32_t)us;
-        fp.upr = (uint32_t)((spans + fp.us - 1) / fp.us);
-        fp.rot = rot;
-        // units that write into one rank's buffer in this pass: those of its one sender, and in the
-        // fused first pass its own as well
-        const uint32_t per_rank = fp.upr * (d.dup_self ? 2u : 1u);
-        fp.target = p->flow_epoch * per_rank + (p->extra_arrivals ? 1u : 0u);  // test hook: never reached
-        fp.dep_mask = 0;
-        for (int k = 0; k < i; k++)
-            if (seq.item(k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
-        if ((uint64_t)P * fp.upr > most_units) most_units = (uint64_t)P * fp.upr;
-        fp.eager = (uint64_t)P * fp.upr <= max_warps ? 1u : 0u;
-        // the next pass starts its enumeration where this pass's first receivers are
-        if (d.peer_xor == 0 && d.peer_pre == 0) rot = (rot + d.peer_add) % P;
-    }
+    const uint64_t most_units = flow_pass_table(p, seq, rs.vbytes, max_warps, p->flow_epoch, p->extra_arrivals != 0, fa);
     uint64_t grid = (uint64_t)per_sm * p->sm_count;
     const uint64_t need = (most_units + kVecBlock / 32 - 1) / (kVecBlock / 32);
     if (grid > need) grid = need;
@@ -989,7 +997,6 @@ int sparbit_plan_destroy(sparbit_plan_t* p) {
         drop_graph(p);
         if (p->capture_stream) cudaStreamDestroy(p->capture_stream);
         cudaFree(p->d_descs);
-        cudaFree(p->d_voff);
         cudaFree(p->d_vtasks);
         cudaFree(p->d_vranges);
         cudaFree(p->d_trace);
@@ -1285,6 +1292,70 @@ int sparbit_plan_validate(const sparbit_plan_t* p, int* bad_phase) {
     return SPARBIT_OK;
 }
 
+// Host-side check of the flow executor's bookkeeping for a given vector width and number of
+// resident warps: the units of every pass, decoded exactly as the kernel decodes them, must cover
+// every span of every rank's copies once; the number of units that write into a rank's buffer
+// (through either destination of the fused pass) must be the counter target of that pass; and a
+// pass must wait for every earlier pass that writes the space it reads.
+int sparbit_plan_validate_flow(const sparbit_plan_t* p, int vector_bytes, int resident_warps, int* bad_pass) {
+    if (!p || resident_warps < 1) return SPARBIT_ERR_ARG;
+    if (vector_bytes != 1 && vector_bytes != 2 && vector_bytes != 4 && vector_bytes != 8 && vector_bytes != 16)
+        return SPARBIT_ERR_ARG;
+    if (bad_pass) *bad_pass = -1;
+    if (!flow_possible(p, vector_bytes, -1, p->sched.last_phase(), true)) return SPARBIT_ERR_UNSUPPORTED;
+    const uint32_t P = p->sched.P;
+    const ExecSeq seq = make_seq(p, -1, p->sched.last_phase());
+    try {
+        FlowArgs fa;
+        memset(&fa, 0, sizeof fa);
+        const unsigned epoch = 3;
+        flow_pass_table(p, seq, vector_bytes, (uint64_t)resident_warps, epoch, false, fa);
+        for (int i = 0; i < seq.count(); i++) {
+            const PhaseDesc& d = seq.item(i);
+            const FlowPass& fp = fa.pass[i];
+            auto fail = [&]() {
+                if (bad_pass) *bad_pass = i;
+                return SPARBIT_ERR_ARG;
+            };
+            const uint64_t spans_per_rank = (uint64_t)d.copies * fp.spc;
+            if (spans_per_rank * P > (1ull << 26)) return SPARBIT_ERR_LIMIT;
+            std::vector<uint8_t> covered((size_t)(spans_per_rank * P), 0);
+            std::vector<uint32_t> arrivals(P, 0);
+            for (uint64_t w = 0; w < (uint64_t)P * fp.upr; w++) {
+                const uint32_t x = (uint32_t)(w / fp.upr), k = (uint32_t)(w - (uint64_t)x * fp.upr);
+                uint32_t r = x + fp.rot;
+                if (r >= P) r -= P;
+                const uint64_t s0 = (uint64_t)k * fp.us;
+                uint64_t s1 = s0 + fp.us;
+                if (s1 > spans_per_rank) s1 = spans_per_rank;
+                if (s0 >= s1) return fail();  // an empty unit would still be counted
+                uint32_t dst = P;
+                for (uint64_t sidx = s0; sidx < s1; sidx++) {
+                    uint8_t& c = covered[(size_t)(r * spans_per_rank + sidx)];
+                    if (c) return fail();
+                    c = 1;
+                    const CopyLoc loc = locate_copy(d, P, r, (uint32_t)(sidx / fp.spc));
+                    if (dst != P && dst != loc.dst_rank) return fail();  // one destination rank per unit
+                    dst = loc.dst_rank;
+                }
+                arrivals[dst]++;
+                if (d.dup_self && dst != r) arrivals[r]++;
+            }
+            for (uint8_t c : covered)
+                if (!c) return fail();
+            for (uint32_t q = 0; q < P; q++)
+                if (arrivals[q] * epoch != fp.target) return fail();
+            uint32_t want_mask = 0;
+            for (int k = 0; k < i; k++)
+                if (seq.item(k).dst_space == d.src_space) want_mask |= 1u << k;
+            if (fp.dep_mask != want_mask || (d.src_space == SPACE_SEND && fp.dep_mask)) return fail();
+        }
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    return SPARBIT_OK;
+}
+
 const char* sparbit_strerror(int code) {
     switch (code) {
         case SPARBIT_OK: return "success";
@@ -1363,8 +1434,8 @@ extern "C" {
 
 int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* sendbuf, void* recvbuf,
                               void* stream) {
-    if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;
-    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_ARG;
+    if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
+    if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // needs a P*P*m workspace
     Schedule sched;
     int rc;
     try {
@@ -1373,7 +1444,20 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
         rc = SPARBIT_ERR_NOMEM;
     }
     if (rc) return rc;
-    if (sched.phases.size() > (size_t)kNoallocMaxPhases) return SPARBIT_ERR_LIMIT;
+    // what is executed, as in sparbit_allgather: the own-block copy and the first step as one fused
+    // pass where the schedule has one, then the remaining steps
+    std::vector<PhaseDesc> passes;
+    try {
+        if (sched.has_fused_first) {
+            passes.push_back(sched.fused_first);
+            passes.insert(passes.end(), sched.phases.begin() + 2, sched.phases.end());
+        } else {
+            passes = sched.phases;
+        }
+    } catch (const std::bad_alloc&) {
+        return SPARBIT_ERR_NOMEM;
+    }
+    if (passes.size() > (size_t)kNoallocMaxPhases) return SPARBIT_ERR_LIMIT;
     const size_t send_bytes = (size_t)sched.P * sched.m;
     const size_t recv_bytes = (size_t)sched.P * sched.P * sched.m;
     if (send_bytes == 0) return SPARBIT_OK;
@@ -1394,10 +1478,9 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     while (vbytes > 1 && (bits & (uintptr_t)(vbytes - 1))) vbytes >>= 1;
 
     // grid: enough CTAs for the largest phase, at most what is co-resident
-    const int first = -1, last = sched.last_phase();
     uint64_t need = 1;
-    for (int ph = first; ph <= last; ph++) {
-        const uint64_t tasks = vec_tasks(sched.phase(ph), sched.P, vbytes);
+    for (const PhaseDesc& d : passes) {
+        const uint64_t tasks = vec_tasks(d, sched.P, vbytes);
         if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
         const uint64_t t = (tasks + kVecBlock / 32 - 1) / (kVecBlock / 32);
         if (t > need) need = t;
@@ -1415,8 +1498,8 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     // every call starts from a clean scratch: barrier counter and status word at zero, this
     // collective's descriptors in the table (the call waits below, so the host copy outlives it)
     CU(cudaMemsetAsync(ctl_words, 0, kNoallocCtlBytes, st));
-    const size_t n = sched.phases.size();
-    CU(cudaMemcpyAsync(d_descs, sched.phases.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice, st));
+    const size_t n = passes.size();
+    CU(cudaMemcpyAsync(d_descs, passes.data(), n * sizeof(PhaseDesc), cudaMemcpyHostToDevice, st));
 
     Geom g;
     memset(&g, 0, sizeof g);
@@ -1436,9 +1519,11 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     ctl.timeout_ns = kDefaultTimeoutNs;
     ctl.mbar_extra_tx = 0;
     ctl.trace = nullptr;
-    int first_idx = first + 1, last_idx = last + 1;
+    int first_idx = 0, last_idx = (int)n - 1;
     const PhaseDesc* descs = d_descs;
-    void* args[] = {&g, &descs, &first_idx, &last_idx, &ctl};
+    const VarTask* no_tasks = nullptr;
+    const VarRange* no_ranges = nullptr;
+    void* args[] = {&g, &descs, &first_idx, &last_idx, &ctl, &no_tasks, &no_ranges};
     CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(kVecBlock), args, 0, st));
     unsigned words[2] = {0, 0};
     CU(cudaMemcpyAsync(words, ctl_words, sizeof words, cudaMemcpyDeviceToHost, st));

@@ -665,6 +665,59 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
 }
 
 // ------------------------------------------------------------------------------------------------
+// mirror executor: a whole SMALL collective in one CTA, the receive buffers mirrored on chip
+// ------------------------------------------------------------------------------------------------
+// In the latency regime a pass costs two memory round trips (the loads, then the acknowledged
+// stores: 1.6-2.3 us on B200) however passes are separated.  When all P receive buffers together
+// fit into one SM's shared memory, this kernel keeps a copy of them there: every block that is
+// written to a receive buffer is written to global memory AND to the same place of the on-chip
+// copy, and every forwarded block is read from the on-chip copy of the SENDING rank's receive
+// buffer - the slot the schedule names, with the bytes that were stored there one or more passes
+// earlier - instead of from global memory.  The schedule, the passes and their order are
+// unchanged; a pass boundary is the CTA's barrier, and a pass costs a shared-memory access.
+// Only the own blocks are read from global memory (the send buffer).
+constexpr int kMirrorMaxPasses = 16;
+struct MirrorArgs {
+    PhaseDesc d[kMirrorMaxPasses];
+    int n;
+    int pad_[3];
+};
+
+template <typename V>
+__global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
+    extern __shared__ __align__(16) unsigned char mirror[];  // [P][P] slots of m bytes, as the RECV space
+    chain_trigger();
+    chain_wait();
+    const uint32_t P = g.P;
+    const uint32_t vps = (uint32_t)(g.m / sizeof(V));  // vectors per slot
+    V* mir = reinterpret_cast<V*>(mirror);
+    for (int i = 0; i < ma.n; i++) {
+        if (i) __syncthreads();
+        const PhaseDesc& d = ma.d[i];
+        const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
+        const uint32_t total = P * d.copies * vpc;  // fits: the whole receive space is below 256 KiB
+        const bool from_send = d.src_space == SPACE_SEND;
+        for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+            const uint32_t q = t / vpc;
+            const uint32_t v = t - q * vpc;
+            const uint32_t r = q / d.copies;
+            const uint32_t j = q - r * d.copies;
+            const CopyLoc c = locate_copy(d, P, r, j);
+            const V x = from_send ? ld_cg<V>(reinterpret_cast<const V*>(g.base[SPACE_SEND] + (uint64_t)r * g.m) + v)
+                                  : mir[(c.src_rank * P + c.src_slot) * vps + v];
+            const uint32_t at = (c.dst_rank * P + c.dst_slot) * vps + v;
+            mir[at] = x;
+            st_cg<V>(reinterpret_cast<V*>(g.base[SPACE_RECV]) + at, x);
+            if (d.dup_self) {
+                const uint32_t at2 = (r * P + c.dst_slot) * vps + v;
+                mir[at2] = x;
+                st_cg<V>(reinterpret_cast<V*>(g.base[SPACE_RECV]) + at2, x);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // flow executor: the whole collective in one cooperative kernel WITHOUT grid-wide barriers
 // ------------------------------------------------------------------------------------------------
 // Algorithm 1 ends every step with MPI_Waitall, but what a rank sends in step i+1 depends only on

@@ -65,10 +65,8 @@ struct Geom {
     uint64_t m;               // bytes per block (slot pitch)
     char*    base[3];         // SEND, RECV, WORK
     uint64_t rank_pitch[3];   // bytes between consecutive ranks' buffers: m, P*m, P*m
-    // Variable block sizes (allgatherv): device array of P+1 prefix sums of the blocks' byte
-    // counts, else null.  Block b is voff[b+1]-voff[b] bytes and sits at voff[b] both inside the
-    // concatenated send buffer and inside every rank's receive buffer (pitch voff[P]).
-    const uint64_t* voff;
+    // Variable block sizes (allgatherv): m is 0, the send pitch 0 and the receive pitch the sum
+    // of all block sizes; the kernels then work from task records that carry byte offsets.
 };
 
 struct CopyLoc {

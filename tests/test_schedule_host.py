@@ -180,3 +180,30 @@ def test_descriptors_are_race_free_and_in_bounds(algo):
     with pytest.raises(sp.SparbitError) as e:
         sp.Plan(10000, 16).validate()
     assert e.value.code == sp.ERR_LIMIT
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_flow_units_and_counters_are_consistent(algo):
+    """The flow executor's bookkeeping, checked on the host for many communicator sizes, block
+    sizes (one span, ragged spans, many spans per block), vector widths and numbers of warps."""
+    ran = 0
+    for P in list(range(1, 34)) + [61, 64, 100, 128, 253, 256, 1000]:
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
+            continue
+        for m, vb in ((512, 16), (1040, 16), (4096, 16), (65536, 16), (1000, 8), (36, 1)):
+            if P > 256 and m > 4096:
+                continue
+            plan = sp.Plan(P, m, algo)
+            for warps in (1, 64, 4736):
+                code = plan.validate_flow(vb, warps)
+                assert code in (sp.OK, sp.ERR_UNSUPPORTED)
+                # the only things this executor cannot take: more passes than a counter line holds
+                if code == sp.ERR_UNSUPPORTED:
+                    assert plan.last_phase + 2 > 32
+                else:
+                    ran += 1
+            plan.destroy()
+    assert ran > 100
+    assert sp.Plan(8, 64).validate_flow(16) == sp.ERR_UNSUPPORTED   # blocks shorter than a warp row

@@ -14,6 +14,7 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 import seeded_inputs as si
 import paper_2109_08751_b200 as sp
 from paper_2109_08751_b200 import binding
@@ -41,7 +42,8 @@ def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
     # two different collectives back to back: the second finds the first one's descriptors and
     # barrier words in the shared scratch and must not be disturbed by them
     cases = [(13, 4096, sp.ALGO_SPARBIT, 11), (64, 1040, sp.ALGO_SPARBIT, 12),
-             (16, 272, sp.ALGO_RECURSIVE_DOUBLING, 13), (9, 100, sp.ALGO_RING, 14)]
+             (16, 272, sp.ALGO_RECURSIVE_DOUBLING, 13), (9, 100, sp.ALGO_RING, 14),
+             (10, 48, sp.ALGO_NEIGHBOR_EXCHANGE, 15)]
     stream = torch.cuda.Stream(device=dev)
     for P, m, algo, seed in cases:
         for call in range(2):
@@ -52,7 +54,43 @@ def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
             binding.sparbit_allgather_noalloc(P, m, send, got, stream, algo=algo)
             want = regular(P, m, algo, send, dev)
             assert torch.equal(got, want), (P, m, algo, call)          # bit-exact, as everywhere
-            assert torch.equal(got.view(P, P * m)[P - 1], send)         # and it is the allgather
+            # and both are what the CPU oracle computes, over the whole receive space
+            ref, _ = oracle.allgather(algo, P, m, host_send)
+            assert np.array_equal(got.cpu().numpy(), ref.reshape(-1)), (P, m, algo, call)
+
+
+def test_noalloc_leaves_the_amount_of_free_device_memory_alone():
+    """The point of the entry point: after the first call on the device (module load, address
+    look-up) later calls of any size, algorithm and alignment must not change what the driver
+    reports as free device memory, i.e. nothing is allocated behind the caller's back."""
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    # all buffers first, so that torch's own allocator is quiet during the measured calls
+    cases = [(8, 64, sp.ALGO_SPARBIT), (21, 5000, sp.ALGO_SPARBIT), (32, 16384, sp.ALGO_RECURSIVE_DOUBLING),
+             (12, 3, sp.ALGO_RING), (30, 2048, sp.ALGO_NEIGHBOR_EXCHANGE), (200, 1024, sp.ALGO_SPARBIT)]
+    bufs = []
+    for P, m, algo in cases:
+        host_send = si.send_blocks(P, m, 3 + P)
+        bufs.append((host_send, torch.from_numpy(host_send.reshape(-1)).to(dev),
+                     torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)))
+    stream = torch.cuda.Stream(device=dev)
+    binding.sparbit_allgather_noalloc(cases[0][0], cases[0][1], bufs[0][1], bufs[0][2], stream, algo=cases[0][2])
+    torch.cuda.synchronize(dev)
+    for attempt in range(2):   # the figure is device-wide: one repeat, should anything else have moved it
+        free_before = torch.cuda.mem_get_info(dev)[0]
+        changed = []
+        for (P, m, algo), (host_send, send, recv) in zip(cases, bufs):
+            binding.sparbit_allgather_noalloc(P, m, send, recv, stream, algo=algo)
+            if torch.cuda.mem_get_info(dev)[0] != free_before:
+                changed.append((P, m, algo))
+        if not changed:
+            break
+    assert not changed, changed
+    for (P, m, algo), (host_send, send, recv) in zip(cases, bufs):
+        ref, _ = oracle.allgather(algo, P, m, host_send)
+        assert np.array_equal(recv.cpu().numpy(), ref.reshape(-1)), (P, m, algo)
 
 
 def test_noalloc_refuses_what_does_not_fit_its_scratch():
@@ -60,6 +98,9 @@ def test_noalloc_refuses_what_does_not_fit_its_scratch():
     # host-side checks: nothing is enqueued, the pointers are never touched
     assert lib.sparbit_allgather_noalloc(64, 16, sp.ALGO_RING, 4096, 1 << 20, None) == sp.ERR_LIMIT
     assert lib.sparbit_allgather_noalloc(8, 16, sp.ALGO_BRUCK, 4096, 1 << 20, None) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_allgather_noalloc(58, 16, sp.ALGO_NEIGHBOR_EXCHANGE, 4096, 1 << 20, None) == sp.ERR_LIMIT
+    assert lib.sparbit_allgather_noalloc(7, 16, sp.ALGO_NEIGHBOR_EXCHANGE, 4096, 1 << 20, None) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_allgather_noalloc(8, 16, 5, 4096, 1 << 20, None) == sp.ERR_ARG
     assert lib.sparbit_allgather_noalloc(6, 16, sp.ALGO_RECURSIVE_DOUBLING, 4096, 1 << 20, None) \
         == sp.ERR_UNSUPPORTED
     assert lib.sparbit_allgather_noalloc(0, 16, sp.ALGO_SPARBIT, 4096, 1 << 20, None) == sp.ERR_ARG
