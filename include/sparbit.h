@@ -74,19 +74,28 @@ enum {
  * as ONE pass (the own block is read once from sendbuf and written both to its own slot and to
  * the first peer's): same state after phase 0, one pass less. */
 enum {
-    SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: FLOW for collectives that move 1 to
-                                    6 GB (SPARBIT_TUNE_FLOW_*), the graph chain otherwise */
+    SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
+                                    buffers in all, FLOW for collectives that move 1 to 6 GB, the
+                                    graph chain otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
                                     re-parameterise the least recently used graph) */
     SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
-    SPARBIT_EXEC_FLOW = 4        /* one cooperative kernel without grid barriers: Algorithm 1's
+    SPARBIT_EXEC_FLOW = 4,       /* one cooperative kernel without grid barriers: Algorithm 1's
                                     Waitall is kept per rank (counters of what each rank has
                                     received), so a pass starts where its senders are ready while
                                     the pass before is still finishing elsewhere.  Whole
                                     collectives of fixed-size blocks of at least 32 vectors on the
                                     vector engine; other calls run as GRAPH */
+    SPARBIT_EXEC_MIRROR = 5      /* a whole small collective in ONE CTA: every block written to a
+                                    receive buffer is also kept in an on-chip copy of the receive
+                                    buffers (shared memory), and every forwarded block is read from
+                                    that copy of the sending rank's buffer, so a pass costs a
+                                    shared-memory access instead of two trips to global memory.
+                                    Same passes, same order, same slots.  Needs P*P*m to fit into
+                                    one SM's shared memory (227 KB on B200), fixed-size blocks, at
+                                    most 16 passes, not Bruck; other calls run as GRAPH */
 };
 
 /* Which copy engine a phase uses. */
@@ -132,7 +141,7 @@ sparbit_plan_t* sparbit_plan(int P, size_t block_bytes);
  * unknown enum), ERR_OVERFLOW (P*P*block_bytes does not fit in 63 bits, or P > 2^24),
  * ERR_UNSUPPORTED (recursive doubling with P not a power of two, neighbor exchange with odd P:
  * Section II-A defines them for those P only), ERR_NOMEM.  Host-only.
- * Environment: when exec is AUTO, SPARBIT_EXEC=persistent|graph|stream|flow replaces the
+ * Environment: when exec is AUTO, SPARBIT_EXEC=persistent|graph|stream|flow|mirror replaces the
  * automatic choice; SPARBIT_COPY=vector|bulk presets the copy engine (sparbit_plan_set_copy_path
  * still overrides it).  Other values are ignored.
  */
@@ -151,7 +160,7 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
  * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Both copy
  * engines (the bulk engine when all counts and the buffers are multiples of 16 bytes; COPY_AUTO
  * applies its thresholds to the average block) and the GRAPH, STREAM and PERSISTENT executors;
- * FLOW is refused (ERR_UNSUPPORTED: its work units assume equal blocks), and so is Bruck (its
+ * FLOW and MIRROR are refused (ERR_UNSUPPORTED: they assume equal blocks), and so is Bruck (its
  * rotated workspace assumes equal blocks).  P is limited to 8192 here and P * T to 2^48 bytes
  * (ERR_LIMIT, ERR_OVERFLOW beyond: the plan keeps one 16-byte task record per 4 KiB of every
  * copy, with 48-bit offsets).  Other errors as for sparbit_plan_create.  Host-only.
@@ -303,7 +312,8 @@ enum {
     SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS = 3,  /* EXEC_FLOW: largest unit, in warp spans of 1 KiB (8) */
     SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (10^9) */
     SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES = 5, /* ... and below this (6*10^9); GRAPH otherwise */
-    SPARBIT_TUNE_COUNT_ = 6
+    SPARBIT_TUNE_MIRROR_MAX_BYTES = 6,     /* EXEC_AUTO: MIRROR when P*P*m is at most this (64 KiB) */
+    SPARBIT_TUNE_COUNT_ = 7
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

@@ -16,17 +16,17 @@ OK = 0
 ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT = \
     range(1, 10)
 ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK, ALGO_NEIGHBOR_EXCHANGE = range(5)
-EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_FLOW = range(5)
+EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_FLOW, EXEC_MIRROR = range(6)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
 SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
 MAP_SEQUENTIAL, MAP_CYCLIC = range(2)
 (TUNE_BULK_MIN_BLOCK_BYTES, TUNE_BULK_MIN_MOVED_BYTES, TUNE_FLOW_UNITS_PER_WARP, TUNE_FLOW_MAX_UNIT_SPANS,
- TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES) = range(6)
+ TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES, TUNE_MIRROR_MAX_BYTES) = range(7)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
               ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}
 EXEC_NAMES = {EXEC_AUTO: "auto", EXEC_PERSISTENT: "persistent", EXEC_GRAPH: "graph", EXEC_STREAM: "stream",
-              EXEC_FLOW: "flow"}
+              EXEC_FLOW: "flow", EXEC_MIRROR: "mirror"}
 COPY_NAMES = {COPY_AUTO: "auto", COPY_VECTOR: "vector", COPY_BULK: "bulk"}
 
 MSG_DTYPE = np.dtype([("phase", "<i4"), ("src_rank", "<i4"), ("dst_rank", "<i4"), ("src_space", "<i4"),

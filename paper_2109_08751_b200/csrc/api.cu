@@ -42,12 +42,12 @@ struct GraphKey {
     void* recv = nullptr;
     void* work = nullptr;
     int first = 0, last = -2;
-    int path = 0, vec = 0;
+    int path = 0, vec = 0, exec = 0;
     unsigned long long timeout_ns = 0;
     unsigned extra_tx = 0;
     bool same_shape(const GraphKey& o) const {
-        return first == o.first && last == o.last && path == o.path && vec == o.vec && timeout_ns == o.timeout_ns &&
-               extra_tx == o.extra_tx;
+        return first == o.first && last == o.last && path == o.path && vec == o.vec && exec == o.exec &&
+               timeout_ns == o.timeout_ns && extra_tx == o.extra_tx;
     }
     bool same_buffers(const GraphKey& o) const { return send == o.send && recv == o.recv && work == o.work; }
 };
@@ -89,6 +89,7 @@ struct sparbit_plan_s {
     unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
     unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
     int flow_vbytes = 0;             // vector width those launches ran with
+    size_t mirror_smem_set[17] = {};  // dynamic shared memory already granted to the mirror kernel, by vector width
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -108,6 +109,7 @@ struct sparbit_plan_s {
         8,            // FLOW_MAX_UNIT_SPANS
         1000000000u,  // FLOW_MIN_MOVED_BYTES
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
+        64u << 10,    // MIRROR_MAX_BYTES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -139,7 +141,7 @@ struct sparbit_plan_s {
 namespace {
 
 // SPARBIT_EXEC / SPARBIT_COPY in the environment override what AUTO would pick (not an explicit
-// request): persistent|graph|stream|flow and vector|bulk.  Anything else is ignored.
+// request): persistent|graph|stream|flow|mirror and vector|bulk.  Anything else is ignored.
 int env_choice(const char* name, const char* const* words, const int* values, int n, int fallback) {
     const char* v = getenv(name);
     if (!v) return fallback;
@@ -148,9 +150,10 @@ int env_choice(const char* name, const char* const* words, const int* values, in
     return fallback;
 }
 int env_exec(int fallback) {
-    static const char* const w[] = {"persistent", "graph", "stream", "flow"};
-    static const int x[] = {SPARBIT_EXEC_PERSISTENT, SPARBIT_EXEC_GRAPH, SPARBIT_EXEC_STREAM, SPARBIT_EXEC_FLOW};
-    return env_choice("SPARBIT_EXEC", w, x, 4, fallback);
+    static const char* const w[] = {"persistent", "graph", "stream", "flow", "mirror"};
+    static const int x[] = {SPARBIT_EXEC_PERSISTENT, SPARBIT_EXEC_GRAPH, SPARBIT_EXEC_STREAM, SPARBIT_EXEC_FLOW,
+                            SPARBIT_EXEC_MIRROR};
+    return env_choice("SPARBIT_EXEC", w, x, 5, fallback);
 }
 int env_copy(int fallback) {
     static const char* const w[] = {"vector", "bulk"};
@@ -302,6 +305,17 @@ const void* pick_persistent_vec(int vbytes, bool list = false) {
     }
 }
 template <typename V>
+const void* mirror_vec_fn() { return (const void*)mirror_vec_kernel<V>; }
+const void* pick_mirror_vec(int vbytes) {
+    switch (vbytes) {
+        case 16: return mirror_vec_fn<uint4>();
+        case 8: return mirror_vec_fn<uint2>();
+        case 4: return mirror_vec_fn<unsigned>();
+        case 2: return mirror_vec_fn<unsigned short>();
+        default: return mirror_vec_fn<unsigned char>();
+    }
+}
+template <typename V>
 const void* flow_vec_fn() { return (const void*)flow_vec_kernel<V, kVecUnroll>; }
 const void* pick_flow_vec(int vbytes) {
     switch (vbytes) {
@@ -366,6 +380,17 @@ struct Resolved {
     int vbytes;  // vector width for the vector engine
 };
 
+// The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers fit
+// into one CTA's shared memory together, between the send and the receive space only.
+bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_limit) {
+    if (p->variable || p->sched.algo == ALGO_BRUCK) return false;
+    if (first != -1 || last != p->sched.last_phase()) return false;
+    const ExecSeq seq = make_seq(p, first, last);
+    if (seq.count() < 1 || seq.count() > kMirrorMaxPasses) return false;
+    const unsigned __int128 bytes = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
+    return bytes <= (unsigned __int128)smem_limit;
+}
+
 bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, bool assume_coop = false) {
     if (p->variable || !(p->coop || assume_coop)) return false;
     if (first != -1 || last != p->sched.last_phase()) return false;
@@ -382,6 +407,9 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 }
 
 // Executor for SPARBIT_EXEC_AUTO, from measurements on B200.
+//  - Up to 64 KiB of receive buffers in all, the mirror executor: one CTA, passes separated by its
+//    own barrier and fed from shared memory (P = 8, m = 64 B: 4.1 us against 6.2 for the chain;
+//    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain.
 //  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
 //    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
@@ -394,6 +422,9 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.
 int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) &&
+        (uint64_t)p->sched.P * p->sched.P * p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES])
+        return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
@@ -402,6 +433,9 @@ int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
 }
 
 int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
+    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) &&
+        (uint64_t)p->sched.P * p->sched.P * p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES])
+        return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
@@ -442,6 +476,9 @@ Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv, in
     int exec = p->exec_req;
     if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p, r.vbytes, first, last);
     if (exec == SPARBIT_EXEC_PERSISTENT && !p->coop) exec = SPARBIT_EXEC_GRAPH;
+    if (exec == SPARBIT_EXEC_MIRROR && !mirror_possible(p, first, last, (size_t)p->max_smem_optin))
+        exec = SPARBIT_EXEC_GRAPH;
+    if (exec == SPARBIT_EXEC_MIRROR) r.copy = SPARBIT_COPY_VECTOR;
     if (exec == SPARBIT_EXEC_FLOW) {
         // the flow executor runs whole collectives of fixed-size blocks on the vector engine, every
         // copy at least one warp row long; anything else goes to the graph chain
@@ -588,6 +625,8 @@ void drop_graph(sparbit_plan_s* p) {
 
 constexpr size_t kGraphCacheEntries = 4;
 
+int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st);
+
 int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     GraphKey key;
     key.send = g.base[SPACE_SEND];
@@ -597,6 +636,7 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     key.last = last;
     key.path = rs.copy;
     key.vec = rs.vbytes;
+    key.exec = rs.exec;
     key.timeout_ns = p->timeout_ns;
     key.extra_tx = p->mbar_extra_tx;
     sparbit_plan_s::GraphEntry* hit = nullptr;
@@ -607,7 +647,8 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
         if (!p->capture_stream) CU(cudaStreamCreateWithFlags(&p->capture_stream, cudaStreamNonBlocking));
         const uint64_t launches_before = p->kernel_launches;
         CU(cudaStreamBeginCapture(p->capture_stream, cudaStreamCaptureModeThreadLocal));
-        int rc = launch_stream(p, rs, g, first, last, p->capture_stream);
+        int rc = rs.exec == SPARBIT_EXEC_MIRROR ? launch_mirror(p, rs, g, first, last, p->capture_stream)
+                                                : launch_stream(p, rs, g, first, last, p->capture_stream);
         cudaGraph_t graph = nullptr;
         cudaError_t ce = cudaStreamEndCapture(p->capture_stream, &graph);
         p->kernel_launches = launches_before;  // captured, not launched
@@ -651,7 +692,7 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
     hit->stamp = ++p->gstamp;
     CU(cudaGraphLaunch(hit->exec, st));
     p->graph_launches++;
-    p->kernel_launches += (uint64_t)make_seq(p, first, last).count();
+    p->kernel_launches += rs.exec == SPARBIT_EXEC_MIRROR ? 1u : (uint64_t)make_seq(p, first, last).count();
     return SPARBIT_OK;
 }
 
@@ -725,6 +766,47 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     CU(cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), block,
                                    rs.copy == SPARBIT_COPY_BULK ? args_bulk : args_vec, smem, st));
     p->bar_base += (unsigned)(last_idx - first_idx) * ctl.expected;  // one barrier between consecutive passes
+    p->kernel_launches++;
+    return SPARBIT_OK;
+}
+
+// The whole collective in one CTA with the receive buffers mirrored in shared memory.
+int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+    const uint32_t P = p->sched.P;
+    const ExecSeq seq = make_seq(p, first, last);
+    MirrorArgs ma;
+    memset(&ma, 0, sizeof ma);
+    ma.n = seq.count();
+    uint64_t most = 1;  // vectors of the largest pass
+    for (int i = 0; i < ma.n; i++) {
+        ma.d[i] = seq.item(i);
+        const uint64_t v = (uint64_t)P * ma.d[i].copies * (ma.d[i].copy_bytes / (uint64_t)rs.vbytes);
+        if (v > most) most = v;
+    }
+    // four vectors per thread and pass when there are that many, CTA sizes in steps of two warps
+    uint64_t threads = (most + 3) / 4;
+    threads = (threads + 63) / 64 * 64;
+    if (threads > 1024) threads = 1024;
+    const size_t smem = (size_t)P * P * p->sched.m;
+    const void* fn = pick_mirror_vec(rs.vbytes);
+    if (smem > p->mirror_smem_set[rs.vbytes]) {
+        CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        p->mirror_smem_set[rs.vbytes] = smem;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    Geom gg = g;
+    void* args[] = {&gg, &ma};
+    CU(cudaLaunchKernelExC(&cfg, fn, args));
     p->kernel_launches++;
     return SPARBIT_OK;
 }
@@ -850,6 +932,7 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
         case SPARBIT_EXEC_PERSISTENT: rc = launch_persistent(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_GRAPH: rc = launch_graph(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_FLOW: rc = launch_flow(p, rs, g, first, last, st); break;
+        case SPARBIT_EXEC_MIRROR: rc = launch_graph(p, rs, g, first, last, st); break;  // a graph of one kernel
         default: rc = launch_stream(p, rs, g, first, last, st); break;
     }
     if (rc == SPARBIT_OK) {
@@ -869,7 +952,7 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
     if (!out) return SPARBIT_ERR_ARG;
     *out = nullptr;
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
-    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_FLOW) return SPARBIT_ERR_ARG;
+    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_MIRROR) return SPARBIT_ERR_ARG;
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
     int rc;
@@ -895,8 +978,9 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     if (P > 8192) return SPARBIT_ERR_LIMIT;  // the task lists are built copy by copy: P*(P-1) entries at least
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
     if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // rotated workspace: fixed sizes only
-    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_FLOW) return SPARBIT_ERR_ARG;
-    if (exec == SPARBIT_EXEC_FLOW) return SPARBIT_ERR_UNSUPPORTED;  // its units assume equal blocks
+    if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_MIRROR) return SPARBIT_ERR_ARG;
+    if (exec == SPARBIT_EXEC_FLOW || exec == SPARBIT_EXEC_MIRROR)
+        return SPARBIT_ERR_UNSUPPORTED;  // both lay their work out for equal blocks
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
     int rc;
@@ -976,7 +1060,7 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     p->exec_req = exec;
     if (exec == SPARBIT_EXEC_AUTO) {  // variable-size plans have no flow executor
         const int e = env_exec(SPARBIT_EXEC_AUTO);
-        if (e != SPARBIT_EXEC_FLOW) p->exec_req = e;
+        if (e != SPARBIT_EXEC_FLOW && e != SPARBIT_EXEC_MIRROR) p->exec_req = e;
     }
     p->copy_req = env_copy(SPARBIT_COPY_AUTO);
     *out = p;

@@ -19,7 +19,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 ALGOS = [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK, sp.ALGO_NEIGHBOR_EXCHANGE]
-EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_FLOW]
+EXECS = [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_STREAM, sp.EXEC_FLOW, sp.EXEC_MIRROR]
 COPIES = [sp.COPY_VECTOR, sp.COPY_BULK]
 G = si.GUARD_BYTES
 
@@ -163,11 +163,12 @@ def test_state_after_every_phase(dev, algo, P, exec_mode):
 
 # ---------------------------------------------------------------- brute force over P
 @pytest.mark.parametrize("exec_mode,m", [(sp.EXEC_PERSISTENT, 16), (sp.EXEC_FLOW, 512), (sp.EXEC_FLOW, 1040),
-                                         (sp.EXEC_FLOW, 16)])
+                                         (sp.EXEC_FLOW, 16), (sp.EXEC_MIRROR, 16), (sp.EXEC_MIRROR, 52)])
 def test_every_p_up_to_64(dev, exec_mode, m):
-    """Every communicator size, on both single-kernel executors.  The flow executor takes blocks
+    """Every communicator size, on the single-kernel executors.  The flow executor takes blocks
     of at least 32 vectors (512 B: one warp row; 1040 B: two ragged spans per block) and hands
-    smaller ones to the graph chain."""
+    smaller ones to the graph chain; the mirror executor takes what fits into one SM's shared
+    memory (all of these at 16 B, up to P = 64 at 52 B) and hands the rest to the graph chain."""
     for P in range(1, 65):
         run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=2 if m != 16 else 1)
 
@@ -185,7 +186,7 @@ def test_comparators_many_p(dev, algo):
 
 # ---------------------------------------------------------------- any block size, any alignment
 @pytest.mark.parametrize("m", [1, 2, 3, 6, 10, 20, 100, 1000, 4100, 16400])
-@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_FLOW])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_FLOW, sp.EXEC_MIRROR])
 def test_odd_block_sizes(dev, m, exec_mode):
     run_case(dev, 7, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 31 + m, iters=1)
 
@@ -287,6 +288,38 @@ def test_flow_all_algorithms_changing_data(dev, algo):
         run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 77 + P, iters=3)
 
 
+@pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_NEIGHBOR_EXCHANGE])
+def test_mirror_all_algorithms_changing_data(dev, algo):
+    """The mirror executor on every algorithm it takes, up to the largest receive space that
+    fits one SM's shared memory, at misaligned addresses too, with new data on every call."""
+    for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 65536), (1, 4096), (12, 100), (7, 4500)):
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
+            continue
+        run_case(dev, P, m, algo, sp.EXEC_MIRROR, sp.COPY_AUTO, 90 + P, iters=3)
+    run_case(dev, 9, 96, algo if algo != sp.ALGO_RECURSIVE_DOUBLING and algo != sp.ALGO_NEIGHBOR_EXCHANGE
+             else sp.ALGO_SPARBIT, sp.EXEC_MIRROR, sp.COPY_AUTO, 5, iters=1, shift_send=4, shift_recv=8)
+
+
+def test_mirror_runs_where_it_fits_and_hands_over_where_not(dev):
+    for P, m, want in ((8, 64, sp.EXEC_MIRROR), (6, 4096, sp.EXEC_MIRROR), (13, 4096, sp.EXEC_GRAPH),
+                       (64, 64, sp.EXEC_GRAPH), (20, 16, sp.EXEC_MIRROR)):
+        plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
+        send = torch.from_numpy(si.send_blocks(P, m, 1).reshape(-1)).to(dev)
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        plan.allgather(send, recv)
+        assert plan.status() == sp.OK and plan.exec_mode == want, (P, m)
+        assert all(torch.equal(recv.view(P, P * m)[r], send) for r in range(P))
+        plan.destroy()
+    # a ring of 20 ranks has 19 passes: more than the kernel's parameter table holds
+    plan = sp.Plan(20, 16, sp.ALGO_RING, sp.EXEC_MIRROR)
+    send = torch.from_numpy(si.send_blocks(20, 16, 1).reshape(-1)).to(dev)
+    recv = torch.full((20 * 20 * 16,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_GRAPH
+
+
 # ---------------------------------------------------------------- host-buffer entry point, streams, bookkeeping
 @pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_BRUCK])
 def test_host_entry_point(dev, algo):
@@ -319,6 +352,14 @@ def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
     phases = plan.num_steps  # the own-block copy and step 0 run as one fused pass
     if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_FLOW):
         assert (kernels, graphs) == (2, 0)
+    elif exec_mode == sp.EXEC_MIRROR:
+        assert (kernels, graphs) == (2 * phases, 2)     # 256 KiB of receive buffers: runs as a graph chain
+        exec_mode = sp.EXEC_GRAPH
+        small = sp.Plan(8, 64, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
+        small.allgather(send[: 8 * 64], recv, stream)
+        small.allgather(send[: 8 * 64], recv, stream)
+        assert small.status() == sp.OK and small.launch_counts() == (2, 2)   # one kernel in a cached graph
+        small.destroy()
     elif exec_mode == sp.EXEC_GRAPH:
         assert (kernels, graphs) == (2 * phases, 2)
     else:

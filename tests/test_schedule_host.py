@@ -134,7 +134,11 @@ def test_strerror_covers_every_code():
 
 
 def test_exec_mode_resolution():
-    assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH             # measured best at every size
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR            # 4 KiB of receive buffers: one CTA, on chip
+    assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
+    assert sp.Plan(32, 128).exec_mode == sp.EXEC_GRAPH           # 128 KiB: one CTA is too slow for it
+    assert sp.Plan(32, 128, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
+    assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_GRAPH
     assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH         # 8.6 GB moved: chain + bulk engine
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
@@ -162,7 +166,7 @@ def test_environment_overrides_only_the_automatic_choice(monkeypatch):
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_FLOW
     assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_GRAPH                  # not offered there
     monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
-    assert sp.Plan(8, 64).exec_mode == sp.EXEC_GRAPH
+    assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR
 
 
 @pytest.mark.parametrize("algo", ALGOS)
