@@ -249,7 +249,7 @@ def run_ours(args):
     algo = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
             "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}[args.algo]
     exec_mode = {"auto": sp.EXEC_AUTO, "persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH,
-                 "stream": sp.EXEC_STREAM, "flow": sp.EXEC_FLOW}[args.exec]
+                 "stream": sp.EXEC_STREAM, "flow": sp.EXEC_FLOW, "mirror": sp.EXEC_MIRROR}[args.exec]
     copy = {"auto": sp.COPY_AUTO, "vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}[args.copy]
 
     plan = sp.Plan(P, m, algo, exec_mode)
@@ -294,6 +294,9 @@ def run_ours(args):
             time.sleep(0.25)
         k0, g0 = plan.launch_counts()
         round_ms, per_ms = [], []
+        # a time stamp between every two collectives costs about 2 us of GPU time: taken only where
+        # a collective is long enough not to notice (else min/avg/max are over the rounds)
+        stamp_each = est_ms / args.steps >= 0.1
         t_wall0 = time.time()
         for _ in range(rounds):
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
@@ -301,11 +304,13 @@ def run_ours(args):
             ev[0].record(stream)
             for it in range(args.steps):
                 plan.allgather(sends[it & 1], recv, stream)
-                ev[it + 1].record(stream)
+                if stamp_each or it == args.steps - 1:
+                    ev[it + 1].record(stream)
             stream.synchronize()
             barrier()
             round_ms.append(max_over_ranks(ev[0].elapsed_time(ev[-1]), dev, use_dist))
-            per_ms += [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+            per_ms += ([ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)] if stamp_each
+                       else [ev[0].elapsed_time(ev[-1]) / args.steps])
         t_wall1 = time.time()
         k1, g1 = plan.launch_counts()
     assert plan.status() == sp.OK
@@ -457,8 +462,9 @@ def run_cpu_sweep(args):
 
 
 def run_sweep(args):
-    """Latency and bandwidth curves: every point timed with the paper's protocol (5 warm-ups, 50
-    timed collectives, min / avg / max), one JSON line per (algorithm, executor, engine, P, m)."""
+    """Latency and bandwidth curves: every point timed with the paper's protocol (5 warm-ups, then
+    batches of 50 timed collectives; min / avg / max over ten batches), one JSON line per
+    (algorithm, executor, engine, P, m)."""
     import torch
     import paper_2109_08751_b200 as sp
 
@@ -475,10 +481,16 @@ def run_sweep(args):
         points += [(128, 65536, ["sparbit"])]
     if args.sweep == "small":  # configs 1 and 2 and their neighbourhood: latency only
         points += [(P, m, ["sparbit"]) for P in (6, 8, 13, 16, 32, 64) for m in (64, 4096)]
+    if args.sweep == "engines":  # what the engine and executor thresholds rest on
+        points += [(P, m, ["sparbit"]) for P in (61, 128, 256, 509) for m in (4096, 8192, 16384, 32768, 65536)
+                   if P * P * m <= (20 << 30)]
+        points += [(1000, 1024, ["sparbit"]), (700, 1024, ["sparbit"]), (360, 8192, ["sparbit"])]
     algos = {"sparbit": sp.ALGO_SPARBIT, "ring": sp.ALGO_RING, "rd": sp.ALGO_RECURSIVE_DOUBLING,
              "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}
     execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
-             "flow": sp.EXEC_FLOW}
+             "flow": sp.EXEC_FLOW, "mirror": sp.EXEC_MIRROR}
+    if args.sweep == "engines":
+        execs = {"graph": sp.EXEC_GRAPH, "flow": sp.EXEC_FLOW}
     copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
     stream = torch.cuda.Stream(device=dev)
     cores = min(os.cpu_count() or 1, 16)
@@ -501,31 +513,39 @@ def run_sweep(args):
             for ename, e, cname, c in combos:
                 if ename == "stream" and name in ("ring", "ne") and m >= 32768:
                     continue  # same kernels as the graph chain; skipped to bound the sweep
-                if cname == "bulk" and (m % 16 or ename == "flow"):
+                if cname == "bulk" and (m % 16 or ename in ("flow", "mirror")):
+                    continue
+                if ename == "mirror" and P * P * m > (224 << 10):
                     continue
                 plan = sp.Plan(P, m, algos[name], e)
                 plan.set_copy_path(c)
                 if name == "bruck":
                     plan.set_workspace(work, P * P * m)
+                # the paper's protocol (5 warm-ups, 50 timed runs), the way its benchmark times them:
+                # a batch of 50 back-to-back collectives between two time stamps, divided by 50
+                # (a time stamp between every two collectives would itself cost 2 us each); ten
+                # such batches give the minimum, average and maximum
+                us = []
                 with torch.cuda.stream(stream):
                     for it in range(5):
                         plan.allgather(sends[it & 1], recv, stream)
                     stream.synchronize()
-                    ev = [torch.cuda.Event(enable_timing=True) for _ in range(51)]
                     k_before = plan.launch_counts()[0]
-                    ev[0].record(stream)
-                    for it in range(50):
-                        plan.allgather(sends[it & 1], recv, stream)
-                        ev[it + 1].record(stream)
-                    stream.synchronize()
+                    for _ in range(10):
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record(stream)
+                        for it in range(50):
+                            plan.allgather(sends[it & 1], recv, stream)
+                        e1.record(stream)
+                        stream.synchronize()
+                        us.append(e0.elapsed_time(e1) / 50 * 1e3)
                 assert plan.status() == sp.OK
                 ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
-                us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(50)]
                 avg = float(np.mean(us))
                 print(json.dumps({
                     "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
                     "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
-                    "launches_per_collective": (plan.launch_counts()[0] - k_before) / 50,
+                    "launches_per_collective": (plan.launch_counts()[0] - k_before) / 500,
                     "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
                     "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
                     "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
@@ -690,7 +710,7 @@ def main():
     ap.add_argument("--P", type=int, default=P_DEFAULT)
     ap.add_argument("--m", type=int, default=M_DEFAULT)
     ap.add_argument("--algo", choices=["sparbit", "ring", "ne", "rd", "bruck"], default="sparbit")
-    ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "flow"], default="auto")
+    ap.add_argument("--exec", choices=["auto", "persistent", "graph", "stream", "flow", "mirror"], default="auto")
     ap.add_argument("--copy", choices=["auto", "vector", "bulk"], default="auto")
     ap.add_argument("--seed", type=int, default=si.BASE_SEED + 5)
     ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
@@ -698,7 +718,7 @@ def main():
                          "(0 = one round, for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "all"], default=None,
+    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     ap.add_argument("--sweep-auto-only", action="store_true",
                     help="with --sweep: only the executor and engine the library picks by itself")

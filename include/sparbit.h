@@ -85,9 +85,11 @@ enum {
     SPARBIT_EXEC_FLOW = 4,       /* one cooperative kernel without grid barriers: Algorithm 1's
                                     Waitall is kept per rank (counters of what each rank has
                                     received), so a pass starts where its senders are ready while
-                                    the pass before is still finishing elsewhere.  Whole
-                                    collectives of fixed-size blocks of at least 32 vectors on the
-                                    vector engine; other calls run as GRAPH */
+                                    the pass before is still finishing elsewhere.  Leading passes
+                                    too small to keep every warp busy run as chained per-pass
+                                    kernels in front of it.  Whole collectives of fixed-size
+                                    blocks of at least 32 vectors on the vector engine; other
+                                    calls run as GRAPH */
     SPARBIT_EXEC_MIRROR = 5      /* a whole small collective in ONE CTA: every block written to a
                                     receive buffer is also kept in an on-chip copy of the receive
                                     buffers (shared memory), and every forwarded block is read from
@@ -283,11 +285,15 @@ int sparbit_plan_partition_messages(const sparbit_plan_t* plan, int G, int mappi
  * resident_warps warps, the work units of every pass, decoded the way the kernel decodes them,
  * must cover each rank's copies exactly once; the units that write into a rank's buffer must
  * number what the counter of that (rank, pass) is compared with; and a pass must wait for every
- * earlier pass that writes the space it reads.  SPARBIT_OK, SPARBIT_ERR_ARG with the offending
- * pass in *bad_pass (may be NULL), SPARBIT_ERR_UNSUPPORTED if the plan cannot run on FLOW with
- * that vector width, SPARBIT_ERR_LIMIT for more than 2^26 spans in a pass.  Host-only.
+ * earlier pass of the kernel that writes the space it reads.  *first_flow_pass (may be NULL)
+ * receives the position, in the executed sequence of passes, of the first pass the flow kernel
+ * takes (the ones before it run as per-pass kernels).  SPARBIT_OK, SPARBIT_ERR_ARG with the
+ * offending pass in *bad_pass (may be NULL), SPARBIT_ERR_UNSUPPORTED if no pass of the plan can
+ * run in the flow kernel with that vector width and warp count, SPARBIT_ERR_LIMIT for more than
+ * 2^26 spans in a pass.  Host-only.
  */
-int sparbit_plan_validate_flow(const sparbit_plan_t* plan, int vector_bytes, int resident_warps, int* bad_pass);
+int sparbit_plan_validate_flow(const sparbit_plan_t* plan, int vector_bytes, int resident_warps,
+                               int* first_flow_pass, int* bad_pass);
 
 /* Bytes of workspace the plan needs: 0, or P*P*m for Bruck. */
 size_t sparbit_plan_workspace_bytes(const sparbit_plan_t* plan);
@@ -313,7 +319,12 @@ enum {
     SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (10^9) */
     SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES = 5, /* ... and below this (6*10^9); GRAPH otherwise */
     SPARBIT_TUNE_MIRROR_MAX_BYTES = 6,     /* EXEC_AUTO: MIRROR when P*P*m is at most this (64 KiB) */
-    SPARBIT_TUNE_COUNT_ = 7
+    SPARBIT_TUNE_FLOW_MIN_PASS_SPANS = 7,  /* EXEC_FLOW: the flow kernel takes the passes at the end of
+                                              the collective that have at least this many 1 KiB warp
+                                              spans in all (0, the default: one per resident warp,
+                                              4736 on B200; 1: every pass); smaller leading passes run
+                                              as chained per-pass kernels in front of it */
+    SPARBIT_TUNE_COUNT_ = 8
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

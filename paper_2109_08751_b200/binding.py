@@ -21,7 +21,8 @@ COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
 SPACE_SEND, SPACE_RECV, SPACE_WORKSPACE = range(3)
 MAP_SEQUENTIAL, MAP_CYCLIC = range(2)
 (TUNE_BULK_MIN_BLOCK_BYTES, TUNE_BULK_MIN_MOVED_BYTES, TUNE_FLOW_UNITS_PER_WARP, TUNE_FLOW_MAX_UNIT_SPANS,
- TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES, TUNE_MIRROR_MAX_BYTES) = range(7)
+ TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES, TUNE_MIRROR_MAX_BYTES,
+ TUNE_FLOW_MIN_PASS_SPANS) = range(8)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
               ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}
@@ -48,7 +49,7 @@ SYMBOLS = {
     "sparbit_plan_step_info": (_i, [_vp, _i, _pi, _pi, _pi]),
     "sparbit_plan_messages": (_i, [_vp, _i, _vp, _sz, ctypes.POINTER(_sz)]),
     "sparbit_plan_validate": (_i, [_vp, _pi]),
-    "sparbit_plan_validate_flow": (_i, [_vp, _i, _i, _pi]),
+    "sparbit_plan_validate_flow": (_i, [_vp, _i, _i, _pi, _pi]),
     "sparbit_rank_device": (_i, [_i, _i, _i, _i]),
     "sparbit_plan_partition": (_i, [_vp, _i, _i, _i, ctypes.POINTER(_u64)]),
     "sparbit_plan_partition_messages": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _sz, ctypes.POINTER(_sz)]),
@@ -203,10 +204,12 @@ class Plan:
     def validate_flow(self, vector_bytes: int = 16, resident_warps: int = 4736) -> int:
         """Host-side check of the flow executor's units and counters; returns the library's code
         (OK, or ERR_UNSUPPORTED when the plan cannot run on that executor) and raises on a fault."""
-        bad = ctypes.c_int()
-        code = lib.sparbit_plan_validate_flow(self._h, vector_bytes, resident_warps, ctypes.byref(bad))
+        bad, first = ctypes.c_int(), ctypes.c_int()
+        code = lib.sparbit_plan_validate_flow(self._h, vector_bytes, resident_warps, ctypes.byref(first),
+                                              ctypes.byref(bad))
         if code not in (OK, ERR_UNSUPPORTED):
             raise SparbitError(code, f"sparbit_plan_validate_flow (pass {bad.value})")
+        self.first_flow_pass = first.value
         return code
 
     @property

@@ -110,6 +110,7 @@ struct sparbit_plan_s {
         1000000000u,  // FLOW_MIN_MOVED_BYTES
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
+        0,            // FLOW_MIN_PASS_SPANS (0: one span per resident warp)
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -391,19 +392,38 @@ bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_l
     return bytes <= (unsigned __int128)smem_limit;
 }
 
-bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, bool assume_coop = false) {
-    if (p->variable || !(p->coop || assume_coop)) return false;
-    if (first != -1 || last != p->sched.last_phase()) return false;
-    const ExecSeq seq = make_seq(p, first, last);
-    if (seq.count() < 1 || seq.count() > kFlowMaxPasses) return false;
-    for (int i = 0; i < seq.count(); i++) {
+// Which passes of a call the flow kernel takes: the longest run of passes at the END of the
+// executed sequence that it can take (fixed-size blocks of at least 32 vectors, at most
+// kFlowMaxPasses of them) and that are large enough to keep every one of `max_warps` warps busy
+// (FLOW_MIN_PASS_SPANS warp spans in all, by default one per warp): below that a pass is bound by latency, and there a
+// kernel boundary is cheaper than a counter hand-off.  The passes before run as chained per-pass
+// kernels.  Returns the position of the first flow pass, or the sequence length if there is none.
+int flow_first_pass(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint64_t max_warps) {
+    const int n = seq.count();
+    int f = n;
+    for (int i = n - 1; i >= 0 && n - i <= kFlowMaxPasses; i--) {
         const PhaseDesc& d = seq.item(i);
         const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
-        if (vpc < 32) return false;
+        if (vpc < 32) break;
         const uint64_t spc = (vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll);
-        if (((uint64_t)p->sched.P * d.copies * spc) >> 31) return false;
+        const uint64_t spans = (uint64_t)p->sched.P * d.copies * spc;
+        if (spans >> 31) break;
+        const uint64_t least = p->tune[SPARBIT_TUNE_FLOW_MIN_PASS_SPANS] ? p->tune[SPARBIT_TUNE_FLOW_MIN_PASS_SPANS] : max_warps;
+        if (spans < least) break;
+        f = i;
     }
-    return true;
+    return f;
+}
+
+constexpr uint64_t kFlowWarpsB200 = 148 * 2 * 16;  // resident warps of the flow kernel on a B200
+
+bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, bool assume_b200 = false) {
+    if (p->variable || !(p->coop || assume_b200)) return false;
+    if (first != -1 || last != p->sched.last_phase()) return false;
+    const ExecSeq seq = make_seq(p, first, last);
+    if (seq.count() < 1) return false;
+    const uint64_t warps = assume_b200 || !p->sm_count ? kFlowWarpsB200 : (uint64_t)p->sm_count * 2 * (kVecBlock / 32);
+    return flow_first_pass(p, seq, vbytes, warps) < seq.count();
 }
 
 // Executor for SPARBIT_EXEC_AUTO, from measurements on B200.
@@ -579,9 +599,11 @@ struct PhaseArgs {
 // (griddepcontrol.launch_dependents) and itself waits for its predecessor to complete and flush
 // (griddepcontrol.wait) before it touches memory, so the launch latency of phase i+1 hides behind
 // phase i while the Waitall between phases stays intact.
-int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
+int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st,
+                  int seq_end = -1) {
     const ExecSeq seq = make_seq(p, first, last);
-    for (int i = 0; i < seq.count(); i++) {
+    const int end = seq_end < 0 ? seq.count() : seq_end;  // only the first seq_end passes, if given
+    for (int i = 0; i < end; i++) {
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
         cfg.stream = st;
@@ -815,15 +837,15 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
 // enumeration starts, which earlier passes a unit has to wait for, and the counter value that
 // says "all units of this launch that write into this rank in this pass are done".  Returns the
 // unit count of the largest pass.
-uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint64_t max_warps, unsigned epoch,
-                         bool never_reached, FlowArgs& fa) {
+uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int f, int vbytes, uint64_t max_warps,
+                         unsigned epoch, bool never_reached, FlowArgs& fa) {
     const uint32_t P = p->sched.P;
-    const int n = seq.count();
+    const int n = seq.count() - f;  // the kernel's passes: positions f.. of the sequence
     fa.n = (uint32_t)n;
     uint64_t most_units = 1;
     uint32_t rot = 0;
     for (int i = 0; i < n; i++) {
-        const PhaseDesc& d = seq.item(i);
+        const PhaseDesc& d = seq.item(f + i);
         FlowPass& fp = fa.pass[i];
         const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
         fp.spc = (uint32_t)((vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll));
@@ -843,9 +865,9 @@ uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes
         // fused first pass its own as well
         const uint32_t per_rank = fp.upr * (d.dup_self ? 2u : 1u);
         fp.target = epoch * per_rank + (never_reached ? 1u : 0u);  // test hook: a target that is never reached
-        fp.dep_mask = 0;
+        fp.dep_mask = 0;  // passes before f are complete when the kernel starts (stream order)
         for (int k = 0; k < i; k++)
-            if (seq.item(k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
+            if (seq.item(f + k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
         if ((uint64_t)P * fp.upr > most_units) most_units = (uint64_t)P * fp.upr;
         fp.eager = (uint64_t)P * fp.upr <= max_warps ? 1u : 0u;
         // the next pass starts its enumeration where this pass's first receivers are
@@ -854,11 +876,23 @@ uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes
     return most_units;
 }
 
-// The whole collective as one cooperative kernel without grid barriers (flow_vec_kernel).
+// The collective's small leading passes as chained per-pass kernels, all the others in one
+// cooperative kernel without grid barriers (flow_vec_kernel).
 int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
-    const int n = seq.count();
+    const void* fn = pick_flow_vec(rs.vbytes);
+    int per_sm = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kVecBlock, 0));
+    if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "flow kernel does not fit on an SM");
+    if (per_sm > 2) per_sm = 2;
+    const uint64_t max_warps = (uint64_t)per_sm * p->sm_count * (kVecBlock / 32);
+    const int f = flow_first_pass(p, seq, rs.vbytes, max_warps);
+    if (f >= seq.count()) return launch_stream(p, rs, g, first, last, st);  // (resolve() rules this out)
+    if (f > 0) {
+        int rc = launch_stream(p, rs, g, first, last, st, f);
+        if (rc) return rc;
+    }
     if (!p->d_flow_cnt) {
         CU(cudaMalloc((void**)&p->d_flow_cnt, (size_t)P * kFlowMaxPasses * sizeof(unsigned)));
         p->flow_epoch = 0;
@@ -866,6 +900,7 @@ int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first,
     }
     if (p->flow_vbytes != rs.vbytes || p->flow_epoch == 0) {
         // counters count units, and a unit's size follows the vector width: start over
+        // (with leading per-pass kernels in front this memset sits between kernels: rare, and correct)
         CU(cudaMemsetAsync(p->d_flow_cnt, 0, (size_t)P * kFlowMaxPasses * sizeof(unsigned), st));
         p->flow_epoch = 0;
         p->flow_vbytes = rs.vbytes;
@@ -873,23 +908,17 @@ int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first,
     p->flow_epoch++;
     FlowArgs fa;
     memset(&fa, 0, sizeof fa);
-    fa.n = (uint32_t)n;
     fa.cnt = p->d_flow_cnt;
     fa.status = p->d_ctl + 1;
     fa.timeout_ns = p->timeout_ns;
-    const void* fn = pick_flow_vec(rs.vbytes);
-    int per_sm = 0;
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kVecBlock, 0));
-    if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "flow kernel does not fit on an SM");
-    if (per_sm > 2) per_sm = 2;
-    const uint64_t max_warps = (uint64_t)per_sm * p->sm_count * (kVecBlock / 32);
-    const uint64_t most_units = flow_pass_table(p, seq, rs.vbytes, max_warps, p->flow_epoch, p->extra_arrivals != 0, fa);
+    const uint64_t most_units =
+        flow_pass_table(p, seq, f, rs.vbytes, max_warps, p->flow_epoch, p->extra_arrivals != 0, fa);
     uint64_t grid = (uint64_t)per_sm * p->sm_count;
     const uint64_t need = (most_units + kVecBlock / 32 - 1) / (kVecBlock / 32);
     if (grid > need) grid = need;
     Geom gg = g;
     const PhaseDesc* descs = p->d_descs;
-    int first_idx = (int)seq.table_index(0);
+    int first_idx = (int)seq.table_index(f);
     void* args[] = {&gg, &descs, &first_idx, &fa};
     // cooperative (all CTAs resident: the waits inside depend on it) and, like the per-pass kernels,
     // launched ahead behind its predecessor in the stream
@@ -1381,21 +1410,27 @@ int sparbit_plan_validate(const sparbit_plan_t* p, int* bad_phase) {
 // every span of every rank's copies once; the number of units that write into a rank's buffer
 // (through either destination of the fused pass) must be the counter target of that pass; and a
 // pass must wait for every earlier pass that writes the space it reads.
-int sparbit_plan_validate_flow(const sparbit_plan_t* p, int vector_bytes, int resident_warps, int* bad_pass) {
+int sparbit_plan_validate_flow(const sparbit_plan_t* p, int vector_bytes, int resident_warps, int* first_flow_pass,
+                               int* bad_pass) {
     if (!p || resident_warps < 1) return SPARBIT_ERR_ARG;
+    if (first_flow_pass) *first_flow_pass = -1;
     if (vector_bytes != 1 && vector_bytes != 2 && vector_bytes != 4 && vector_bytes != 8 && vector_bytes != 16)
         return SPARBIT_ERR_ARG;
     if (bad_pass) *bad_pass = -1;
-    if (!flow_possible(p, vector_bytes, -1, p->sched.last_phase(), true)) return SPARBIT_ERR_UNSUPPORTED;
+    if (p->variable) return SPARBIT_ERR_UNSUPPORTED;
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, -1, p->sched.last_phase());
+    if (seq.count() < 1) return SPARBIT_ERR_UNSUPPORTED;
     try {
         FlowArgs fa;
         memset(&fa, 0, sizeof fa);
         const unsigned epoch = 3;
-        flow_pass_table(p, seq, vector_bytes, (uint64_t)resident_warps, epoch, false, fa);
-        for (int i = 0; i < seq.count(); i++) {
-            const PhaseDesc& d = seq.item(i);
+        const int f = flow_first_pass(p, seq, vector_bytes, (uint64_t)resident_warps);
+        if (f >= seq.count()) return SPARBIT_ERR_UNSUPPORTED;
+        flow_pass_table(p, seq, f, vector_bytes, (uint64_t)resident_warps, epoch, false, fa);
+        if (first_flow_pass) *first_flow_pass = f;
+        for (int i = 0; i < seq.count() - f; i++) {
+            const PhaseDesc& d = seq.item(f + i);
             const FlowPass& fp = fa.pass[i];
             auto fail = [&]() {
                 if (bad_pass) *bad_pass = i;
@@ -1431,7 +1466,7 @@ int sparbit_plan_validate_flow(const sparbit_plan_t* p, int vector_bytes, int re
                 if (arrivals[q] * epoch != fp.target) return fail();
             uint32_t want_mask = 0;
             for (int k = 0; k < i; k++)
-                if (seq.item(k).dst_space == d.src_space) want_mask |= 1u << k;
+                if (seq.item(f + k).dst_space == d.src_space) want_mask |= 1u << k;
             if (fp.dep_mask != want_mask || (d.src_space == SPACE_SEND && fp.dep_mask)) return fail();
         }
     } catch (const std::bad_alloc&) {

@@ -60,9 +60,12 @@ class Guarded:
         self.raw.fill_(self.fill)
 
 
-def run_case(dev, P, m, algo, exec_mode, copy, seed, iters=2, shift_send=0, shift_recv=0, shift_work=0):
+def run_case(dev, P, m, algo, exec_mode, copy, seed, iters=2, shift_send=0, shift_recv=0, shift_work=0, tune=None,
+             ran=None):
     plan = sp.Plan(P, m, algo, exec_mode)
     plan.set_copy_path(copy)
+    for key, value in (tune or {}).items():
+        plan.set_tunable(key, value)
     send = Guarded(P * m, dev, shift_send, fill=0x3C)
     recv = Guarded(P * P * m, dev, shift_recv)
     work = None
@@ -88,6 +91,8 @@ def run_case(dev, P, m, algo, exec_mode, copy, seed, iters=2, shift_send=0, shif
         if work:
             assert work.guards_intact()
             assert np.array_equal(work.view.cpu().numpy(), scratch)
+    if ran is not None:
+        assert plan.exec_mode == ran, (P, m, algo, plan.exec_mode)
     plan.destroy()
 
 
@@ -162,15 +167,25 @@ def test_state_after_every_phase(dev, algo, P, exec_mode):
 
 
 # ---------------------------------------------------------------- brute force over P
-@pytest.mark.parametrize("exec_mode,m", [(sp.EXEC_PERSISTENT, 16), (sp.EXEC_FLOW, 512), (sp.EXEC_FLOW, 1040),
-                                         (sp.EXEC_FLOW, 16), (sp.EXEC_MIRROR, 16), (sp.EXEC_MIRROR, 52)])
-def test_every_p_up_to_64(dev, exec_mode, m):
+ALL_IN_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 1}     # every pass in the flow kernel
+SPLIT_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 40}     # passes of fewer than 40 spans as kernels in front of it
+
+
+@pytest.mark.parametrize("exec_mode,m,tune", [(sp.EXEC_PERSISTENT, 16, None), (sp.EXEC_FLOW, 512, ALL_IN_FLOW),
+                                              (sp.EXEC_FLOW, 1040, ALL_IN_FLOW), (sp.EXEC_FLOW, 1040, SPLIT_FLOW),
+                                              (sp.EXEC_FLOW, 16, None), (sp.EXEC_MIRROR, 16, None),
+                                              (sp.EXEC_MIRROR, 52, None)])
+def test_every_p_up_to_64(dev, exec_mode, m, tune):
     """Every communicator size, on the single-kernel executors.  The flow executor takes blocks
     of at least 32 vectors (512 B: one warp row; 1040 B: two ragged spans per block) and hands
-    smaller ones to the graph chain; the mirror executor takes what fits into one SM's shared
+    smaller ones to the graph chain, and by default leaves passes that cannot keep every warp busy
+    to per-pass kernels in front of it: the tests set that threshold so that the kernel takes
+    every pass, or only those of at least 40 spans; the mirror executor takes what fits into one SM's shared
     memory (all of these at 16 B, up to P = 64 at 52 B) and hands the rest to the graph chain."""
     for P in range(1, 65):
-        run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=2 if m != 16 else 1)
+        ran = sp.EXEC_FLOW if tune is ALL_IN_FLOW else None
+        run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=2 if m != 16 else 1, tune=tune,
+                 ran=ran)
 
 
 @pytest.mark.parametrize("algo", [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_BRUCK,
@@ -188,7 +203,8 @@ def test_comparators_many_p(dev, algo):
 @pytest.mark.parametrize("m", [1, 2, 3, 6, 10, 20, 100, 1000, 4100, 16400])
 @pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_GRAPH, sp.EXEC_FLOW, sp.EXEC_MIRROR])
 def test_odd_block_sizes(dev, m, exec_mode):
-    run_case(dev, 7, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 31 + m, iters=1)
+    run_case(dev, 7, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 31 + m, iters=1,
+             tune=ALL_IN_FLOW if exec_mode == sp.EXEC_FLOW else None)
 
 
 @pytest.mark.parametrize("shifts", [(1, 0, 0), (0, 1, 0), (2, 2, 2), (4, 8, 4), (8, 8, 8), (3, 5, 7), (16, 32, 48)])
@@ -256,6 +272,7 @@ def test_flow_wait_gives_up_instead_of_hanging(dev):
     the plan must work again afterwards, its counters cleared."""
     P, m = 16, 4096
     plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_FLOW)
+    plan.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 1)
     host_send = si.send_blocks(P, m, 1)
     send = torch.from_numpy(host_send.reshape(-1)).to(dev)
     recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
@@ -285,7 +302,8 @@ def test_flow_all_algorithms_changing_data(dev, algo):
             continue
         if algo == sp.ALGO_RING and P > 32:
             continue   # more passes than the flow executor's counter line holds: runs as a graph
-        run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 77 + P, iters=3)
+        run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 77 + P, iters=3, tune=ALL_IN_FLOW, ran=sp.EXEC_FLOW)
+        run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 78 + P, iters=2, tune=SPLIT_FLOW)
 
 
 @pytest.mark.parametrize("algo", [sp.ALGO_SPARBIT, sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING, sp.ALGO_NEIGHBOR_EXCHANGE])
@@ -337,6 +355,7 @@ def test_host_entry_point(dev, algo):
 def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
     P, m = 16, 1024
     plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    plan.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 1)   # the flow kernel takes every pass
     host_send = si.send_blocks(P, m, 3)
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):

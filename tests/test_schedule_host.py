@@ -189,7 +189,10 @@ def test_descriptors_are_race_free_and_in_bounds(algo):
 @pytest.mark.parametrize("algo", ALGOS)
 def test_flow_units_and_counters_are_consistent(algo):
     """The flow executor's bookkeeping, checked on the host for many communicator sizes, block
-    sizes (one span, ragged spans, many spans per block), vector widths and numbers of warps."""
+    sizes (one span, ragged spans, many spans per block), vector widths and numbers of warps.
+    With one warp every pass is large enough for the flow kernel (it then takes the whole
+    collective, or its last 32 passes); with more warps the small leading passes are left to
+    per-pass kernels, more of them the more warps there are."""
     ran = 0
     for P in list(range(1, 34)) + [61, 64, 100, 128, 253, 256, 1000]:
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
@@ -200,14 +203,18 @@ def test_flow_units_and_counters_are_consistent(algo):
             if P > 256 and m > 4096:
                 continue
             plan = sp.Plan(P, m, algo)
-            for warps in (1, 64, 4736):
+            passes = plan.last_phase + 2 - (1 if algo != sp.ALGO_BRUCK and P > 1 else 0)   # fused first pass
+            firsts = []
+            for warps in (1, 64, 4736):   # by default a pass needs one span per resident warp
                 code = plan.validate_flow(vb, warps)
                 assert code in (sp.OK, sp.ERR_UNSUPPORTED)
-                # the only things this executor cannot take: more passes than a counter line holds
-                if code == sp.ERR_UNSUPPORTED:
-                    assert plan.last_phase + 2 > 32
-                else:
-                    ran += 1
+                if warps == 1:
+                    assert code == sp.OK and plan.first_flow_pass == max(0, passes - 32), (algo, P, m)
+                firsts.append(plan.first_flow_pass if code == sp.OK else passes)
+                ran += code == sp.OK
+            assert firsts == sorted(firsts), (algo, P, m, firsts)
             plan.destroy()
-    assert ran > 100
-    assert sp.Plan(8, 64).validate_flow(16) == sp.ERR_UNSUPPORTED   # blocks shorter than a warp row
+    assert ran > 60
+    assert sp.Plan(8, 64).validate_flow(16, 1) == sp.ERR_UNSUPPORTED   # blocks shorter than a warp row
+    big = sp.Plan(256, 4096)
+    assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 3   # 8192 spans in pass 3
