@@ -46,6 +46,18 @@ NCU_TRAFFIC = {
     "sparbit:P256:m65536:persistent:bulk": (8.41e9, "profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md"),
     # phase_bulk_kernel, last phase: 2.15 GB read + 2.10 GB written
     "sparbit:P256:m65536:graph:bulk": (4.25e9, "profiles/phase_bulk_kernel_last_phase_P256_m64k_traffic.md"),
+    # config 3: flow_vec_kernel, whole collective; last pass of the per-pass kernels of either engine
+    "sparbit:P128:m65536:flow:vector": (1.997e9, "profiles/phase_kernels_and_flow_kernel_P128_m64k.md"),
+    "sparbit:P128:m65536:graph:bulk": (1.026e9, "profiles/phase_kernels_and_flow_kernel_P128_m64k.md"),
+    "sparbit:P128:m65536:graph:vector": (1.029e9, "profiles/phase_kernels_and_flow_kernel_P128_m64k.md"),
+    # config 4: flow_vec_kernel, whole collective; last pass of phase_vec_kernel
+    "sparbit:P1000:m1024:flow:vector": (1.89e9, "profiles/phase_vec_and_flow_kernel_P1000_m1k.md"),
+    "sparbit:P1000:m1024:graph:vector": (9.79e8, "profiles/phase_vec_and_flow_kernel_P1000_m1k.md"),
+    # config 5, small blocks: last pass of phase_vec_kernel (captured alone, caches cold)
+    "sparbit:P256:m4096:graph:vector": (2.24e8, "profiles/phase_vec_kernel_P256_small_blocks.md"),
+    "sparbit:P256:m512:graph:vector": (1.68e7, "profiles/phase_vec_kernel_P256_small_blocks.md"),
+    "sparbit:P256:m64:graph:vector": (4.21e6, "profiles/phase_vec_kernel_P256_small_blocks.md"),
+    "sparbit:P256:m8:graph:vector": (5.36e5, "profiles/phase_vec_kernel_P256_small_blocks.md"),
 }
 MIN_TIMED_MS = 250.0   # the timed rounds together last at least this long, whatever --steps is
 
@@ -315,6 +327,7 @@ def run_ours(args):
         k1, g1 = plan.launch_counts()
     assert plan.status() == sp.OK
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ran_exec, ran_copy = plan.exec_mode, plan.copy_path   # what the timed collectives ran on
 
     # the last collective's result, checked against the result's definition on the device
     last_send = sends[(args.steps - 1) & 1]
@@ -351,9 +364,11 @@ def run_ours(args):
     # kernel (persistent, flow), else the last schedule step (half of all bytes for a power of
     # two P), launched exactly as inside the collective and timed with events on the same stream
     launches_per_step = (k1 - k0) / (args.steps * rounds)
-    one_kernel = launches_per_step <= 1
+    # the flow executor's kernel cannot be launched apart from the small per-pass kernels it may
+    # have in front of it: its entry is the whole collective as well
+    one_kernel = launches_per_step <= 1 or ran_exec == sp.EXEC_FLOW
     per_pass_us = None
-    if one_kernel and plan.exec_mode == sp.EXEC_PERSISTENT:
+    if one_kernel and ran_exec == sp.EXEC_PERSISTENT:
         # one more, traced, launch: the persistent kernel's own time stamps, pass by pass
         plan.set_trace(True)
         plan.allgather(sends[0], recv, stream)
@@ -364,7 +379,8 @@ def run_ours(args):
     if one_kernel:
         dom_ms = float(np.mean(per_ms))
         dom_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
-        dom_name = "whole collective in one kernel"
+        dom_name = ("whole collective in one kernel" if launches_per_step <= 1 else
+                    f"whole collective: the flow kernel behind {launches_per_step - 1:g} small per-pass kernel(s)")
     else:
         last = plan.last_phase
         with torch.cuda.stream(stream):
@@ -386,12 +402,12 @@ def run_ours(args):
         avg_ms = float(np.mean(per_ms))
         path_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-        key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[plan.exec_mode]}:{sp.COPY_NAMES[plan.copy_path]}"
+        key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[ran_exec]}:{sp.COPY_NAMES[ran_copy]}"
         roofline = {
             "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
             "traffic": NCU_TRAFFIC.get(key, (None, None))[0],
             "traffic_source": NCU_TRAFFIC.get(key, (None, None))[1], "peak_source": peak_src,
-            "kernel": f"{sp.EXEC_NAMES[plan.exec_mode]} executor, {sp.COPY_NAMES[plan.copy_path]} engine: "
+            "kernel": f"{sp.EXEC_NAMES[ran_exec]} executor, {sp.COPY_NAMES[ran_copy]} engine: "
                       f"{dom_name} ({launches_per_step:g} launch(es) per collective)",
             "algorithmic_bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
             "per_pass_us": per_pass_us,
@@ -405,7 +421,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
             "config": workload_config(args.algo, P, m, world),
-            "executor": {"exec": sp.EXEC_NAMES[plan.exec_mode], "copy": sp.COPY_NAMES[plan.copy_path],
+            "executor": {"exec": sp.EXEC_NAMES[ran_exec], "copy": sp.COPY_NAMES[ran_copy],
                          "recv_GiB_per_gpu": round(P * P * m / 2**30, 3)},
             "rounds": rounds, "timed_ms": float(sum(round_ms)),
             "ms_per_step_rounds": {"min": min(round_ms) / args.steps, "median": ms_per_step,

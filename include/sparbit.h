@@ -95,9 +95,10 @@ enum {
                                     buffers (shared memory), and every forwarded block is read from
                                     that copy of the sending rank's buffer, so a pass costs a
                                     shared-memory access instead of two trips to global memory.
-                                    Same passes, same order, same slots.  Needs P*P*m to fit into
-                                    one SM's shared memory (227 KB on B200), fixed-size blocks, at
-                                    most 16 passes, not Bruck; other calls run as GRAPH */
+                                    Same passes, same order, same slots.  Needs P*P*m (twice that
+                                    for Bruck, whose working buffers are kept the same way) to fit
+                                    into one SM's shared memory (227 KB on B200), fixed-size blocks
+                                    and at most 16 passes; other calls run as GRAPH */
 };
 
 /* Which copy engine a phase uses. */

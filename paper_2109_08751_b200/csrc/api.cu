@@ -381,14 +381,15 @@ struct Resolved {
     int vbytes;  // vector width for the vector engine
 };
 
-// The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers fit
-// into one CTA's shared memory together, between the send and the receive space only.
+// The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers (and,
+// for Bruck, working buffers) fit into one CTA's shared memory together.
 bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_limit) {
-    if (p->variable || p->sched.algo == ALGO_BRUCK) return false;
+    if (p->variable) return false;
     if (first != -1 || last != p->sched.last_phase()) return false;
     const ExecSeq seq = make_seq(p, first, last);
     if (seq.count() < 1 || seq.count() > kMirrorMaxPasses) return false;
-    const unsigned __int128 bytes = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
+    unsigned __int128 bytes = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
+    if (p->sched.algo == ALGO_BRUCK) bytes *= 2;  // its working buffers are mirrored too
     return bytes <= (unsigned __int128)smem_limit;
 }
 
@@ -809,7 +810,11 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
     uint64_t threads = (most + 3) / 4;
     threads = (threads + 63) / 64 * 64;
     if (threads > 1024) threads = 1024;
-    const size_t smem = (size_t)P * P * p->sched.m;
+    size_t smem = (size_t)P * P * p->sched.m;
+    if (p->sched.algo == ALGO_BRUCK) {
+        ma.work_at = (uint32_t)(smem / (size_t)rs.vbytes);
+        smem *= 2;
+    }
     const void* fn = pick_mirror_vec(rs.vbytes);
     if (smem > p->mirror_smem_set[rs.vbytes]) {
         CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

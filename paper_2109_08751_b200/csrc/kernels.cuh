@@ -675,17 +675,21 @@ __global__ void __launch_bounds__(256) persistent_bulk_kernel(Geom g, const Phas
 // buffer - the slot the schedule names, with the bytes that were stored there one or more passes
 // earlier - instead of from global memory.  The schedule, the passes and their order are
 // unchanged; a pass boundary is the CTA's barrier, and a pass costs a shared-memory access.
-// Only the own blocks are read from global memory (the send buffer).
+// Only the own blocks are read from global memory (the send buffer).  Bruck's working buffers are
+// mirrored the same way (twice the shared memory).
 constexpr int kMirrorMaxPasses = 16;
 struct MirrorArgs {
     PhaseDesc d[kMirrorMaxPasses];
     int n;
-    int pad_[3];
+    uint32_t work_at;  // Bruck: where, in vectors, the on-chip copy of the working buffers starts
+    int pad_[2];
 };
 
 template <typename V>
 __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
-    extern __shared__ __align__(16) unsigned char mirror[];  // [P][P] slots of m bytes, as the RECV space
+    // [P][P] slots of m bytes, laid out as the RECV space; for Bruck a second such array for its
+    // working buffers behind it
+    extern __shared__ __align__(16) unsigned char mirror[];
     chain_trigger();
     chain_wait();
     const uint32_t P = g.P;
@@ -697,6 +701,9 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
         const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
         const uint32_t total = P * d.copies * vpc;  // fits: the whole receive space is below 256 KiB
         const bool from_send = d.src_space == SPACE_SEND;
+        const V* msrc = mir + (d.src_space == SPACE_WORK ? ma.work_at : 0u);
+        V* mdst = mir + (d.dst_space == SPACE_WORK ? ma.work_at : 0u);
+        V* gdst = reinterpret_cast<V*>(space_base(g, d.dst_space));
         for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
             const uint32_t q = t / vpc;
             const uint32_t v = t - q * vpc;
@@ -704,14 +711,14 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
             const uint32_t j = q - r * d.copies;
             const CopyLoc c = locate_copy(d, P, r, j);
             const V x = from_send ? ld_cg<V>(reinterpret_cast<const V*>(g.base[SPACE_SEND] + (uint64_t)r * g.m) + v)
-                                  : mir[(c.src_rank * P + c.src_slot) * vps + v];
+                                  : msrc[(c.src_rank * P + c.src_slot) * vps + v];
             const uint32_t at = (c.dst_rank * P + c.dst_slot) * vps + v;
-            mir[at] = x;
-            st_cg<V>(reinterpret_cast<V*>(g.base[SPACE_RECV]) + at, x);
+            mdst[at] = x;
+            st_cg<V>(gdst + at, x);
             if (d.dup_self) {
                 const uint32_t at2 = (r * P + c.dst_slot) * vps + v;
-                mir[at2] = x;
-                st_cg<V>(reinterpret_cast<V*>(g.base[SPACE_RECV]) + at2, x);
+                mdst[at2] = x;
+                st_cg<V>(gdst + at2, x);
             }
         }
     }

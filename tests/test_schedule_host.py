@@ -138,7 +138,8 @@ def test_exec_mode_resolution():
     assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
     assert sp.Plan(32, 128).exec_mode == sp.EXEC_GRAPH           # 128 KiB: one CTA is too slow for it
     assert sp.Plan(32, 128, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
-    assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_GRAPH
+    assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_GRAPH      # 144 KiB
+    assert sp.Plan(8, 64, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR
     assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH         # 8.6 GB moved: chain + bulk engine
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
