@@ -310,7 +310,7 @@ def test_flow_all_algorithms_changing_data(dev, algo):
 def test_mirror_all_algorithms_changing_data(dev, algo):
     """The mirror executor on every algorithm it takes, up to the largest receive space that
     fits one SM's shared memory, at misaligned addresses too, with new data on every call."""
-    for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 65536), (1, 4096), (12, 100), (7, 4500)):
+    for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 32768), (1, 4096), (12, 100), (7, 4500)):
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
             continue
         if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
