@@ -62,6 +62,10 @@ def test_config3_p128_m64k_persistent(dev, copy):
     full_compare(dev, 128, 64 * 1024, sp.ALGO_SPARBIT, sp.EXEC_PERSISTENT, copy, si.BASE_SEED + 3)
 
 
+def test_config3_p128_m64k_flow(dev):
+    full_compare(dev, 128, 64 * 1024, sp.ALGO_SPARBIT, sp.EXEC_FLOW, sp.COPY_AUTO, si.BASE_SEED + 3)
+
+
 def test_config3_auto_is_what_the_benchmark_runs(dev):
     full_compare(dev, 128, 64 * 1024, sp.ALGO_SPARBIT, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 3, iters=1)
 
@@ -128,7 +132,8 @@ BIG_P, BIG_M = 272, 64 * 1024   # 4.85 GB of receive buffers, not a power of two
 
 
 @pytest.mark.parametrize("exec_mode,copy", [(sp.EXEC_GRAPH, sp.COPY_VECTOR), (sp.EXEC_PERSISTENT, sp.COPY_VECTOR),
-                                            (sp.EXEC_PERSISTENT, sp.COPY_BULK), (sp.EXEC_STREAM, sp.COPY_BULK)])
+                                            (sp.EXEC_PERSISTENT, sp.COPY_BULK), (sp.EXEC_STREAM, sp.COPY_BULK),
+                                            (sp.EXEC_FLOW, sp.COPY_VECTOR)])
 def test_offsets_beyond_4gib(dev, exec_mode, copy):
     P, m = BIG_P, BIG_M
     assert P * P * m > 1 << 32
@@ -140,7 +145,7 @@ def test_offsets_beyond_4gib(dev, exec_mode, copy):
     recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
     plan.allgather(send, recv)
     assert plan.status() == sp.OK
-    assert plan.copy_path == copy
+    assert plan.copy_path == copy and plan.exec_mode == exec_mode
     for k in si.sample_indices(8, P * P, seed=99):   # hop counts: one per set bit of the distance
         r, b = divmod(int(k), P)
         assert len(ref.trace(r, b)) - 1 == bin((r - b) % P).count("1")
