@@ -75,8 +75,9 @@ enum {
  * the first peer's): same state after phase 0, one pass less. */
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
-                                    buffers in all, FLOW for collectives that move 1 to 6 GB, the
-                                    graph chain otherwise (thresholds: SPARBIT_TUNE_*) */
+                                    buffers in all (up to 1 MiB for blocks of at most 256 B),
+                                    FLOW for collectives that move 1 to 6 GB, the graph chain
+                                    otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
@@ -95,10 +96,15 @@ enum {
                                     buffers (shared memory), and every forwarded block is read from
                                     that copy of the sending rank's buffer, so a pass costs a
                                     shared-memory access instead of two trips to global memory.
-                                    Same passes, same order, same slots.  Needs P*P*m (twice that
-                                    for Bruck, whose working buffers are kept the same way) to fit
-                                    into one SM's shared memory (227 KB on B200), fixed-size blocks
-                                    and at most 16 passes; other calls run as GRAPH */
+                                    Same passes, same order, same slots.  When P*P*m (twice that
+                                    for Bruck, whose working buffers are kept the same way) does
+                                    not fit one SM's shared memory (227 KB on B200), or exceeds
+                                    64 KiB, a cluster of up to 16 CTAs shares the work: rank r's
+                                    on-chip copy lives in CTA r mod C, a sender stores into the
+                                    receiver's CTA through distributed shared memory, the cluster
+                                    barrier separates the passes.  Needs ceil(P/16)*P*m to fit one
+                                    SM, fixed-size blocks and at most 16 passes; other calls run
+                                    as GRAPH */
 };
 
 /* Which copy engine a phase uses. */
@@ -325,7 +331,10 @@ enum {
                                               spans in all (0, the default: one per resident warp,
                                               4736 on B200; 1: every pass); smaller leading passes run
                                               as chained per-pass kernels in front of it */
-    SPARBIT_TUNE_COUNT_ = 8
+    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BYTES = 8, /* EXEC_AUTO: MIRROR on a cluster of CTAs when P*P*m is at most
+                                              this (1 MiB) ... */
+    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and m at most this (256 B) */
+    SPARBIT_TUNE_COUNT_ = 10
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

@@ -89,7 +89,7 @@ struct sparbit_plan_s {
     unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
     unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
     int flow_vbytes = 0;             // vector width those launches ran with
-    size_t mirror_smem_set[17] = {};  // dynamic shared memory already granted to the mirror kernel, by vector width
+    size_t mirror_smem_set[16] = {};  // dynamic shared memory already granted to the mirror kernels, by form and vector width
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -111,6 +111,8 @@ struct sparbit_plan_s {
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
         0,            // FLOW_MIN_PASS_SPANS (0: one span per resident warp)
+        1u << 20,     // MIRROR_CLUSTER_MAX_BYTES
+        256,          // MIRROR_CLUSTER_MAX_BLOCK
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -317,6 +319,17 @@ const void* pick_mirror_vec(int vbytes) {
     }
 }
 template <typename V>
+const void* cluster_mirror_vec_fn() { return (const void*)cluster_mirror_vec_kernel<V>; }
+const void* pick_cluster_mirror_vec(int vbytes) {
+    switch (vbytes) {
+        case 16: return cluster_mirror_vec_fn<uint4>();
+        case 8: return cluster_mirror_vec_fn<uint2>();
+        case 4: return cluster_mirror_vec_fn<unsigned>();
+        case 2: return cluster_mirror_vec_fn<unsigned short>();
+        default: return cluster_mirror_vec_fn<unsigned char>();
+    }
+}
+template <typename V>
 const void* flow_vec_fn() { return (const void*)flow_vec_kernel<V, kVecUnroll>; }
 const void* pick_flow_vec(int vbytes) {
     switch (vbytes) {
@@ -381,16 +394,25 @@ struct Resolved {
     int vbytes;  // vector width for the vector engine
 };
 
-// The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers (and,
-// for Bruck, working buffers) fit into one CTA's shared memory together.
+// Shared memory one CTA of a cluster of C needs for the mirror executor: the receive buffers (and,
+// for Bruck, working buffers) of its ceil(P / C) ranks.  C = 1: the single-CTA form.
+unsigned __int128 mirror_smem_per_cta(const sparbit_plan_s* p, uint32_t C) {
+    const uint32_t ranks = (p->sched.P + C - 1) / C;
+    unsigned __int128 bytes = (unsigned __int128)ranks * p->sched.P * p->sched.m;
+    if (p->sched.algo == ALGO_BRUCK) bytes *= 2;
+    return bytes;
+}
+
+constexpr uint32_t kMirrorMaxCluster = 16;  // the largest cluster a B200 places (non-portable size)
+
+// The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers fit
+// into the shared memory of one CTA, or of the CTAs of one cluster, together.
 bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_limit) {
     if (p->variable) return false;
     if (first != -1 || last != p->sched.last_phase()) return false;
     const ExecSeq seq = make_seq(p, first, last);
     if (seq.count() < 1 || seq.count() > kMirrorMaxPasses) return false;
-    unsigned __int128 bytes = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
-    if (p->sched.algo == ALGO_BRUCK) bytes *= 2;  // its working buffers are mirrored too
-    return bytes <= (unsigned __int128)smem_limit;
+    return mirror_smem_per_cta(p, kMirrorMaxCluster) <= (unsigned __int128)smem_limit;
 }
 
 // Which passes of a call the flow kernel takes: the longest run of passes at the END of the
@@ -430,7 +452,11 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 // Executor for SPARBIT_EXEC_AUTO, from measurements on B200.
 //  - Up to 64 KiB of receive buffers in all, the mirror executor: one CTA, passes separated by its
 //    own barrier and fed from shared memory (P = 8, m = 64 B: 4.1 us against 6.2 for the chain;
-//    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain.
+//    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain, and a
+//    cluster of CTAs with the copies in distributed shared memory takes over, up to 1 MiB of
+//    receive buffers with blocks of at most 256 B (P = 64, m = 64 B: 10.3 against 14.4; P = 253,
+//    m = 16 B: 18.5 against 22.5): its pass still waits for the acknowledged global stores, so it
+//    gains 10-30 %, not the factor the single CTA gains, and loses beyond those sizes.
 //  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
 //    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
@@ -442,10 +468,18 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.
+// where the mirror executor is the fastest (measured): one CTA up to MIRROR_MAX_BYTES of receive
+// buffers in all, a cluster up to MIRROR_CLUSTER_MAX_BYTES when blocks are at most
+// MIRROR_CLUSTER_MAX_BLOCK bytes
+bool mirror_wins(const sparbit_plan_s* p) {
+    const unsigned __int128 all = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
+    if (all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) return true;
+    return all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BYTES] &&
+           p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK];
+}
+
 int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
-    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) &&
-        (uint64_t)p->sched.P * p->sched.P * p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES])
-        return SPARBIT_EXEC_MIRROR;
+    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) && mirror_wins(p)) return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
@@ -454,9 +488,7 @@ int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
 }
 
 int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
-    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) &&
-        (uint64_t)p->sched.P * p->sched.P * p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES])
-        return SPARBIT_EXEC_MIRROR;
+    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) && mirror_wins(p)) return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
@@ -793,7 +825,8 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
     return SPARBIT_OK;
 }
 
-// The whole collective in one CTA with the receive buffers mirrored in shared memory.
+// The whole collective in one CTA, or in one cluster of CTAs, with the receive buffers mirrored in
+// (distributed) shared memory.
 int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
@@ -806,36 +839,67 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         const uint64_t v = (uint64_t)P * ma.d[i].copies * (ma.d[i].copy_bytes / (uint64_t)rs.vbytes);
         if (v > most) most = v;
     }
-    // four vectors per thread and pass when there are that many, CTA sizes in steps of two warps
-    uint64_t threads = (most + 3) / 4;
-    threads = (threads + 63) / 64 * 64;
-    if (threads > 1024) threads = 1024;
-    size_t smem = (size_t)P * P * p->sched.m;
-    if (p->sched.algo == ALGO_BRUCK) {
-        ma.work_at = (uint32_t)(smem / (size_t)rs.vbytes);
-        smem *= 2;
-    }
-    const void* fn = pick_mirror_vec(rs.vbytes);
-    if (smem > p->mirror_smem_set[rs.vbytes]) {
-        CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        p->mirror_smem_set[rs.vbytes] = smem;
-    }
+    // One CTA while everything fits and is small enough for it (measured: up to 64 KiB); else the
+    // smallest cluster that holds it and leaves a CTA about one vector per thread in the largest pass.
+    uint32_t C = 1;
+    const unsigned __int128 limit = (unsigned __int128)p->max_smem_optin;
+    while (C < kMirrorMaxCluster &&
+           (mirror_smem_per_cta(p, C) > limit || (C < P && mirror_smem_per_cta(p, 1) > (64u << 10) && most / C > 1024)))
+        C *= 2;
     cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3((unsigned)threads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
     Geom gg = g;
     void* args[] = {&gg, &ma};
-    CU(cudaLaunchKernelExC(&cfg, fn, args));
-    p->kernel_launches++;
-    return SPARBIT_OK;
+    for (;;) {
+        const void* fn = C == 1 ? pick_mirror_vec(rs.vbytes) : pick_cluster_mirror_vec(rs.vbytes);
+        const size_t ranks = (P + C - 1) / C;
+        size_t smem = ranks * P * p->sched.m;
+        ma.work_at = 0;
+        if (p->sched.algo == ALGO_BRUCK) {
+            ma.work_at = (uint32_t)(smem / (size_t)rs.vbytes);
+            smem *= 2;
+        }
+        // four vectors per thread and pass when there are that many, CTA sizes in steps of two warps
+        uint64_t threads = (most / C + 3) / 4;
+        threads = (threads + 63) / 64 * 64;
+        if (threads > 1024) threads = 1024;
+        size_t& granted = p->mirror_smem_set[(C == 1 ? 0 : 8) + (rs.vbytes == 16 ? 4 : rs.vbytes == 8 ? 3 : rs.vbytes == 4 ? 2 : rs.vbytes == 2 ? 1 : 0)];
+        if (smem > granted) {
+            CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            if (C > 8) CU(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            granted = smem;
+        }
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(C);
+        cfg.blockDim = dim3((unsigned)threads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (C > 1) {
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = C;
+            attr[1].val.clusterDim.y = 1;
+            attr[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+            // can the device place this cluster at all?  If not, a smaller one that still holds the
+            // buffers, else the per-pass kernels
+            int fit = 0;
+            if (cudaOccupancyMaxActiveClusters(&fit, fn, &cfg) != cudaSuccess || fit < 1) {
+                (void)cudaGetLastError();
+                if (C > 2 && mirror_smem_per_cta(p, C / 2) <= limit) {
+                    C /= 2;
+                    continue;
+                }
+                return launch_stream(p, rs, g, first, last, st);
+            }
+        }
+        CU(cudaLaunchKernelExC(&cfg, fn, args));
+        p->kernel_launches++;
+        return SPARBIT_OK;
+    }
 }
 
 // The flow executor's pass table (host only): how each pass is cut into units, where its rank

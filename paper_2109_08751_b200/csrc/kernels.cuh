@@ -724,6 +724,102 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
     }
 }
 
+// The same idea on a thread-block CLUSTER, for collectives whose receive buffers fit into the
+// shared memory of up to 16 SMs together: rank r's on-chip copy lives in CTA r mod C of the cluster
+// (ranks c, c+C, c+2C, ... one after the other).  A CTA executes the copies its own ranks SEND: it
+// reads the block from its local shared memory and stores it into the destination rank's CTA through
+// distributed shared memory (st.shared::cluster) and into global memory; the hardware cluster barrier
+// (arrive.release / wait.acquire) is the Waitall.  A pass costs a shared-memory read, a posted remote
+// write and that barrier.  The last barrier keeps every CTA alive until nobody writes into it any more.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_shared_addr, uint32_t cta) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_shared_addr), "r"(cta));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+template <typename V>
+__device__ __forceinline__ void st_cluster(uint32_t addr, V v);
+template <>
+__device__ __forceinline__ void st_cluster<uint4>(uint32_t addr, uint4 v) {
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+template <>
+__device__ __forceinline__ void st_cluster<uint2>(uint32_t addr, uint2 v) {
+    asm volatile("st.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
+}
+template <>
+__device__ __forceinline__ void st_cluster<unsigned>(uint32_t addr, unsigned v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+template <>
+__device__ __forceinline__ void st_cluster<unsigned short>(uint32_t addr, unsigned short v) {
+    asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+template <>
+__device__ __forceinline__ void st_cluster<unsigned char>(uint32_t addr, unsigned char v) {
+    asm volatile("st.shared::cluster.u8 [%0], %1;" ::"r"(addr), "r"((uint32_t)v) : "memory");
+}
+
+template <typename V>
+__global__ void __launch_bounds__(1024, 1) cluster_mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
+    // this CTA's ranks (c, c + C, ...), each [P] slots of m bytes; for Bruck the working buffers behind
+    extern __shared__ __align__(16) unsigned char mirror[];
+    chain_trigger();
+    chain_wait();
+    const uint32_t P = g.P;
+    const uint32_t C = cluster_nctarank();
+    const uint32_t c = cluster_ctarank();
+    const uint32_t mine = c < P ? (P - c + C - 1) / C : 0u;  // ranks this CTA holds
+    const uint32_t vps = (uint32_t)(g.m / sizeof(V));        // vectors per slot
+    V* mir = reinterpret_cast<V*>(mirror);
+    const uint32_t mir_base = smem_u32(mirror);
+    for (int i = 0; i < ma.n; i++) {
+        // every CTA of the cluster passes here the same number of times: the Waitall, and before
+        // the first pass the guarantee that all CTAs of the cluster have started
+        cluster_sync_all();
+        const PhaseDesc& d = ma.d[i];
+        const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
+        const uint32_t total = mine * d.copies * vpc;
+        const bool from_send = d.src_space == SPACE_SEND;
+        const uint32_t src_at = d.src_space == SPACE_WORK ? ma.work_at : 0u;
+        const uint32_t dst_at = d.dst_space == SPACE_WORK ? ma.work_at : 0u;
+        V* gdst = reinterpret_cast<V*>(space_base(g, d.dst_space));
+        for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+            const uint32_t q = t / vpc;
+            const uint32_t v = t - q * vpc;
+            const uint32_t lr = q / d.copies;  // which of this CTA's ranks sends
+            const uint32_t j = q - lr * d.copies;
+            const uint32_t r = c + lr * C;
+            const CopyLoc loc = locate_copy(d, P, r, j);
+            const V x = from_send ? ld_cg<V>(reinterpret_cast<const V*>(g.base[SPACE_SEND] + (uint64_t)r * g.m) + v)
+                                  : mir[src_at + (lr * P + loc.src_slot) * vps + v];
+            // the receiving rank's copy: CTA dst_rank mod C, its (dst_rank / C)-th rank
+            const uint32_t there = dst_at + ((loc.dst_rank / C) * P + loc.dst_slot) * vps + v;
+            st_cluster<V>(map_to_cta(mir_base + there * (uint32_t)sizeof(V), loc.dst_rank % C), x);
+            st_cg<V>(gdst + (loc.dst_rank * P + loc.dst_slot) * vps + v, x);
+            if (d.dup_self) {
+                mir[dst_at + (lr * P + loc.dst_slot) * vps + v] = x;
+                st_cg<V>(gdst + (r * P + loc.dst_slot) * vps + v, x);
+            }
+        }
+    }
+    cluster_sync_all();  // nobody leaves while a neighbour may still store into its shared memory
+}
+
 // ------------------------------------------------------------------------------------------------
 // flow executor: the whole collective in one cooperative kernel WITHOUT grid-wide barriers
 // ------------------------------------------------------------------------------------------------

@@ -174,14 +174,15 @@ SPLIT_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 40}     # passes of fewer than 40 spa
 @pytest.mark.parametrize("exec_mode,m,tune", [(sp.EXEC_PERSISTENT, 16, None), (sp.EXEC_FLOW, 512, ALL_IN_FLOW),
                                               (sp.EXEC_FLOW, 1040, ALL_IN_FLOW), (sp.EXEC_FLOW, 1040, SPLIT_FLOW),
                                               (sp.EXEC_FLOW, 16, None), (sp.EXEC_MIRROR, 16, None),
-                                              (sp.EXEC_MIRROR, 52, None)])
+                                              (sp.EXEC_MIRROR, 52, None), (sp.EXEC_MIRROR, 600, None)])
 def test_every_p_up_to_64(dev, exec_mode, m, tune):
     """Every communicator size, on the single-kernel executors.  The flow executor takes blocks
     of at least 32 vectors (512 B: one warp row; 1040 B: two ragged spans per block) and hands
     smaller ones to the graph chain, and by default leaves passes that cannot keep every warp busy
     to per-pass kernels in front of it: the tests set that threshold so that the kernel takes
-    every pass, or only those of at least 40 spans; the mirror executor takes what fits into one SM's shared
-    memory (all of these at 16 B, up to P = 64 at 52 B) and hands the rest to the graph chain."""
+    every pass, or only those of at least 40 spans; the mirror executor runs in one CTA up to 64 KiB of
+    receive buffers (all of these at 16 B) and in a cluster of 2 to 16 CTAs above that (52 B from
+    P = 36 on, 600 B from P = 11 on)."""
     for P in range(1, 65):
         ran = sp.EXEC_FLOW if tune is ALL_IN_FLOW else None
         run_case(dev, P, m, sp.ALGO_SPARBIT, exec_mode, sp.COPY_AUTO, 1000 + P, iters=2 if m != 16 else 1, tune=tune,
@@ -310,12 +311,15 @@ def test_flow_all_algorithms_changing_data(dev, algo):
 def test_mirror_all_algorithms_changing_data(dev, algo):
     """The mirror executor on every algorithm it takes, up to the largest receive space that
     fits one SM's shared memory, at misaligned addresses too, with new data on every call."""
-    for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 32768), (1, 4096), (12, 100), (7, 4500)):
+    for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 32768), (1, 4096), (12, 100), (7, 4500),
+                 (16, 4096), (13, 8192), (32, 1000), (64, 208), (128, 64), (100, 96), (253, 24)):
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
             continue
         if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
             continue
-        if algo == sp.ALGO_BRUCK and 2 * P * P * m > 220 * 1024:
+        if algo == sp.ALGO_RING and P > 17 or algo == sp.ALGO_NEIGHBOR_EXCHANGE and P > 32:
+            continue   # more passes than the kernel's parameter table holds
+        if algo == sp.ALGO_BRUCK and 2 * ((P + 15) // 16) * P * m > 220 * 1024:
             continue   # Bruck mirrors its working buffers as well
         run_case(dev, P, m, algo, sp.EXEC_MIRROR, sp.COPY_AUTO, 90 + P, iters=3, ran=sp.EXEC_MIRROR)
     run_case(dev, 9, 96, algo if algo != sp.ALGO_RECURSIVE_DOUBLING and algo != sp.ALGO_NEIGHBOR_EXCHANGE
@@ -323,8 +327,10 @@ def test_mirror_all_algorithms_changing_data(dev, algo):
 
 
 def test_mirror_runs_where_it_fits_and_hands_over_where_not(dev):
-    for P, m, want in ((8, 64, sp.EXEC_MIRROR), (6, 4096, sp.EXEC_MIRROR), (13, 4096, sp.EXEC_GRAPH),
-                       (64, 64, sp.EXEC_GRAPH), (20, 16, sp.EXEC_MIRROR)):
+    # one CTA up to 227 KB, a cluster of up to 16 CTAs up to 16 x 227 KB, the graph chain beyond
+    for P, m, want in ((8, 64, sp.EXEC_MIRROR), (6, 4096, sp.EXEC_MIRROR), (13, 4096, sp.EXEC_MIRROR),
+                       (64, 64, sp.EXEC_MIRROR), (20, 16, sp.EXEC_MIRROR), (256, 48, sp.EXEC_MIRROR),
+                       (64, 4096, sp.EXEC_GRAPH), (256, 64, sp.EXEC_GRAPH)):
         plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
         send = torch.from_numpy(si.send_blocks(P, m, 1).reshape(-1)).to(dev)
         recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
@@ -374,8 +380,7 @@ def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
     if exec_mode in (sp.EXEC_PERSISTENT, sp.EXEC_FLOW):
         assert (kernels, graphs) == (2, 0)
     elif exec_mode == sp.EXEC_MIRROR:
-        assert (kernels, graphs) == (2 * phases, 2)     # 256 KiB of receive buffers: runs as a graph chain
-        exec_mode = sp.EXEC_GRAPH
+        assert (kernels, graphs) == (2, 2)     # 256 KiB of receive buffers: one cluster kernel in a cached graph
         small = sp.Plan(8, 64, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
         small.allgather(send[: 8 * 64], recv, stream)
         small.allgather(send[: 8 * 64], recv, stream)

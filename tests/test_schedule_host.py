@@ -136,8 +136,11 @@ def test_strerror_covers_every_code():
 def test_exec_mode_resolution():
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR            # 4 KiB of receive buffers: one CTA, on chip
     assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
-    assert sp.Plan(32, 128).exec_mode == sp.EXEC_GRAPH           # 128 KiB: one CTA is too slow for it
-    assert sp.Plan(32, 128, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
+    assert sp.Plan(32, 128).exec_mode == sp.EXEC_MIRROR          # 128 KiB, small blocks: a cluster of CTAs
+    assert sp.Plan(128, 64).exec_mode == sp.EXEC_MIRROR          # 1 MiB: still
+    assert sp.Plan(128, 128).exec_mode == sp.EXEC_GRAPH          # 2 MiB: the chain is faster
+    assert sp.Plan(16, 4096).exec_mode == sp.EXEC_GRAPH          # 1 MiB of large blocks: the chain too
+    assert sp.Plan(16, 4096, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
     assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_GRAPH      # 144 KiB
     assert sp.Plan(8, 64, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR
     assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH         # 8.6 GB moved: chain + bulk engine
