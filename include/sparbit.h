@@ -75,7 +75,7 @@ enum {
  * the first peer's): same state after phase 0, one pass less. */
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
-                                    buffers in all (up to 1 MiB for blocks of at most 256 B),
+                                    buffers in all (up to 1 MiB for blocks of at most 4 KiB),
                                     FLOW for collectives that move 1 to 6 GB, the graph chain
                                     otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
@@ -101,10 +101,12 @@ enum {
                                     not fit one SM's shared memory (227 KB on B200), or exceeds
                                     64 KiB, a cluster of up to 16 CTAs shares the work: rank r's
                                     on-chip copy lives in CTA r mod C, a sender stores into the
-                                    receiver's CTA through distributed shared memory, the cluster
-                                    barrier separates the passes.  Needs ceil(P/16)*P*m to fit one
-                                    SM, fixed-size blocks and at most 16 passes; other calls run
-                                    as GRAPH */
+                                    receiver's CTA through distributed shared memory, and a CTA
+                                    starts a pass when the bytes its ranks receive in the passes
+                                    before have arrived (one mbarrier per pass counts them; bounded
+                                    wait, time-out through sparbit_plan_status).  Needs
+                                    ceil(P/16)*P*m to fit one SM, fixed-size blocks and at most 16
+                                    passes; other calls run as GRAPH */
 };
 
 /* Which copy engine a phase uses. */
@@ -333,8 +335,12 @@ enum {
                                               as chained per-pass kernels in front of it */
     SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BYTES = 8, /* EXEC_AUTO: MIRROR on a cluster of CTAs when P*P*m is at most
                                               this (1 MiB) ... */
-    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and m at most this (256 B) */
-    SPARBIT_TUNE_COUNT_ = 10
+    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and m at most this (4 KiB) */
+    SPARBIT_TUNE_MIRROR_CTA_VECTORS = 10,  /* EXEC_MIRROR: the cluster is doubled while a CTA would get more
+                                              vectors than this in the largest pass (256) */
+    SPARBIT_TUNE_MIRROR_THREAD_VECTORS = 11, /* EXEC_MIRROR: vectors of the largest pass per thread (4), CTAs
+                                              of at most 1024 threads */
+    SPARBIT_TUNE_COUNT_ = 12
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

@@ -112,7 +112,9 @@ struct sparbit_plan_s {
         64u << 10,    // MIRROR_MAX_BYTES
         0,            // FLOW_MIN_PASS_SPANS (0: one span per resident warp)
         1u << 20,     // MIRROR_CLUSTER_MAX_BYTES
-        256,          // MIRROR_CLUSTER_MAX_BLOCK
+        4096,         // MIRROR_CLUSTER_MAX_BLOCK
+        256,          // MIRROR_CTA_VECTORS
+        4,            // MIRROR_THREAD_VECTORS
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -320,11 +322,14 @@ const void* pick_mirror_vec(int vbytes) {
 }
 template <typename V>
 const void* cluster_mirror_vec_fn() { return (const void*)cluster_mirror_vec_kernel<V>; }
+template <typename V>
+const void* cluster_mirror_async_fn() { return (const void*)cluster_mirror_async_kernel<V>; }
+// st.async moves 4, 8 or 16 bytes: smaller vectors take the form with a cluster barrier per pass
 const void* pick_cluster_mirror_vec(int vbytes) {
     switch (vbytes) {
-        case 16: return cluster_mirror_vec_fn<uint4>();
-        case 8: return cluster_mirror_vec_fn<uint2>();
-        case 4: return cluster_mirror_vec_fn<unsigned>();
+        case 16: return cluster_mirror_async_fn<uint4>();
+        case 8: return cluster_mirror_async_fn<uint2>();
+        case 4: return cluster_mirror_async_fn<unsigned>();
         case 2: return cluster_mirror_vec_fn<unsigned short>();
         default: return cluster_mirror_vec_fn<unsigned char>();
     }
@@ -454,9 +459,10 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //    own barrier and fed from shared memory (P = 8, m = 64 B: 4.1 us against 6.2 for the chain;
 //    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain, and a
 //    cluster of CTAs with the copies in distributed shared memory takes over, up to 1 MiB of
-//    receive buffers with blocks of at most 256 B (P = 64, m = 64 B: 10.3 against 14.4; P = 253,
-//    m = 16 B: 18.5 against 22.5): its pass still waits for the acknowledged global stores, so it
-//    gains 10-30 %, not the factor the single CTA gains, and loses beyond those sizes.
+//    receive buffers with blocks of at most 4 KiB (P = 64, m = 64 B: 8.2 against 14.4; P = 128,
+//    m = 64 B: 10.3 against 16.4; P = 256, m = 8 B: 14.4 against 20.5; P = 16, m = 4 KiB: 8.2
+//    against 9.2): a pass is one push through the SM-to-SM network and an mbarrier, about 0.8 us.
+//    Beyond 1 MiB sixteen SMs' bandwidth eats the gain (P = 64, m = 512 B: 14.4 against 12.3).
 //  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
 //    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
@@ -468,9 +474,9 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.
-// where the mirror executor is the fastest (measured): one CTA up to MIRROR_MAX_BYTES of receive
+// Where the mirror executor is the fastest (measured): one CTA up to MIRROR_MAX_BYTES of receive
 // buffers in all, a cluster up to MIRROR_CLUSTER_MAX_BYTES when blocks are at most
-// MIRROR_CLUSTER_MAX_BLOCK bytes
+// MIRROR_CLUSTER_MAX_BLOCK bytes.
 bool mirror_wins(const sparbit_plan_s* p) {
     const unsigned __int128 all = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
     if (all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) return true;
@@ -833,18 +839,25 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
     MirrorArgs ma;
     memset(&ma, 0, sizeof ma);
     ma.n = seq.count();
+    ma.status = p->d_ctl + 1;
+    ma.timeout_ns = p->timeout_ns;
+    ma.extra_tx = p->mbar_extra_tx;
     uint64_t most = 1;  // vectors of the largest pass
     for (int i = 0; i < ma.n; i++) {
         ma.d[i] = seq.item(i);
-        const uint64_t v = (uint64_t)P * ma.d[i].copies * (ma.d[i].copy_bytes / (uint64_t)rs.vbytes);
+        const uint64_t vpc = ma.d[i].copy_bytes / (uint64_t)rs.vbytes;
+        const uint64_t v = (uint64_t)P * ma.d[i].copies * vpc;
         if (v > most) most = v;
+        ma.magic_vpc[i] = ((1ull << 40) + vpc - 1) / (vpc ? vpc : 1);
+        ma.magic_copies[i] = ((1ull << 40) + ma.d[i].copies - 1) / (ma.d[i].copies ? ma.d[i].copies : 1);
     }
-    // One CTA while everything fits and is small enough for it (measured: up to 64 KiB); else the
-    // smallest cluster that holds it and leaves a CTA about one vector per thread in the largest pass.
+    // One CTA while everything fits and is small enough for it (MIRROR_MAX_BYTES); else the smallest
+    // cluster that holds it and leaves a CTA at most MIRROR_CTA_VECTORS vectors in the largest pass.
     uint32_t C = 1;
     const unsigned __int128 limit = (unsigned __int128)p->max_smem_optin;
     while (C < kMirrorMaxCluster &&
-           (mirror_smem_per_cta(p, C) > limit || (C < P && mirror_smem_per_cta(p, 1) > (64u << 10) && most / C > 1024)))
+           (mirror_smem_per_cta(p, C) > limit || (C < P && mirror_smem_per_cta(p, 1) > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] &&
+            most / C > p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS])))
         C *= 2;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
@@ -860,7 +873,8 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
             smem *= 2;
         }
         // four vectors per thread and pass when there are that many, CTA sizes in steps of two warps
-        uint64_t threads = (most / C + 3) / 4;
+        const uint64_t per_thread = p->tune[SPARBIT_TUNE_MIRROR_THREAD_VECTORS];
+        uint64_t threads = (most / C + per_thread - 1) / per_thread;
         threads = (threads + 63) / 64 * 64;
         if (threads > 1024) threads = 1024;
         size_t& granted = p->mirror_smem_set[(C == 1 ? 0 : 8) + (rs.vbytes == 16 ? 4 : rs.vbytes == 8 ? 3 : rs.vbytes == 4 ? 2 : rs.vbytes == 2 ? 1 : 0)];
@@ -1318,6 +1332,8 @@ int sparbit_plan_set_copy_path(sparbit_plan_t* p, int copy_path) {
 
 int sparbit_plan_set_tunable(sparbit_plan_t* p, int key, uint64_t value) {
     if (!p || key < 0 || key >= SPARBIT_TUNE_COUNT_) return SPARBIT_ERR_ARG;
+    if ((key == SPARBIT_TUNE_MIRROR_CTA_VECTORS || key == SPARBIT_TUNE_MIRROR_THREAD_VECTORS) && value == 0)
+        return SPARBIT_ERR_ARG;  // divisors
     if (p->tune[key] == value) return SPARBIT_OK;
     if (p->launched) {
         // cached graphs were cut into launches with the old value

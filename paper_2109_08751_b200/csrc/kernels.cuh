@@ -682,7 +682,15 @@ struct MirrorArgs {
     PhaseDesc d[kMirrorMaxPasses];
     int n;
     uint32_t work_at;  // Bruck: where, in vectors, the on-chip copy of the working buffers starts
-    int pad_[2];
+    uint32_t extra_tx;  // cluster form, test hook: bytes expected on top of a pass's own (never arrive)
+    int pad_;
+    unsigned* status;   // cluster form: device status word (DEV_*)
+    unsigned long long timeout_ns;
+    // ceil(2^40 / x) for x = vectors per copy and x = copies per rank of each pass, so that t / x
+    // is a multiplication and a shift (exact while t * x < 2^40; t counts the vectors sent in a
+    // pass, fewer than the shared memory holds bytes: 2^18)
+    unsigned long long magic_vpc[kMirrorMaxPasses];
+    unsigned long long magic_copies[kMirrorMaxPasses];
 };
 
 template <typename V>
@@ -704,10 +712,11 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
         const V* msrc = mir + (d.src_space == SPACE_WORK ? ma.work_at : 0u);
         V* mdst = mir + (d.dst_space == SPACE_WORK ? ma.work_at : 0u);
         V* gdst = reinterpret_cast<V*>(space_base(g, d.dst_space));
+        const unsigned long long mv = ma.magic_vpc[i], mc = ma.magic_copies[i];
         for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
-            const uint32_t q = t / vpc;
+            const uint32_t q = (uint32_t)((t * mv) >> 40);  // t / vpc
             const uint32_t v = t - q * vpc;
-            const uint32_t r = q / d.copies;
+            const uint32_t r = (uint32_t)((q * mc) >> 40);  // q / copies
             const uint32_t j = q - r * d.copies;
             const CopyLoc c = locate_copy(d, P, r, j);
             const V x = from_send ? ld_cg<V>(reinterpret_cast<const V*>(g.base[SPACE_SEND] + (uint64_t)r * g.m) + v)
@@ -818,6 +827,105 @@ __global__ void __launch_bounds__(1024, 1) cluster_mirror_vec_kernel(Geom g, con
         }
     }
     cluster_sync_all();  // nobody leaves while a neighbour may still store into its shared memory
+}
+
+// The cluster form without a barrier between the passes, for vectors of 4, 8 and 16 bytes.  A copy
+// is pushed with st.async: the store into the receiving CTA's shared memory completes bytes on an
+// mbarrier IN THAT CTA, one mbarrier per pass, armed at the start with the bytes the CTA's ranks
+// receive in that pass (every rank receives `copies` blocks of `copy_bytes` per pass, twice that
+// when the pass also files the own block).  What a rank sends in pass i it has received in passes
+// before i, and its on-chip copy sits in the CTA that sends for it, so a CTA's Waitall is a wait on
+// its OWN mbarriers of the passes before: no round trip, no cluster-wide barrier, and the global
+// stores of a pass are not waited for before the next one starts (nobody reads them in this
+// kernel; they are complete when the kernel is).  No slot is written twice within a collective, so
+// a CTA that runs ahead cannot overwrite what a slower one still reads.  Waits are bounded; a wait
+// that gives up sets the status word and the thread goes to the final cluster barrier.
+template <typename V>
+__device__ __forceinline__ void st_async_cluster(uint32_t addr, V v, uint32_t bar);
+template <>
+__device__ __forceinline__ void st_async_cluster<uint4>(uint32_t addr, uint4 v, uint32_t bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(bar)
+                 : "memory");
+}
+template <>
+__device__ __forceinline__ void st_async_cluster<uint2>(uint32_t addr, uint2 v, uint32_t bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(addr), "r"(v.x),
+                 "r"(v.y), "r"(bar)
+                 : "memory");
+}
+template <>
+__device__ __forceinline__ void st_async_cluster<unsigned>(uint32_t addr, unsigned v, uint32_t bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(addr), "r"(v), "r"(bar)
+                 : "memory");
+}
+
+template <typename V>
+__global__ void __launch_bounds__(1024, 1) cluster_mirror_async_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
+    extern __shared__ __align__(16) unsigned char mirror[];
+    __shared__ __align__(8) unsigned long long pass_bar[kMirrorMaxPasses];
+    chain_trigger();
+    const uint32_t P = g.P;
+    const uint32_t C = cluster_nctarank();
+    const uint32_t c = cluster_ctarank();
+    const uint32_t mine = c < P ? (P - c + C - 1) / C : 0u;  // ranks this CTA holds
+    const uint32_t vps = (uint32_t)(g.m / sizeof(V));        // vectors per slot
+    V* mir = reinterpret_cast<V*>(mirror);
+    const uint32_t mir_base = smem_u32(mirror);
+    const uint32_t bar_base = smem_u32(pass_bar);
+    const uint32_t lgC = 31u - (uint32_t)__clz(C);  // cluster sizes are powers of two
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < ma.n; i++) mbar_init(bar_base + 8u * i, 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; i < ma.n; i++) {
+            const PhaseDesc& d = ma.d[i];
+            mbar_expect_tx(bar_base + 8u * i, mine * d.copies * (uint32_t)d.copy_bytes * (d.dup_self ? 2u : 1u) + ma.extra_tx);
+        }
+    }
+    cluster_sync_all();  // every CTA of the cluster runs and its mbarriers are armed
+    chain_wait();        // (all of the above touches no global memory: it overlaps the kernel before)
+    bool ok = true;
+    for (int i = 0; i < ma.n && ok; i++) {
+        // the Waitall of the pass before, for this CTA's ranks (all threads, so that a thread
+        // without work in some pass has still seen every earlier pass arrive)
+        // (every thread polls: measured faster than one poller per warp or per CTA handing the
+        // result on)
+        if (i > 0) ok = mbar_wait_bounded(bar_base + 8u * (i - 1), 0u, ma.status, ma.timeout_ns);
+        if (!ok) break;
+        const PhaseDesc& d = ma.d[i];
+        const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
+        const uint32_t total = mine * d.copies * vpc;
+        const bool from_send = d.src_space == SPACE_SEND;
+        const uint32_t src_at = d.src_space == SPACE_WORK ? ma.work_at : 0u;
+        const uint32_t dst_at = d.dst_space == SPACE_WORK ? ma.work_at : 0u;
+        const uint32_t bar = bar_base + 8u * i;
+        V* gdst = reinterpret_cast<V*>(space_base(g, d.dst_space));
+        const unsigned long long mv = ma.magic_vpc[i], mc = ma.magic_copies[i];
+        const V* gsend = reinterpret_cast<const V*>(g.base[SPACE_SEND]);
+        for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+            const uint32_t q = (uint32_t)((t * mv) >> 40);   // t / vpc
+            const uint32_t v = t - q * vpc;
+            const uint32_t lr = (uint32_t)((q * mc) >> 40);  // q / copies: which of this CTA's ranks sends
+            const uint32_t j = q - lr * d.copies;
+            const uint32_t r = c + (lr << lgC);
+            const CopyLoc loc = locate_copy(d, P, r, j);
+            const V x = from_send ? ld_cg<V>(gsend + (uint64_t)r * vps + v) : mir[src_at + (lr * P + loc.src_slot) * vps + v];
+            // the receiving rank's copy: CTA dst_rank mod C, its (dst_rank / C)-th rank
+            const uint32_t to = loc.dst_rank & (C - 1u);
+            const uint32_t there = dst_at + ((loc.dst_rank >> lgC) * P + loc.dst_slot) * vps + v;
+            st_async_cluster<V>(map_to_cta(mir_base + there * (uint32_t)sizeof(V), to), x, map_to_cta(bar, to));
+            st_cg<V>(gdst + (loc.dst_rank * P + loc.dst_slot) * vps + v, x);
+            if (d.dup_self) {
+                const uint32_t here = dst_at + (lr * P + loc.dst_slot) * vps + v;
+                st_async_cluster<V>(map_to_cta(mir_base + here * (uint32_t)sizeof(V), c), x, map_to_cta(bar, c));
+                st_cg<V>(gdst + (r * P + loc.dst_slot) * vps + v, x);
+            }
+        }
+    }
+    // nothing may still be on its way into this CTA when it leaves, and no CTA leaves before the others
+    if (ok) mbar_wait_bounded(bar_base + 8u * (ma.n - 1), 0u, ma.status, ma.timeout_ns);
+    __syncwarp();  // threads that gave up in different passes meet again before the aligned barrier
+    cluster_sync_all();
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -49,7 +49,7 @@ int main(void) {
         free(m);
     }
     CHECK(sparbit_plan_workspace_bytes(plan) == 0);
-    CHECK(sparbit_plan_exec_mode(plan) == SPARBIT_EXEC_GRAPH); /* 676 KiB of receive buffers */
+    CHECK(sparbit_plan_exec_mode(plan) == SPARBIT_EXEC_MIRROR); /* 676 KiB of receive buffers in 4 KiB blocks: a cluster of CTAs */
     {
         uint64_t v = 0;
         CHECK(sparbit_plan_get_tunable(plan, SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES, &v) == SPARBIT_OK && v == 8192);

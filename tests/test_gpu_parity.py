@@ -312,7 +312,8 @@ def test_mirror_all_algorithms_changing_data(dev, algo):
     """The mirror executor on every algorithm it takes, up to the largest receive space that
     fits one SM's shared memory, at misaligned addresses too, with new data on every call."""
     for P, m in ((8, 64), (6, 4096), (13, 1024), (16, 800), (2, 32768), (1, 4096), (12, 100), (7, 4500),
-                 (16, 4096), (13, 8192), (32, 1000), (64, 208), (128, 64), (100, 96), (253, 24)):
+                 (16, 4096), (13, 8192), (32, 1000), (64, 208), (128, 64), (100, 96), (253, 24),
+                 (40, 100), (40, 70), (40, 75)):   # the last three: clusters on 4-, 2- and 1-byte vectors
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
             continue
         if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
@@ -324,6 +325,9 @@ def test_mirror_all_algorithms_changing_data(dev, algo):
         run_case(dev, P, m, algo, sp.EXEC_MIRROR, sp.COPY_AUTO, 90 + P, iters=3, ran=sp.EXEC_MIRROR)
     run_case(dev, 9, 96, algo if algo != sp.ALGO_RECURSIVE_DOUBLING and algo != sp.ALGO_NEIGHBOR_EXCHANGE
              else sp.ALGO_SPARBIT, sp.EXEC_MIRROR, sp.COPY_AUTO, 5, iters=1, shift_send=4, shift_recv=8)
+    if algo in (sp.ALGO_SPARBIT, sp.ALGO_BRUCK):
+        run_case(dev, 40, 96, algo, sp.EXEC_MIRROR, sp.COPY_AUTO, 6, iters=2, shift_send=4, shift_recv=8, ran=sp.EXEC_MIRROR)
+        run_case(dev, 40, 96, algo, sp.EXEC_MIRROR, sp.COPY_AUTO, 7, iters=2, shift_send=2, shift_recv=6, ran=sp.EXEC_MIRROR)
 
 
 def test_mirror_runs_where_it_fits_and_hands_over_where_not(dev):
@@ -460,6 +464,26 @@ def test_persistent_trace_gives_one_stamp_per_pass(dev, copy):
     plan.set_trace(False)
     plan.allgather(send, recv)
     assert plan.status() == sp.OK and len(plan.get_trace()) == 0
+
+
+def test_cluster_mirror_wait_gives_up_instead_of_hanging(dev):
+    """The cluster form of the mirror executor waits for a pass's bytes on mbarriers: with more bytes
+    expected than ever arrive every wait must time out, the status word must say so, and the plan
+    must work again afterwards."""
+    P, m = 64, 64
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
+    host_send = si.send_blocks(P, m, 3)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.set_mbarrier_test(16, 5_000_000)   # 5 ms
+    plan.allgather(send, recv)
+    assert plan.status() == sp.ERR_TIMEOUT
+    plan.set_mbarrier_test(0, 0)
+    recv.fill_(si.SENTINEL)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_MIRROR
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
 
 
 @pytest.mark.parametrize("exec_mode", [sp.EXEC_PERSISTENT, sp.EXEC_STREAM])

@@ -139,9 +139,10 @@ def test_exec_mode_resolution():
     assert sp.Plan(32, 128).exec_mode == sp.EXEC_MIRROR          # 128 KiB, small blocks: a cluster of CTAs
     assert sp.Plan(128, 64).exec_mode == sp.EXEC_MIRROR          # 1 MiB: still
     assert sp.Plan(128, 128).exec_mode == sp.EXEC_GRAPH          # 2 MiB: the chain is faster
-    assert sp.Plan(16, 4096).exec_mode == sp.EXEC_GRAPH          # 1 MiB of large blocks: the chain too
-    assert sp.Plan(16, 4096, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
-    assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_GRAPH      # 144 KiB
+    assert sp.Plan(16, 4096).exec_mode == sp.EXEC_MIRROR         # 1 MiB of 4 KiB blocks: the last that gain
+    assert sp.Plan(8, 8192).exec_mode == sp.EXEC_GRAPH           # 512 KiB of larger blocks: the chain
+    assert sp.Plan(8, 8192, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
+    assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR     # 144 KiB, and as much of working buffers
     assert sp.Plan(8, 64, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR
     assert sp.Plan(256, 65536).exec_mode == sp.EXEC_GRAPH         # 8.6 GB moved: chain + bulk engine
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
