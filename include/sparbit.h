@@ -105,8 +105,9 @@ enum {
                                     starts a pass when the bytes its ranks receive in the passes
                                     before have arrived (one mbarrier per pass counts them; bounded
                                     wait, time-out through sparbit_plan_status).  Needs
-                                    ceil(P/16)*P*m to fit one SM, fixed-size blocks and at most 16
-                                    passes; other calls run as GRAPH */
+                                    ceil(P/16)*P*m to fit one SM, fixed-size blocks, at most 16
+                                    passes and a call that starts at the first pass (the on-chip
+                                    copy starts empty); other calls run as GRAPH */
 };
 
 /* Which copy engine a phase uses. */

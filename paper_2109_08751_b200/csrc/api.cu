@@ -414,7 +414,7 @@ constexpr uint32_t kMirrorMaxCluster = 16;  // the largest cluster a B200 places
 // into the shared memory of one CTA, or of the CTAs of one cluster, together.
 bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_limit) {
     if (p->variable) return false;
-    if (first != -1 || last != p->sched.last_phase()) return false;
+    if (first != -1) return false;  // the on-chip copy starts empty: a call has to begin at the beginning
     const ExecSeq seq = make_seq(p, first, last);
     if (seq.count() < 1 || seq.count() > kMirrorMaxPasses) return false;
     return mirror_smem_per_cta(p, kMirrorMaxCluster) <= (unsigned __int128)smem_limit;

@@ -166,6 +166,37 @@ def test_state_after_every_phase(dev, algo, P, exec_mode):
             assert np.array_equal(work.cpu().numpy(), scratch), ph
 
 
+@pytest.mark.parametrize("algo,P", [(sp.ALGO_SPARBIT, 5), (sp.ALGO_SPARBIT, 21), (sp.ALGO_SPARBIT, 32),
+                                    (sp.ALGO_SPARBIT, 61), (sp.ALGO_BRUCK, 13), (sp.ALGO_BRUCK, 24),
+                                    (sp.ALGO_RING, 6), (sp.ALGO_RECURSIVE_DOUBLING, 32),
+                                    (sp.ALGO_NEIGHBOR_EXCHANGE, 28)])
+def test_mirror_state_after_every_prefix(dev, algo, P):
+    """The mirror executor takes calls that start at the beginning (its on-chip copy starts empty): run
+    passes -1..k for every k, each time into sentinel-filled buffers; the whole state in global memory
+    (receive and working buffers, sentinel included) must be the oracle's after step k.  P = 5..24
+    run in one CTA, P = 28..61 on a cluster (Bruck at 24 too: twice the shared memory)."""
+    m = 272
+    plan = sp.Plan(P, m, algo, sp.EXEC_MIRROR)
+    ref = oracle.Plan(algo, P)
+    host_send = si.send_blocks(P, m, 78)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.empty((P * P * m,), dtype=torch.uint8, device=dev)
+    work = torch.empty((P * P * m,), dtype=torch.uint8, device=dev)
+    if algo == sp.ALGO_BRUCK:
+        plan.set_workspace(work, P * P * m)
+    for k in range(-1, ref.last_phase + 1):
+        recv.fill_(si.SENTINEL)
+        work.fill_(si.SENTINEL)
+        plan.allgather_steps(send, recv, -1, k)
+        assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_MIRROR
+        want = si.sentinel_buffer(P * P * m)
+        scratch = si.sentinel_buffer(P * P * m)
+        ref.run(m, host_send.reshape(-1), want, scratch, first=-1, last=k)
+        assert np.array_equal(recv.cpu().numpy(), want), k
+        if algo == sp.ALGO_BRUCK:
+            assert np.array_equal(work.cpu().numpy(), scratch), k
+
+
 # ---------------------------------------------------------------- brute force over P
 ALL_IN_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 1}     # every pass in the flow kernel
 SPLIT_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 40}     # passes of fewer than 40 spans as kernels in front of it
