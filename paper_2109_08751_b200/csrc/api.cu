@@ -110,7 +110,7 @@ struct sparbit_plan_s {
         1000000000u,  // FLOW_MIN_MOVED_BYTES
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
-        0,            // FLOW_MIN_PASS_SPANS (0: one span per resident warp)
+        1,            // FLOW_MIN_PASS_SPANS (every pass; 0: passes of at least one span per resident warp)
         1u << 20,     // MIRROR_CLUSTER_MAX_BYTES
         4096,         // MIRROR_CLUSTER_MAX_BLOCK
         256,          // MIRROR_CTA_VECTORS
@@ -422,10 +422,13 @@ bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_l
 
 // Which passes of a call the flow kernel takes: the longest run of passes at the END of the
 // executed sequence that it can take (fixed-size blocks of at least 32 vectors, at most
-// kFlowMaxPasses of them) and that are large enough to keep every one of `max_warps` warps busy
-// (FLOW_MIN_PASS_SPANS warp spans in all, by default one per warp): below that a pass is bound by latency, and there a
-// kernel boundary is cheaper than a counter hand-off.  The passes before run as chained per-pass
-// kernels.  Returns the position of the first flow pass, or the sequence length if there is none.
+// kFlowMaxPasses of them) and that have at least FLOW_MIN_PASS_SPANS warp spans in all (0 stands
+// for one per resident warp).  The passes before run as chained per-pass kernels.  A small pass
+// alone is cheaper behind a kernel boundary than behind a counter hand-off, but in the collectives
+// the flow executor is chosen for (1 GB moved and more) taking every pass measured equal or up to
+// 2 % faster than any split (one launch instead of several, and the small passes overlap their
+// neighbours), so the default is 1.  Returns the position of the first flow pass, or the sequence
+// length if there is none.
 int flow_first_pass(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint64_t max_warps) {
     const int n = seq.count();
     int f = n;

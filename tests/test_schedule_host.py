@@ -208,9 +208,10 @@ def test_flow_units_and_counters_are_consistent(algo):
             if P > 256 and m > 4096:
                 continue
             plan = sp.Plan(P, m, algo)
+            plan.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)   # a pass needs one span per resident warp
             passes = plan.last_phase + 2 - (1 if algo != sp.ALGO_BRUCK and P > 1 else 0)   # fused first pass
             firsts = []
-            for warps in (1, 64, 4736):   # by default a pass needs one span per resident warp
+            for warps in (1, 64, 4736):
                 code = plan.validate_flow(vb, warps)
                 assert code in (sp.OK, sp.ERR_UNSUPPORTED)
                 if warps == 1:
@@ -222,4 +223,6 @@ def test_flow_units_and_counters_are_consistent(algo):
     assert ran > 60
     assert sp.Plan(8, 64).validate_flow(16, 1) == sp.ERR_UNSUPPORTED   # blocks shorter than a warp row
     big = sp.Plan(256, 4096)
+    assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 0   # by default every pass
+    big.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)
     assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 3   # 8192 spans in pass 3
