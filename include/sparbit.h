@@ -357,9 +357,11 @@ int sparbit_plan_launch_counts(const sparbit_plan_t* plan, uint64_t* kernel_laun
 
 /*
  * Synchronises the plan's last stream and reports the device status word: SPARBIT_OK, or
- * SPARBIT_ERR_TIMEOUT if a grid barrier of the persistent executor gave up (all CTAs then left
- * the kernel early and the receive buffers are incomplete).  Clears the condition so the plan
- * can be used again.  *device_status (may be NULL) receives the raw word.
+ * SPARBIT_ERR_TIMEOUT if a wait inside a kernel gave up (the kernel then returned early and the
+ * receive buffers are incomplete).  Clears the condition so the plan can be used again.
+ * *device_status (may be NULL) receives the raw word: 0 = none; 1 = a grid barrier of the
+ * persistent executor or a wait of the flow executor for a rank's counters; 2 = a wait for bytes
+ * on an mbarrier (bulk engine, cluster form of the mirror executor).
  */
 int sparbit_plan_status(sparbit_plan_t* plan, int* device_status);
 

@@ -323,6 +323,30 @@ def test_flow_wait_gives_up_instead_of_hanging(dev):
         assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
 
 
+def test_two_flow_collectives_at_once(dev):
+    """Two plans, two streams, both on the flow executor at the same time.  Each kernel's waits
+    need all of its CTAs resident; the cooperative launch sees to that (the second kernel starts
+    when the first has left room), so both must finish, and with the right bytes."""
+    cases = [(64, 16384, 11), (48, 32768, 12)]
+    plans, sends, recvs, streams, wants = [], [], [], [], []
+    for P, m, seed in cases:
+        plans.append(sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_FLOW))
+        host_send = si.send_blocks(P, m, seed)
+        sends.append(torch.from_numpy(host_send.reshape(-1)).to(dev))
+        recvs.append(torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev))
+        streams.append(torch.cuda.Stream(device=dev))
+        wants.append(host_send.reshape(-1))
+    torch.cuda.synchronize()
+    for it in range(6):
+        for plan, send, recv, st in zip(plans, sends, recvs, streams):
+            plan.allgather(send, recv, st)
+    for (P, m, _), plan, recv, want in zip(cases, plans, recvs, wants):
+        assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_FLOW
+        got = recv.cpu().numpy().reshape(P, P * m)
+        assert all(np.array_equal(got[r], want) for r in range(P))
+        plan.destroy()
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_flow_all_algorithms_changing_data(dev, algo):
     """Every algorithm on the flow executor, several calls in a row on one plan (the counters
