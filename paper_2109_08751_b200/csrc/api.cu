@@ -653,7 +653,11 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        // The bulk kernel lets its dependents launch at once; across two calls that would bring the
+        // next collective's kernels onto the SMs while this one's last, largest pass still needs
+        // every slot (measured: 242 us against 175 at P = 256, m = 8 KiB back to back).  So the first
+        // kernel of a call on that engine is an ordinary launch.
+        cfg.numAttrs = (i == 0 && rs.copy == SPARBIT_COPY_BULK) ? 0 : 1;
         PhaseArgs a;
         a.g = g;
         a.d = seq.item(i);
