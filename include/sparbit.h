@@ -75,7 +75,7 @@ enum {
  * the first peer's): same state after phase 0, one pass less. */
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
-                                    buffers in all (up to 1 MiB for blocks of at most 4 KiB),
+                                    buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB),
                                     FLOW for collectives that move 1 to 6 GB, the graph chain
                                     otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
@@ -335,9 +335,11 @@ enum {
                                               or up to 2 % faster than any split; 0: one per resident
                                               warp, 4736 on B200); smaller leading passes run as chained
                                               per-pass kernels in front of it */
-    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BYTES = 8, /* EXEC_AUTO: MIRROR on a cluster of CTAs when P*P*m is at most
-                                              this (1 MiB) ... */
-    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and m at most this (4 KiB) */
+    SPARBIT_TUNE_MIRROR_MAX_VECTORS = 8,   /* EXEC_AUTO: MIRROR only when the largest pass moves at most this
+                                              many vectors (40960: 1 MiB of receive buffers in 16-byte
+                                              vectors) ... */
+    SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and, where P*P*m exceeds MIRROR_MAX_BYTES, m is at most
+                                              this (4 KiB) */
     SPARBIT_TUNE_MIRROR_CTA_VECTORS = 10,  /* EXEC_MIRROR: the cluster is doubled while a CTA would get more
                                               vectors than this in the largest pass (256) */
     SPARBIT_TUNE_MIRROR_THREAD_VECTORS = 11, /* EXEC_MIRROR: vectors of the largest pass per thread (4), CTAs

@@ -111,7 +111,7 @@ struct sparbit_plan_s {
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
         1,            // FLOW_MIN_PASS_SPANS (every pass; 0: passes of at least one span per resident warp)
-        1u << 20,     // MIRROR_CLUSTER_MAX_BYTES
+        40960,        // MIRROR_MAX_VECTORS
         4096,         // MIRROR_CLUSTER_MAX_BLOCK
         256,          // MIRROR_CTA_VECTORS
         4,            // MIRROR_THREAD_VECTORS
@@ -461,8 +461,10 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //  - Up to 64 KiB of receive buffers in all, the mirror executor: one CTA, passes separated by its
 //    own barrier and fed from shared memory (P = 8, m = 64 B: 4.1 us against 6.2 for the chain;
 //    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain, and a
-//    cluster of CTAs with the copies in distributed shared memory takes over, up to 1 MiB of
-//    receive buffers with blocks of at most 4 KiB (P = 64, m = 64 B: 8.2 against 14.4; P = 128,
+//    cluster of CTAs with the copies in distributed shared memory takes over, up to 40 Ki vectors
+//    in the largest pass (1 MiB of receive buffers in 16-byte vectors; blocks of a few bytes make
+//    as many vectors of a few bytes: P = 253, m = 1 B runs on a cluster too, 14.4 against 20.2 for
+//    the chain and 36.8 in one CTA) with blocks of at most 4 KiB (P = 64, m = 64 B: 8.2 against 14.4; P = 128,
 //    m = 64 B: 10.3 against 16.4; P = 256, m = 8 B: 14.4 against 20.5; P = 16, m = 4 KiB: 8.2
 //    against 9.2): a pass is one push through the SM-to-SM network and an mbarrier, about 0.8 us.
 //    Beyond 1 MiB sixteen SMs' bandwidth eats the gain (P = 64, m = 512 B: 14.4 against 12.3).
@@ -477,18 +479,28 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.
-// Where the mirror executor is the fastest (measured): one CTA up to MIRROR_MAX_BYTES of receive
-// buffers in all, a cluster up to MIRROR_CLUSTER_MAX_BYTES when blocks are at most
-// MIRROR_CLUSTER_MAX_BLOCK bytes.
-bool mirror_wins(const sparbit_plan_s* p) {
+// Where the mirror executor is the fastest (measured): what decides is the number of vectors of
+// the largest pass, which sixteen SMs have to push - at most MIRROR_MAX_VECTORS (1 MiB of receive
+// buffers in 16-byte vectors; far less in blocks of a few bytes, which make vectors of a few
+// bytes) - and, beyond the MIRROR_MAX_BYTES that one CTA takes, blocks of at most
+// MIRROR_CLUSTER_MAX_BLOCK bytes (larger blocks mean few ranks and few passes: the chain is cheap).
+bool mirror_wins(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    const ExecSeq seq = make_seq(p, first, last);
+    uint64_t most = 0;
+    for (int i = 0; i < seq.count(); i++) {
+        const PhaseDesc& d = seq.item(i);
+        const uint64_t v = (uint64_t)p->sched.P * d.copies * (d.copy_bytes / (uint64_t)vbytes);
+        if (v > most) most = v;
+    }
+    if (most > p->tune[SPARBIT_TUNE_MIRROR_MAX_VECTORS]) return false;
     const unsigned __int128 all = (unsigned __int128)p->sched.P * p->sched.P * p->sched.m;
-    if (all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) return true;
-    return all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BYTES] &&
+    return all <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] ||
            p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK];
 }
 
 int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
-    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) && mirror_wins(p)) return SPARBIT_EXEC_MIRROR;
+    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) && mirror_wins(p, vbytes, first, last))
+        return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
@@ -497,7 +509,8 @@ int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
 }
 
 int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
-    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) && mirror_wins(p)) return SPARBIT_EXEC_MIRROR;
+    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) && mirror_wins(p, vbytes, -1, p->sched.last_phase()))
+        return SPARBIT_EXEC_MIRROR;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
@@ -858,13 +871,16 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         ma.magic_vpc[i] = ((1ull << 40) + vpc - 1) / (vpc ? vpc : 1);
         ma.magic_copies[i] = ((1ull << 40) + ma.d[i].copies - 1) / (ma.d[i].copies ? ma.d[i].copies : 1);
     }
-    // One CTA while everything fits and is small enough for it (MIRROR_MAX_BYTES); else the smallest
-    // cluster that holds it and leaves a CTA at most MIRROR_CTA_VECTORS vectors in the largest pass.
+    // One CTA while everything fits and is small enough for it (MIRROR_MAX_BYTES, and at most
+    // eight times MIRROR_CTA_VECTORS vectors in the largest pass: blocks of a few bytes make many
+    // vectors of few bytes); else the smallest cluster that holds it and leaves a CTA at most
+    // MIRROR_CTA_VECTORS vectors in the largest pass.
     uint32_t C = 1;
     const unsigned __int128 limit = (unsigned __int128)p->max_smem_optin;
+    const bool spread = mirror_smem_per_cta(p, 1) > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] ||
+                        most > 8 * p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS];
     while (C < kMirrorMaxCluster &&
-           (mirror_smem_per_cta(p, C) > limit || (C < P && mirror_smem_per_cta(p, 1) > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] &&
-            most / C > p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS])))
+           (mirror_smem_per_cta(p, C) > limit || (C < P && spread && most / C > p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS])))
         C *= 2;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
