@@ -507,7 +507,15 @@ def run_sweep(args):
              "flow": sp.EXEC_FLOW, "mirror": sp.EXEC_MIRROR}
     if args.sweep == "engines":
         execs = {"graph": sp.EXEC_GRAPH, "flow": sp.EXEC_FLOW}
-    copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
+    if args.sweep == "mirror":  # where the mirror executor (one CTA, then a cluster) wins and where it stops winning
+        points += [(P, m, ["sparbit"]) for P, m in (
+            (8, 64), (16, 64), (32, 64), (64, 64), (128, 64), (64, 256), (32, 512), (45, 512), (16, 1024),
+            (8, 4096), (16, 4096), (256, 8), (253, 1), (253, 3), (128, 128), (64, 512), (100, 200), (181, 64),
+            (4, 16384), (8, 8192))]
+        execs = {"graph": sp.EXEC_GRAPH, "mirror": sp.EXEC_MIRROR}
+        copies = {"vector": sp.COPY_VECTOR}
+    else:
+        copies = {"vector": sp.COPY_VECTOR, "bulk": sp.COPY_BULK}
     stream = torch.cuda.Stream(device=dev)
     cores = min(os.cpu_count() or 1, 16)
     for P, m, names in points:
@@ -531,8 +539,8 @@ def run_sweep(args):
                     continue  # same kernels as the graph chain; skipped to bound the sweep
                 if cname == "bulk" and (m % 16 or ename in ("flow", "mirror")):
                     continue
-                if ename == "mirror" and P * P * m > (224 << 10):
-                    continue
+                if ename == "mirror" and (P + 15) // 16 * P * m > (224 << 10):
+                    continue  # fits no cluster
                 plan = sp.Plan(P, m, algos[name], e)
                 plan.set_copy_path(c)
                 if name == "bruck":
@@ -734,7 +742,7 @@ def main():
                          "(0 = one round, for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "all"], default=None,
+    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "mirror", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     ap.add_argument("--sweep-auto-only", action="store_true",
                     help="with --sweep: only the executor and engine the library picks by itself")
