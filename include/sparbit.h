@@ -76,21 +76,21 @@ enum {
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
                                     buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB),
-                                    FLOW for collectives that move 1 to 6 GB, the graph chain
+                                    FLOW for collectives that move 0.45 to 6 GB, the graph chain
                                     otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
                                     re-parameterise the least recently used graph) */
     SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
-    SPARBIT_EXEC_FLOW = 4,       /* one cooperative kernel without grid barriers: Algorithm 1's
-                                    Waitall is kept per rank (counters of what each rank has
-                                    received), so a pass starts where its senders are ready while
-                                    the pass before is still finishing elsewhere.  Leading passes
-                                    too small to keep every warp busy run as chained per-pass
-                                    kernels in front of it.  Whole collectives of fixed-size
-                                    blocks of at least 32 vectors on the vector engine; other
-                                    calls run as GRAPH */
+    SPARBIT_EXEC_FLOW = 4,       /* one kernel (all CTAs resident) without grid barriers:
+                                    Algorithm 1's Waitall is kept per rank (counters of what each
+                                    rank has received), so a pass starts where its senders are
+                                    ready while the pass before is still finishing elsewhere.
+                                    Takes every pass by default (SPARBIT_TUNE_FLOW_MIN_PASS_SPANS
+                                    leaves small leading passes to chained per-pass kernels).
+                                    Whole collectives of fixed-size blocks of at least 32 vectors
+                                    on the vector engine; other calls run as GRAPH */
     SPARBIT_EXEC_MIRROR = 5      /* a whole small collective in ONE CTA: every block written to a
                                     receive buffer is also kept in an on-chip copy of the receive
                                     buffers (shared memory), and every forwarded block is read from
@@ -326,7 +326,7 @@ enum {
     SPARBIT_TUNE_FLOW_UNITS_PER_WARP = 2,  /* EXEC_FLOW: a pass is cut into units of 1..4 warp spans
                                               so that every warp gets at least about this many (1) */
     SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS = 3,  /* EXEC_FLOW: largest unit, in warp spans of 1 KiB (8) */
-    SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (10^9) */
+    SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (4.5*10^8) */
     SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES = 5, /* ... and below this (6*10^9); GRAPH otherwise */
     SPARBIT_TUNE_MIRROR_MAX_BYTES = 6,     /* EXEC_AUTO: MIRROR when P*P*m is at most this (64 KiB) */
     SPARBIT_TUNE_FLOW_MIN_PASS_SPANS = 7,  /* EXEC_FLOW: the flow kernel takes the passes at the end of
@@ -344,7 +344,13 @@ enum {
                                               vectors than this in the largest pass (256) */
     SPARBIT_TUNE_MIRROR_THREAD_VECTORS = 11, /* EXEC_MIRROR: vectors of the largest pass per thread (4), CTAs
                                               of at most 1024 threads */
-    SPARBIT_TUNE_COUNT_ = 12
+    SPARBIT_TUNE_FLOW_COOPERATIVE = 12,    /* EXEC_FLOW: 1 = every launch of the flow kernel is a cooperative
+                                              launch; 0 (default) = only the first one and those that go to
+                                              another stream than the flow launch before (any plan, same
+                                              device): launches that follow one another in ONE stream are
+                                              ordered anyway, start ahead of their predecessor's end and save
+                                              2-2.5 us each */
+    SPARBIT_TUNE_COUNT_ = 13
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

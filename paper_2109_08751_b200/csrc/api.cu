@@ -107,7 +107,7 @@ struct sparbit_plan_s {
         1000000000u,  // BULK_MIN_MOVED_BYTES
         1,            // FLOW_UNITS_PER_WARP
         8,            // FLOW_MAX_UNIT_SPANS
-        1000000000u,  // FLOW_MIN_MOVED_BYTES
+        450000000u,   // FLOW_MIN_MOVED_BYTES
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
         1,            // FLOW_MIN_PASS_SPANS (every pass; 0: passes of at least one span per resident warp)
@@ -115,6 +115,7 @@ struct sparbit_plan_s {
         4096,         // MIRROR_CLUSTER_MAX_BLOCK
         256,          // MIRROR_CTA_VECTORS
         4,            // MIRROR_THREAD_VECTORS
+        0,            // FLOW_COOPERATIVE
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -473,9 +474,11 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
 //    - are most of it), so there the host's cost decides: one graph launch (2.6 us) instead of one
 //    launch per pass (4 us each).  The graph chain it is.
-//  - From about 1 GB moved (150 us and more) the flow executor is 1-4 % ahead of the chain: the
-//    start-up and drain of every pass overlap with its neighbours (P = 1000, m = 1 KiB: 323 us
-//    against 334; P = 512, m = 4 KiB: 334 against 347; P = 128, m = 64 KiB: 333 against 338).
+//  - From about 0.45 GB moved (80 us and more) the flow executor is 1-4 % ahead of the chain: the
+//    start-up and drain of every pass overlap with its neighbours (P = 256, m = 4 KiB: 90.9 us
+//    against 92.5; P = 1000, m = 1 KiB: 324.7 against 336.5; P = 509, m = 4 KiB: 331.1 against
+//    347.1; P = 128, m = 64 KiB: 332.4 against 338.7 on the bulk engine).  At 0.27 GB it is
+//    behind (P = 128, m = 8 KiB: 48.7 against 47.1).
 //  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.
@@ -984,6 +987,15 @@ uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int f, int
 
 // The collective's small leading passes as chained per-pass kernels, all the others in one
 // cooperative kernel without grid barriers (flow_vec_kernel).
+// the stream the last flow kernel of this process went to, per device
+constexpr int kFlowDevices = 64;
+struct FlowStream {
+    bool seen = false;
+    cudaStream_t stream = nullptr;
+};
+std::mutex g_flow_mutex;
+FlowStream g_flow_last[kFlowDevices];
+
 int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
@@ -1026,21 +1038,32 @@ int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first,
     const PhaseDesc* descs = p->d_descs;
     int first_idx = (int)seq.table_index(f);
     void* args[] = {&gg, &descs, &first_idx, &fa};
-    // cooperative (all CTAs resident: the waits inside depend on it) and, like the per-pass kernels,
-    // launched ahead behind its predecessor in the stream
+    // The waits inside need all CTAs of the grid resident.  A cooperative launch guarantees that,
+    // but cannot start ahead of its predecessor's end as the per-pass kernels do (2-2.5 us per
+    // collective).  An ordinary launch of a grid that fits the device is just as safe as long as
+    // no other kernel of this kind can hold part of the SMs at the same time: kernels in ONE
+    // stream are ordered (the successor's CTAs only wait for the predecessor's end), and every
+    // other kernel of this library finishes without waiting for anybody.  So: an ordinary launch
+    // when the flow launch before this one (any plan, this device) went to the same stream, a
+    // cooperative one otherwise - that one starts only when it fits as a whole, behind or in
+    // front of the other stream's kernel, never interleaved with it.
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kVecBlock);
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    std::lock_guard<std::mutex> lock(g_flow_mutex);
+    FlowStream& prev = g_flow_last[p->device >= 0 && p->device < kFlowDevices ? p->device : 0];
+    cfg.numAttrs = (prev.seen && prev.stream == st && !p->tune[SPARBIT_TUNE_FLOW_COOPERATIVE]) ? 1 : 2;
     CU(cudaLaunchKernelExC(&cfg, fn, args));
+    prev.seen = true;
+    prev.stream = st;
     p->kernel_launches++;
     return SPARBIT_OK;
 }
