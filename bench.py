@@ -306,25 +306,33 @@ def run_ours(args):
             time.sleep(0.25)
         k0, g0 = plan.launch_counts()
         round_ms, per_ms = [], []
-        # a time stamp between every two collectives costs about 2 us of GPU time: taken only where
-        # a collective is long enough not to notice (else min/avg/max are over the rounds)
+        # A time stamp between every two collectives costs about 2 us of GPU time (the next
+        # collective's first kernel can no longer start ahead of the last one's end), so the timed
+        # rounds carry two stamps each; the spread of single collectives comes from one extra
+        # stamped round after the timed region, where a collective is long enough to stand it.
         stamp_each = est_ms / args.steps >= 0.1
         t_wall0 = time.time()
         for _ in range(rounds):
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             barrier()
+            e0.record(stream)
+            for it in range(args.steps):
+                plan.allgather(sends[it & 1], recv, stream)
+            e1.record(stream)
+            stream.synchronize()
+            barrier()
+            round_ms.append(max_over_ranks(e0.elapsed_time(e1), dev, use_dist))
+            per_ms.append(e0.elapsed_time(e1) / args.steps)
+        t_wall1 = time.time()
+        k1, g1 = plan.launch_counts()
+        if stamp_each:
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
             ev[0].record(stream)
             for it in range(args.steps):
                 plan.allgather(sends[it & 1], recv, stream)
-                if stamp_each or it == args.steps - 1:
-                    ev[it + 1].record(stream)
+                ev[it + 1].record(stream)
             stream.synchronize()
-            barrier()
-            round_ms.append(max_over_ranks(ev[0].elapsed_time(ev[-1]), dev, use_dist))
-            per_ms += ([ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)] if stamp_each
-                       else [ev[0].elapsed_time(ev[-1]) / args.steps])
-        t_wall1 = time.time()
-        k1, g1 = plan.launch_counts()
+            per_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     assert plan.status() == sp.OK
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ran_exec, ran_copy = plan.exec_mode, plan.copy_path   # what the timed collectives ran on
@@ -377,7 +385,7 @@ def run_ours(args):
         per_pass_us = [round(float(x) / 1e3, 1) for x in np.diff(stamps)]
         plan.set_trace(False)
     if one_kernel:
-        dom_ms = float(np.mean(per_ms))
+        dom_ms = float(np.mean(round_ms)) / args.steps   # the timed rounds (no stamps in between)
         dom_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
         dom_name = ("whole collective in one kernel" if launches_per_step <= 1 else
                     f"whole collective: the flow kernel behind {launches_per_step - 1:g} small per-pass kernel(s)")
@@ -399,7 +407,7 @@ def run_ours(args):
 
     if rank == 0:
         peak, peak_src = measured_peak()
-        avg_ms = float(np.mean(per_ms))
+        avg_ms = float(np.mean(round_ms)) / args.steps   # the timed rounds (no stamps in between)
         path_bytes = algorithmic_bytes(P, m, algo != sp.ALGO_BRUCK)
         achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
         key = f"{args.algo}:P{P}:m{m}:{sp.EXEC_NAMES[ran_exec]}:{sp.COPY_NAMES[ran_copy]}"
@@ -426,7 +434,9 @@ def run_ours(args):
             "rounds": rounds, "timed_ms": float(sum(round_ms)),
             "ms_per_step_rounds": {"min": min(round_ms) / args.steps, "median": ms_per_step,
                                    "max": max(round_ms) / args.steps},
-            "us_per_collective": {"min": min(per_ms) * 1e3, "avg": avg_ms * 1e3, "max": max(per_ms) * 1e3},
+            "us_per_collective": {"min": min(per_ms) * 1e3, "avg": avg_ms * 1e3, "max": max(per_ms) * 1e3,
+                                  "min_max_from": ("one extra round with a time stamp after every collective, "
+                                                   "outside the timed region" if stamp_each else "the timed rounds")},
             "pct_of_hbm_peak": 100.0 * value / world / peak,
             "pct_of_nominal_hbm": 100.0 * value / world / NOMINAL_HBM_GBS,
             "GBps_from_min_time": world * effective_bytes(P, m) / (min(per_ms) * 1e-3) / 1e9,
@@ -580,6 +590,53 @@ def run_sweep(args):
                     "checked": ok}), flush=True)
                 plan.destroy()
         del sends, recv, work
+        torch.cuda.empty_cache()
+    return 0
+
+
+def run_flow_wait_bound(args):
+    """What the flow executor loses to waiting of any kind: the same collectives with and without
+    the units' waits for their source rank's counters (a measurement hook of the library; without
+    them blocks are forwarded before they have arrived, so that run's result is wrong and is not
+    checked).  The difference bounds what finer readiness tracking, per (rank, slot) instead of
+    per (rank, pass), could gain.  One JSON line per point; same timing protocol as --sweep."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peak()
+    stream = torch.cuda.Stream(device=dev)
+    for P, m in ((256, 4096), (128, 16384), (256, 8192), (512, 4096), (128, 65536), (1000, 1024), (256, 32768)):
+        sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        out = {"P": P, "m": m, "GB_moved": round(effective_bytes(P, m) / 1e9, 3)}
+        for label, skip in (("graph", None), ("flow", 0), ("flow_no_waits", 1)):
+            plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_GRAPH if skip is None else sp.EXEC_FLOW)
+            if skip:
+                plan.set_tunable(sp.TUNE_FLOW_SKIP_WAITS, 1)
+            us = []
+            with torch.cuda.stream(stream):
+                for it in range(5):
+                    plan.allgather(sends[it & 1], recv, stream)
+                stream.synchronize()
+                for _ in range(10):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    for it in range(50):
+                        plan.allgather(sends[it & 1], recv, stream)
+                    e1.record(stream)
+                    stream.synchronize()
+                    us.append(e0.elapsed_time(e1) / 50 * 1e3)
+            assert plan.status() == sp.OK
+            if not skip:
+                assert bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
+            out[label + "_us"] = round(float(np.mean(us)), 2)
+            out[label + "_pct_measured_peak"] = round(100 * effective_bytes(P, m) / float(np.mean(us)) / 1e3 / peak, 1)
+            plan.destroy()
+        out["waiting_costs_pct"] = round(100 * (out["flow_us"] - out["flow_no_waits_us"]) / out["flow_us"], 2)
+        print(json.dumps(out), flush=True)
+        del sends, recv
         torch.cuda.empty_cache()
     return 0
 
@@ -754,6 +811,9 @@ def main():
     ap.add_argument("--mapping-study", action="store_true",
                     help="blocks per Sparbit step that cross devices under the sequential and cyclic "
                          "rank-to-device mappings (host only), one JSON line per (P, G, mapping)")
+    ap.add_argument("--flow-wait-bound", action="store_true",
+                    help="the flow executor with and without its waits (timing only): what any finer "
+                         "readiness tracking could gain at most")
     ap.add_argument("--allgatherv", action="store_true",
                     help="variable block sizes on the Sparbit schedule, one JSON line per size mix")
     args = ap.parse_args()
@@ -763,6 +823,8 @@ def main():
         return run_mapping_study(args)
     if args.allgatherv:
         return run_allgatherv(args)
+    if args.flow_wait_bound:
+        return run_flow_wait_bound(args)
     if args.heatmap:
         return run_heatmap(args)
     if args.sweep:

@@ -350,7 +350,13 @@ enum {
                                               device): launches that follow one another in ONE stream are
                                               ordered anyway, start ahead of their predecessor's end and save
                                               2-2.5 us each */
-    SPARBIT_TUNE_COUNT_ = 13
+    SPARBIT_TUNE_FLOW_SKIP_WAITS = 13,     /* measurement hook, EXEC_FLOW: 1 = no unit waits for its source
+                                              rank's counters.  The receive buffers are then WRONG (blocks
+                                              are forwarded before they have arrived); the time is what the
+                                              kernel would take if waiting cost nothing, the bound on what any
+                                              finer readiness tracking could gain (bench.py
+                                              --flow-wait-bound).  0 by default */
+    SPARBIT_TUNE_COUNT_ = 14
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

@@ -116,6 +116,7 @@ struct sparbit_plan_s {
         256,          // MIRROR_CTA_VECTORS
         4,            // MIRROR_THREAD_VECTORS
         0,            // FLOW_COOPERATIVE
+        0,            // FLOW_SKIP_WAITS
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -977,6 +978,7 @@ uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int f, int
         fp.dep_mask = 0;  // passes before f are complete when the kernel starts (stream order)
         for (int k = 0; k < i; k++)
             if (seq.item(f + k).dst_space == d.src_space) fp.dep_mask |= 1u << k;
+        if (p->tune[SPARBIT_TUNE_FLOW_SKIP_WAITS]) fp.dep_mask = 0;  // measurement hook: wrong results, timing only
         if ((uint64_t)P * fp.upr > most_units) most_units = (uint64_t)P * fp.upr;
         fp.eager = (uint64_t)P * fp.upr <= max_warps ? 1u : 0u;
         // the next pass starts its enumeration where this pass's first receivers are
