@@ -641,6 +641,51 @@ def run_flow_wait_bound(args):
     return 0
 
 
+def run_placement_study(args):
+    """The same collective (Sparbit, --P, --m, executor and engine as AUTO picks them), timed with
+    the receive buffer at different places in device memory: before it is allocated, a pad of the
+    given size is allocated and kept.  Same protocol as --sweep.  One JSON line per pad size."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peak()
+    P, m = args.P, args.m
+    stream = torch.cuda.Stream(device=dev)
+    for pad_mib in (0, 2, 64, 256, 512, 1024, 1536):
+        torch.cuda.empty_cache()
+        pad = torch.empty(max(pad_mib << 20, 1), dtype=torch.uint8, device=dev)
+        sends = [torch.from_numpy(si.send_blocks(P, m, args.seed + k).reshape(-1)).to(dev) for k in range(2)]
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        plan = sp.Plan(P, m)
+        us = []
+        with torch.cuda.stream(stream):
+            for it in range(5):
+                plan.allgather(sends[it & 1], recv, stream)
+            stream.synchronize()
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for it in range(50):
+                    plan.allgather(sends[it & 1], recv, stream)
+                e1.record(stream)
+                stream.synchronize()
+                us.append(e0.elapsed_time(e1) / 50 * 1e3)
+        assert plan.status() == sp.OK
+        ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
+        avg = float(np.mean(us))
+        print(json.dumps({"P": P, "m": m, "pad_MiB": pad_mib,
+                          "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
+                          "recv_address": hex(recv.data_ptr()),
+                          "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
+                          "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
+                          "checked": ok}), flush=True)
+        plan.destroy()
+        del sends, recv, pad
+    return 0
+
+
 def run_allgatherv(args):
     """Blocks of different sizes on the Sparbit schedule (P = 256, about 64 KiB per block on
     average): equal sizes through the variable-size path, uniformly drawn sizes, and a mix with
@@ -814,6 +859,8 @@ def main():
     ap.add_argument("--flow-wait-bound", action="store_true",
                     help="the flow executor with and without its waits (timing only): what any finer "
                          "readiness tracking could gain at most")
+    ap.add_argument("--placement-study", action="store_true",
+                    help="the same collective with its receive buffer at different places in device memory")
     ap.add_argument("--allgatherv", action="store_true",
                     help="variable block sizes on the Sparbit schedule, one JSON line per size mix")
     args = ap.parse_args()
@@ -825,6 +872,8 @@ def main():
         return run_allgatherv(args)
     if args.flow_wait_bound:
         return run_flow_wait_bound(args)
+    if args.placement_study:
+        return run_placement_study(args)
     if args.heatmap:
         return run_heatmap(args)
     if args.sweep:
