@@ -323,6 +323,37 @@ def test_flow_wait_gives_up_instead_of_hanging(dev):
         assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
 
 
+def test_flow_launch_forms_and_the_measurement_hook(dev):
+    """The flow kernel as a cooperative launch every time (the tunable), as an ordinary launch
+    behind a flow launch in the same stream (the default from the second call on), and with its
+    waits switched off (a measurement hook: the call must complete and report no error; its result
+    is wrong by design and is not looked at)."""
+    P, m = 48, 8192
+    host_send = si.send_blocks(P, m, 21)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+    for coop in (1, 0):
+        plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_FLOW)
+        plan.set_tunable(sp.TUNE_FLOW_COOPERATIVE, coop)
+        for _ in range(3):
+            recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+            plan.allgather(send, recv)
+            assert plan.status() == sp.OK and plan.exec_mode == sp.EXEC_FLOW
+            assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+        plan.destroy()
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, sp.EXEC_FLOW)
+    plan.set_tunable(sp.TUNE_FLOW_SKIP_WAITS, 1)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    plan.set_tunable(sp.TUNE_FLOW_SKIP_WAITS, 0)
+    recv.fill_(si.SENTINEL)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+    plan.destroy()
+
+
 def test_two_flow_collectives_at_once(dev):
     """Two plans, two streams, both on the flow executor at the same time.  Each kernel's waits
     need all of its CTAs resident; the cooperative launch sees to that (the second kernel starts
