@@ -421,7 +421,8 @@ int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint
  * stream as for sparbit_allgather.  Unlike sparbit_allgather it WAITS: the work is enqueued on
  * `stream`, then the call synchronises that stream, on every call, and the return value is
  * final - SPARBIT_OK, or SPARBIT_ERR_TIMEOUT if the grid barrier gave up (recvbuf is then
- * incomplete).
+ * incomplete).  Because it waits it cannot be used on a stream that is being captured: such a
+ * call returns SPARBIT_ERR_UNSUPPORTED and enqueues nothing.
  *
  * Limit: the array holds 28 pass descriptors, i.e. any Sparbit or recursive-doubling collective
  * this library accepts (at most 24 passes), rings of at most 29 ranks and neighbor exchanges of
@@ -429,7 +430,7 @@ int sparbit_plan_set_barrier_test(sparbit_plan_t* plan, int extra_arrivals, uint
  * Bruck needs a P*P*m workspace and is refused with SPARBIT_ERR_UNSUPPORTED.
  *
  * The first call on each device looks up the array's device address (once per device, with that
- * device current); make that first call before any stream capture begins.  All calls on a
+ * device current).  All calls on a
  * device share the one array, and it keeps what the previous call left: each call re-writes the
  * descriptors and clears the barrier words on `stream` before its kernel.  Calls whose GPU work
  * overlaps (two host threads on one device) race on the scratch: serialise them.

@@ -1716,13 +1716,18 @@ int sparbit_allgather_noalloc(int P, size_t block_bytes, int algo, const void* s
     if (!sendbuf || !recvbuf) return SPARBIT_ERR_ARG;
     if (ranges_overlap(sendbuf, send_bytes, recvbuf, recv_bytes)) return SPARBIT_ERR_ALIAS;
 
+    // this entry point waits for its stream; a capturing stream cannot be waited for
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    CU(cudaStreamIsCapturing(st, &capturing));
+    if (capturing != cudaStreamCaptureStatusNone) return SPARBIT_ERR_UNSUPPORTED;
+
     int device = -1;
     CU(cudaGetDevice(&device));
     NoallocDevice* nd = nullptr;
     rc = noalloc_setup(device, nd);
     if (rc) return rc;
     if (!nd->coop) return SPARBIT_ERR_UNSUPPORTED;
-    cudaStream_t st = (cudaStream_t)stream;
 
     // vector width from the alignment of the buffers and m (no workspace here)
     uintptr_t bits = (uintptr_t)sendbuf | (uintptr_t)recvbuf | (uintptr_t)sched.m;

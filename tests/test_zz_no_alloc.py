@@ -107,3 +107,32 @@ def test_noalloc_refuses_what_does_not_fit_its_scratch():
     assert lib.sparbit_allgather_noalloc(8, 16, sp.ALGO_SPARBIT, 4096, 4100, None) == sp.ERR_ALIAS
     assert lib.sparbit_allgather_noalloc(8, 0, sp.ALGO_SPARBIT, None, None, None) == sp.OK
     assert "limit" in lib.sparbit_strerror(sp.ERR_LIMIT).decode()
+
+
+def test_noalloc_refuses_a_capturing_stream_and_leaves_the_capture_intact():
+    """The entry point waits for its stream, which a stream under capture does not allow: the call
+    must say so before it enqueues anything, and the caller's capture must go on undisturbed."""
+    dev = torch.device("cuda", 0)
+    P, m = 8, 256
+    send = torch.from_numpy(si.send_blocks(P, m, 9).reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    other = torch.zeros(1024, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        torch.cuda.synchronize()
+        graph.capture_begin()
+        other.add_(1.0)
+        rc = binding.lib.sparbit_allgather_noalloc(P, m, sp.ALGO_SPARBIT, send.data_ptr(), recv.data_ptr(),
+                                                   ctypes.c_void_p(stream.cuda_stream))
+        other.add_(1.0)
+        graph.capture_end()
+    assert rc == sp.ERR_UNSUPPORTED
+    graph.replay()
+    torch.cuda.synchronize()
+    assert float(other[0]) == 2.0                                   # the capture held both additions
+    assert bool((recv == si.SENTINEL).all())                        # and nothing of the collective
+    rc = binding.lib.sparbit_allgather_noalloc(P, m, sp.ALGO_SPARBIT, send.data_ptr(), recv.data_ptr(),
+                                               ctypes.c_void_p(stream.cuda_stream))
+    assert rc == sp.OK
+    assert all(torch.equal(recv.view(P, P * m)[r], send) for r in range(P))
