@@ -740,6 +740,9 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
 // distributed shared memory (st.shared::cluster) and into global memory; the hardware cluster barrier
 // (arrive.release / wait.acquire) is the Waitall.  A pass costs a shared-memory read, a posted remote
 // write and that barrier.  The last barrier keeps every CTA alive until nobody writes into it any more.
+// (The barrier's release also waits for the pass's global stores, one of the two round trips the
+// mirror is there to avoid: this form runs vectors of 1 and 2 bytes only, which st.async does not
+// move; wider vectors take cluster_mirror_async_kernel below.)
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
