@@ -227,3 +227,27 @@ def test_flow_units_and_counters_are_consistent(algo):
     assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 0   # by default every pass
     big.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)
     assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 3   # 8192 spans in pass 3
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_every_rank_sends_and_receives_the_same_number_of_blocks_in_a_pass(algo):
+    """What the cluster form of the mirror executor counts on: it arms, per pass, an mbarrier in
+    every CTA with the bytes that CTA's ranks will receive, computed as ranks x blocks-per-rank x
+    block size.  That is right only if, in every pass, every rank receives exactly as many blocks
+    as every rank sends (one slot each, no slot twice)."""
+    for P in list(range(1, 40)) + [61, 64, 100, 128, 253, 256]:
+        if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
+            continue
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
+            continue
+        plan = sp.Plan(P, 16, algo)
+        for phase in range(-1, plan.last_phase + 1):
+            msgs = plan.messages(phase)
+            if len(msgs) == 0:
+                continue
+            sent = np.bincount(msgs["src_rank"], minlength=P)
+            got = np.bincount(msgs["dst_rank"], minlength=P)
+            assert (sent == sent[0]).all() and (got == sent[0]).all(), (algo, P, phase)
+            slots = set(zip(msgs["dst_space"].tolist(), msgs["dst_rank"].tolist(), msgs["dst_slot"].tolist()))
+            assert len(slots) == len(msgs), (algo, P, phase)
+        plan.destroy()
