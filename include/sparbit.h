@@ -171,9 +171,10 @@ int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_p
  * The plan is then used with sparbit_allgather, sparbit_allgather_steps and
  * sparbit_allgather_host exactly like a fixed-size plan (introspection included).  Both copy
  * engines (the bulk engine when all counts and the buffers are multiples of 16 bytes; COPY_AUTO
- * applies its thresholds to the average block) and the GRAPH, STREAM and PERSISTENT executors;
- * FLOW and MIRROR are refused (ERR_UNSUPPORTED: they assume equal blocks), and so is Bruck (its
- * rotated workspace assumes equal blocks).  P is limited to 8192 here and P * T to 2^48 bytes
+ * applies its thresholds to the average block) and the GRAPH, STREAM and PERSISTENT executors,
+ * and MIRROR in one CTA where P * T fits one SM's shared memory (EXEC_AUTO uses it up to 64 KiB;
+ * larger plans run as GRAPH).  FLOW is refused (ERR_UNSUPPORTED: its units assume equal blocks),
+ * and so is Bruck (its rotated workspace assumes equal blocks).  P is limited to 8192 here and P * T to 2^48 bytes
  * (ERR_LIMIT, ERR_OVERFLOW beyond: the plan keeps one 16-byte task record per 4 KiB of every
  * copy, with 48-bit offsets).  Other errors as for sparbit_plan_create.  Host-only.
  */

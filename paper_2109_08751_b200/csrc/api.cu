@@ -89,7 +89,6 @@ struct sparbit_plan_s {
     unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
     unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
     int flow_vbytes = 0;             // vector width those launches ran with
-    size_t mirror_smem_set[16] = {};  // dynamic shared memory already granted to the mirror kernels, by form and vector width
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -415,10 +414,13 @@ constexpr uint32_t kMirrorMaxCluster = 16;  // the largest cluster a B200 places
 // The mirror executor takes whole collectives of fixed-size blocks whose P receive buffers fit
 // into the shared memory of one CTA, or of the CTAs of one cluster, together.
 bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_limit) {
-    if (p->variable) return false;
     if (first != -1) return false;  // the on-chip copy starts empty: a call has to begin at the beginning
+    if (smem_limit < 1024) return false;
+    smem_limit -= 1024;  // the kernels' own static shared memory (mbarriers) comes out of the same limit
     const ExecSeq seq = make_seq(p, first, last);
     if (seq.count() < 1 || seq.count() > kMirrorMaxPasses) return false;
+    if (p->variable)  // blocks of different sizes: one CTA only
+        return (unsigned __int128)p->sched.P * p->voff.back() <= (unsigned __int128)smem_limit;
     return mirror_smem_per_cta(p, kMirrorMaxCluster) <= (unsigned __int128)smem_limit;
 }
 
@@ -489,6 +491,8 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 // bytes) - and, beyond the MIRROR_MAX_BYTES that one CTA takes, blocks of at most
 // MIRROR_CLUSTER_MAX_BLOCK bytes (larger blocks mean few ranks and few passes: the chain is cheap).
 bool mirror_wins(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    if (p->variable)  // one CTA: up to what one CTA takes of equal blocks
+        return (unsigned __int128)p->sched.P * p->voff.back() <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES];
     const ExecSeq seq = make_seq(p, first, last);
     uint64_t most = 0;
     for (int i = 0; i < seq.count(); i++) {
@@ -857,9 +861,88 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
 
 // The whole collective in one CTA, or in one cluster of CTAs, with the receive buffers mirrored in
 // (distributed) shared memory.
+// The mirror kernels take their dynamic shared memory up to the device's opt-in maximum.  The limit
+// is a property of the function, not of a plan: it is raised once per device and kernel, to the
+// maximum (asking for less per launch costs nothing), so that no plan can lower it under another.
+constexpr int kSmemDevices = 64;
+std::mutex g_smem_mutex;
+bool g_smem_granted[kSmemDevices][24];
+int vec_slot(int vbytes) { return vbytes == 16 ? 4 : vbytes == 8 ? 3 : vbytes == 4 ? 2 : vbytes == 2 ? 1 : 0; }
+int grant_max_smem(const sparbit_plan_s* p, const void* fn, int slot, bool big_cluster) {
+    std::lock_guard<std::mutex> lock(g_smem_mutex);
+    const int dev = p->device >= 0 && p->device < kSmemDevices ? p->device : 0;
+    if (g_smem_granted[dev][slot]) return SPARBIT_OK;
+    cudaFuncAttributes fa;
+    CU(cudaFuncGetAttributes(&fa, fn));  // the limit covers static and dynamic shared memory together
+    CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, p->max_smem_optin - (int)fa.sharedSizeBytes));
+    if (big_cluster) CU(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    g_smem_granted[dev][slot] = true;
+    return SPARBIT_OK;
+}
+
+template <typename V>
+const void* mirror_list_fn() { return (const void*)mirror_list_kernel<V>; }
+const void* pick_mirror_list(int vbytes) {
+    switch (vbytes) {
+        case 16: return mirror_list_fn<uint4>();
+        case 8: return mirror_list_fn<uint2>();
+        case 4: return mirror_list_fn<unsigned>();
+        case 2: return mirror_list_fn<unsigned short>();
+        default: return mirror_list_fn<unsigned char>();
+    }
+}
+
+// blocks of different sizes: one CTA, a warp per listed task
+int launch_mirror_list(sparbit_plan_s* p, const Resolved& rs, const Geom& g, const ExecSeq& seq, cudaStream_t st) {
+    MirrorListArgs ma;
+    memset(&ma, 0, sizeof ma);
+    ma.n = seq.count();
+    uint64_t most = 1;  // tasks of the largest pass
+    for (int i = 0; i < ma.n; i++) {
+        const PhaseDesc& d = seq.item(i);
+        const size_t ti = seq.table_index(i);
+        ma.pass[i].list = p->d_vtasks + p->vtask_lo[ti];
+        ma.pass[i].count = p->vtask_hi[ti] - p->vtask_lo[ti];
+        ma.pass[i].src_space = d.src_space;
+        ma.pass[i].dst_space = d.dst_space;
+        ma.pass[i].dup_self = d.dup_self;
+        if (ma.pass[i].count > most) most = ma.pass[i].count;
+        // lanes per task: about the vectors of an average task of this pass
+        uint64_t bytes = 0;
+        for (size_t t = p->vtask_lo[ti]; t < p->vtask_hi[ti]; t++) bytes += (p->vtasks[t].a >> 48) + 1;
+        const uint64_t avg = ma.pass[i].count ? bytes / ma.pass[i].count / (uint64_t)rs.vbytes : 1;
+        uint32_t group = 4;
+        while (group < 32 && group < avg) group *= 2;
+        ma.pass[i].group = group;
+    }
+    const void* fn = pick_mirror_list(rs.vbytes);
+    const size_t smem = (size_t)p->sched.P * p->voff.back();
+    int rc = grant_max_smem(p, fn, 16 + vec_slot(rs.vbytes), false);
+    if (rc) return rc;
+    uint64_t threads = most * 32;  // a warp per task of the largest pass, as far as a CTA goes
+    if (threads > 1024) threads = 1024;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    Geom gg = g;
+    void* args[] = {&gg, &ma};
+    CU(cudaLaunchKernelExC(&cfg, fn, args));
+    p->kernel_launches++;
+    return SPARBIT_OK;
+}
+
 int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
+    if (p->variable) return launch_mirror_list(p, rs, g, seq, st);
     MirrorArgs ma;
     memset(&ma, 0, sizeof ma);
     ma.n = seq.count();
@@ -880,7 +963,7 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
     // vectors of few bytes); else the smallest cluster that holds it and leaves a CTA at most
     // MIRROR_CTA_VECTORS vectors in the largest pass.
     uint32_t C = 1;
-    const unsigned __int128 limit = (unsigned __int128)p->max_smem_optin;
+    const unsigned __int128 limit = (unsigned __int128)p->max_smem_optin - 1024;  // as in mirror_possible
     const bool spread = mirror_smem_per_cta(p, 1) > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] ||
                         most > 8 * p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS];
     while (C < kMirrorMaxCluster &&
@@ -904,11 +987,9 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         uint64_t threads = (most / C + per_thread - 1) / per_thread;
         threads = (threads + 63) / 64 * 64;
         if (threads > 1024) threads = 1024;
-        size_t& granted = p->mirror_smem_set[(C == 1 ? 0 : 8) + (rs.vbytes == 16 ? 4 : rs.vbytes == 8 ? 3 : rs.vbytes == 4 ? 2 : rs.vbytes == 2 ? 1 : 0)];
-        if (smem > granted) {
-            CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            if (C > 8) CU(cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-            granted = smem;
+        {
+            const int grc = grant_max_smem(p, fn, (C == 1 ? 0 : 8) + vec_slot(rs.vbytes), C > 1);
+            if (grc) return grc;
         }
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(C);
@@ -1139,8 +1220,7 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     if (algo < SPARBIT_ALGO_SPARBIT || algo > SPARBIT_ALGO_NEIGHBOR_EXCHANGE) return SPARBIT_ERR_ARG;
     if (algo == SPARBIT_ALGO_BRUCK) return SPARBIT_ERR_UNSUPPORTED;  // rotated workspace: fixed sizes only
     if (exec < SPARBIT_EXEC_AUTO || exec > SPARBIT_EXEC_MIRROR) return SPARBIT_ERR_ARG;
-    if (exec == SPARBIT_EXEC_FLOW || exec == SPARBIT_EXEC_MIRROR)
-        return SPARBIT_ERR_UNSUPPORTED;  // both lay their work out for equal blocks
+    if (exec == SPARBIT_EXEC_FLOW) return SPARBIT_ERR_UNSUPPORTED;  // lays its work out for equal blocks
     sparbit_plan_s* p = new (std::nothrow) sparbit_plan_s();
     if (!p) return SPARBIT_ERR_NOMEM;
     int rc;
@@ -1220,7 +1300,7 @@ int sparbit_plan_create_v(int P, const size_t* block_bytes, int algo, int exec, 
     p->exec_req = exec;
     if (exec == SPARBIT_EXEC_AUTO) {  // variable-size plans have no flow executor
         const int e = env_exec(SPARBIT_EXEC_AUTO);
-        if (e != SPARBIT_EXEC_FLOW && e != SPARBIT_EXEC_MIRROR) p->exec_req = e;
+        if (e != SPARBIT_EXEC_FLOW) p->exec_req = e;
     }
     p->copy_req = env_copy(SPARBIT_COPY_AUTO);
     *out = p;

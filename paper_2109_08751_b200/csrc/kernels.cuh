@@ -733,6 +733,75 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
     }
 }
 
+// The same for blocks of DIFFERENT sizes (allgatherv), in one CTA: the passes' work comes as the task
+// lists the list kernels use (byte offsets inside the source and destination space, at most
+// kVarSegmentBytes each), a group of lanes per task; the on-chip copy is laid out like the receive space
+// (rank r's buffer at r times the sum of all block sizes).
+struct MirrorListPass {
+    const VarTask* list;
+    unsigned long long count;
+    uint32_t src_space, dst_space, dup_self;
+    uint32_t group;  // lanes that share a task (a power of two, 4..32): about the vectors of an average task
+};
+struct MirrorListArgs {
+    MirrorListPass pass[kMirrorMaxPasses];
+    int n;
+    int pad_[3];
+};
+
+template <typename V>
+__global__ void __launch_bounds__(1024, 1) mirror_list_kernel(Geom g, const __grid_constant__ MirrorListArgs ma) {
+    extern __shared__ __align__(16) unsigned char mirror[];
+    chain_trigger();
+    chain_wait();
+    V* mir = reinterpret_cast<V*>(mirror);
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t n_warps = blockDim.x >> 5;
+    const long long pitch = (long long)g.rank_pitch[SPACE_RECV];  // bytes of one receive buffer
+    for (int i = 0; i < ma.n; i++) {
+        if (i) __syncthreads();
+        const MirrorListPass& ps = ma.pass[i];
+        const bool from_send = ps.src_space == SPACE_SEND;
+        const char* sbase = g.base[SPACE_SEND];
+        char* dbase = g.base[SPACE_RECV];
+        const uint32_t G = ps.group, sub = lane & (G - 1u), grp = lane / G, groups = 32u / G;
+        // a warp fetches 32 task records at once (one per lane: one trip to memory instead of 32),
+        // then its groups of G lanes take them one after the other
+        // (each warp takes a contiguous slice of the list, as even as they come)
+        const uint32_t count = (uint32_t)ps.count;  // a list has fewer than 2^27 entries (host-checked)
+        const uint32_t per = (count + n_warps - 1u) / n_warps;
+        const uint32_t lo = warp * per;
+        const uint32_t hi = lo + per < count ? lo + per : count;
+        for (uint32_t t0 = lo; t0 < hi; t0 += 32u) {
+            VarTask mine;
+            mine.a = mine.b = 0;
+            if (t0 + lane < hi) mine = ld_task(ps.list + t0 + lane);
+            const uint32_t have = hi - t0 < 32u ? hi - t0 : 32u;
+            for (uint32_t k0 = 0; k0 < have; k0 += groups) {
+                const uint32_t k = k0 + grp;
+                VarTask e;
+                e.a = __shfl_sync(0xffffffffu, mine.a, (int)(k & 31u));
+                e.b = __shfl_sync(0xffffffffu, mine.b, (int)(k & 31u));
+                if (k >= have) continue;
+                const unsigned long long soff = e.a & kVarOffsetMask;
+                const unsigned long long doff = e.b & kVarOffsetMask;
+                const long long doff2 = (long long)doff + (long long)(short)(e.b >> 48) * pitch;  // dup_self: the sender's own buffer
+                const uint32_t vectors = ((uint32_t)(e.a >> 48) + 1u) / (uint32_t)sizeof(V);
+                for (uint32_t v = sub; v < vectors; v += G) {
+                    const V x = from_send ? ld_cg<V>(reinterpret_cast<const V*>(sbase + soff) + v) : mir[soff / sizeof(V) + v];
+                    mir[doff / sizeof(V) + v] = x;
+                    st_cg<V>(reinterpret_cast<V*>(dbase + doff) + v, x);
+                    if (ps.dup_self) {
+                        mir[(unsigned long long)doff2 / sizeof(V) + v] = x;
+                        st_cg<V>(reinterpret_cast<V*>(dbase + doff2) + v, x);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // The same idea on a thread-block CLUSTER, for collectives whose receive buffers fit into the
 // shared memory of up to 16 SMs together: rank r's on-chip copy lives in CTA r mod C of the cluster
 // (ranks c, c+C, c+2C, ... one after the other).  A CTA executes the copies its own ranks SEND: it

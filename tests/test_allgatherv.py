@@ -89,6 +89,8 @@ def test_create_v_errors_and_introspection():
     assert lib.sparbit_plan_create_v(4, counts, 0, 0, None) == sp.ERR_ARG
     assert lib.sparbit_plan_create_v(4, counts, sp.ALGO_BRUCK, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_FLOW, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
+    assert lib.sparbit_plan_create_v(4, counts, 0, sp.EXEC_MIRROR, ctypes.byref(out)) == sp.OK
+    assert lib.sparbit_plan_destroy(out) == sp.OK
     assert lib.sparbit_plan_create_v(4, counts, 0, 9, ctypes.byref(out)) == sp.ERR_ARG
     assert lib.sparbit_plan_create_v(3, counts, sp.ALGO_RECURSIVE_DOUBLING, 0, ctypes.byref(out)) == sp.ERR_UNSUPPORTED
     many = (ctypes.c_size_t * 8193)(*([16] * 8193))
@@ -144,10 +146,11 @@ def run_v_case(P, counts, algo, exec_mode, seed, shift=0, iters=2, copy=sp.COPY_
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("algo", V_ALGOS)
-@pytest.mark.parametrize("exec_mode", [sp.EXEC_AUTO, sp.EXEC_STREAM, sp.EXEC_PERSISTENT])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_AUTO, sp.EXEC_STREAM, sp.EXEC_PERSISTENT, sp.EXEC_MIRROR])
 @pytest.mark.parametrize("copy", [sp.COPY_VECTOR, sp.COPY_BULK])
 def test_gpu_v_parity_mixed_sizes(algo, exec_mode, copy):
-    """Both copy engines and all three executors.  Byte counts that are not multiples of 16 send
+    """Both copy engines and all four executors (the mirror executor where the receive buffers
+    fit one SM's shared memory, the graph chain in its place where not).  Byte counts that are not multiples of 16 send
     a bulk request to the vector engine (the bulk engine moves 16-byte units), which is part of
     what is checked."""
     for P in (1, 2, 5, 6, 8, 13, 16, 32, 50, 64):
@@ -159,10 +162,36 @@ def test_gpu_v_parity_mixed_sizes(algo, exec_mode, copy):
 
 
 @pytest.mark.gpu
+def test_gpu_v_mirror_is_used_where_it_fits():
+    torch, dev = _gpu()
+    for counts, want in (([64, 0, 200, 16, 48, 1000, 8, 24], sp.EXEC_MIRROR),         # 10.6 KiB in all
+                         ([3000] * 8, sp.EXEC_MIRROR),                                 # 187.5 KiB: on request only
+                         ([4000] * 8, sp.EXEC_GRAPH)):                                 # 250 KiB: fits no SM
+        P, T = len(counts), sum(counts)
+        plan = sp.Plan.create_v(counts, sp.ALGO_SPARBIT, sp.EXEC_MIRROR)
+        host_send = si.send_blocks_v(counts, 5)
+        send = torch.from_numpy(host_send).to(dev)
+        recv = torch.full((P * T,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        plan.allgather(send, recv)
+        assert plan.status() == sp.OK and plan.exec_mode == want, counts
+        assert all(torch.equal(recv.view(P, T)[r], send) for r in range(P))
+        assert plan.launch_counts() == ((1, 1) if want == sp.EXEC_MIRROR else (3, 1))
+        plan.destroy()
+    small = sp.Plan.create_v([64, 0, 200, 16, 48, 1000, 8, 24])
+    assert small.exec_mode == sp.EXEC_MIRROR                  # what AUTO picks below 64 KiB
+    big = sp.Plan.create_v([3000] * 8)
+    assert big.exec_mode == sp.EXEC_GRAPH
+
+
+@pytest.mark.gpu
 def test_gpu_v_all_empty_but_one_and_misaligned():
     run_v_case(9, [0, 0, 0, 4096, 0, 0, 0, 0, 0], sp.ALGO_SPARBIT, sp.EXEC_AUTO, 1)
     run_v_case(9, [16 * (r + 1) for r in range(9)], sp.ALGO_SPARBIT, sp.EXEC_AUTO, 2, shift=4)
     run_v_case(12, [1000 + 7 * r for r in range(12)], sp.ALGO_NEIGHBOR_EXCHANGE, sp.EXEC_AUTO, 3, shift=1)
+    run_v_case(9, [0, 0, 0, 4096, 0, 0, 0, 0, 0], sp.ALGO_SPARBIT, sp.EXEC_MIRROR, 1)
+    run_v_case(9, [16 * (r + 1) for r in range(9)], sp.ALGO_SPARBIT, sp.EXEC_MIRROR, 2, shift=4)
+    run_v_case(12, [1000 + 7 * r for r in range(12)], sp.ALGO_NEIGHBOR_EXCHANGE, sp.EXEC_MIRROR, 3, shift=1)
+    run_v_case(16, [5000] + [0] * 15, sp.ALGO_RING, sp.EXEC_MIRROR, 4, shift=2)
 
 
 @pytest.mark.gpu

@@ -170,7 +170,8 @@ def test_environment_overrides_only_the_automatic_choice(monkeypatch):
     assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_PERSISTENT
     monkeypatch.setenv("SPARBIT_EXEC", "flow")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_FLOW
-    assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_GRAPH                  # not offered there
+    assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_MIRROR                 # flow is not offered there: AUTO's own pick
+    assert sp.Plan.create_v([70000, 80000]).exec_mode == sp.EXEC_GRAPH
     monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR
 
