@@ -12,10 +12,12 @@
 //           of stores through bulk async-groups.  Every load fills one CTA's own shared memory and
 //           every block has one destination (two in the fused first pass, issued as two stores).
 //
-// and four ways to sequence passes: one kernel per pass, chained by programmatic dependent launch
+// and five ways to sequence passes: one kernel per pass, chained by programmatic dependent launch
 // (plain stream launches or a CUDA graph); one persistent cooperative kernel with a bounded-wait
-// grid barrier after every pass; or one cooperative kernel in which every rank's Waitall is a set
-// of per-rank counters instead of a barrier (flow).
+// grid barrier after every pass; one kernel in which every rank's Waitall is a set of per-rank
+// counters instead of a barrier (flow); and, for small collectives, one CTA or one cluster of
+// CTAs that keeps a copy of the receive buffers in (distributed) shared memory and feeds every
+// pass from there (mirror).
 //
 // Loads never use the non-coherent path or L1: data written in one pass is read by other SMs in
 // the next one, possibly inside the same launch.
