@@ -195,6 +195,11 @@ int sparbit_plan_destroy(sparbit_plan_t* plan);
  * the fast paths.  Errors (nothing is launched): ERR_ARG (null plan; null buffer with P*m > 0),
  * ERR_ALIAS (ranges overlap), ERR_WORKSPACE (Bruck without workspace), ERR_CUDA.
  * A device-side barrier time-out is reported later by sparbit_plan_status.
+ * On a stream that is being captured (after the plan's first, uncaptured call) the collective
+ * goes into the caller's graph as plain chained per-pass kernels - the mirror kernel as itself -
+ * whatever executor the plan names: the persistent and the flow kernel take counter values of
+ * one particular launch as arguments and would not replay.  The captured graph may be replayed
+ * any number of times.
  */
 int sparbit_allgather(sparbit_plan_t* plan, const void* sendbuf, void* recvbuf, void* stream);
 

@@ -1169,6 +1169,25 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
     const Resolved rs = resolve(p, send, recv, first, last);
     const Geom g = make_geom(p, send, recv);
     cudaStream_t st = (cudaStream_t)stream;
+    // On a stream that is being captured the work must be replayable as it stands.  The persistent
+    // and the flow kernel take counter values of THIS launch as arguments, and a cached graph
+    // would have to be instantiated in the middle of the caller's capture; so there the passes go
+    // in as plain chained kernels (the mirror kernel as itself), which replay any number of times.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    CU(cudaStreamIsCapturing(st, &capturing));
+    if (capturing != cudaStreamCaptureStatusNone) {
+        Resolved rc_rs = rs;
+        if (rs.exec != SPARBIT_EXEC_MIRROR) rc_rs.exec = SPARBIT_EXEC_STREAM;
+        rc = rc_rs.exec == SPARBIT_EXEC_MIRROR ? launch_mirror(p, rc_rs, g, first, last, st)
+                                               : launch_stream(p, rc_rs, g, first, last, st);
+        if (rc == SPARBIT_OK) {
+            p->copy_last = rc_rs.copy;
+            p->exec_last = rc_rs.exec;
+            p->last_stream = st;
+            p->launched = true;
+        }
+        return rc;
+    }
     switch (rs.exec) {
         case SPARBIT_EXEC_PERSISTENT: rc = launch_persistent(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_GRAPH: rc = launch_graph(p, rs, g, first, last, st); break;

@@ -354,6 +354,41 @@ def test_flow_launch_forms_and_the_measurement_hook(dev):
     plan.destroy()
 
 
+@pytest.mark.parametrize("exec_mode", EXECS + [sp.EXEC_AUTO])
+def test_collective_inside_a_captured_graph_replays(dev, exec_mode):
+    """A collective enqueued on a stream under capture must replay as often as the caller likes:
+    nothing in the captured work may depend on counters of one particular launch.  Each replay
+    runs on new send data and into sentinel-filled buffers."""
+    for P, m in ((16, 2048), (8, 64), (48, 4096)):
+        plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+        send = torch.zeros(P * m, dtype=torch.uint8, device=dev)
+        recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            plan.allgather(send, recv, stream)      # the first call allocates the plan's device state
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            graph.capture_begin()
+            plan.allgather(send, recv, stream)
+            graph.capture_end()
+        for it in range(3):
+            host_send = si.send_blocks(P, m, 30 + it)
+            send.copy_(torch.from_numpy(host_send.reshape(-1)))
+            recv.fill_(si.SENTINEL)
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            want, _ = oracle.allgather(oracle.SPARBIT, P, m, host_send)
+            assert np.array_equal(recv.cpu().numpy(), want.reshape(-1)), (P, m, exec_mode, it)
+        # and the plan still works outside the graph
+        recv.fill_(si.SENTINEL)
+        plan.allgather(send, recv)
+        assert plan.status() == sp.OK
+        assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+        del graph
+        plan.destroy()
+
+
 def test_two_flow_collectives_at_once(dev):
     """Two plans, two streams, both on the flow executor at the same time.  Each kernel's waits
     need all of its CTAs resident; the cooperative launch sees to that (the second kernel starts
