@@ -362,7 +362,14 @@ enum {
                                               kernel would take if waiting cost nothing, the bound on what any
                                               finer readiness tracking could gain (bench.py
                                               --flow-wait-bound).  0 by default */
-    SPARBIT_TUNE_COUNT_ = 14
+    SPARBIT_TUNE_GROUPED_FRONT = 14,       /* GRAPH and STREAM executors, Sparbit: 1 (default) = the leading
+                                              passes whose distance is a multiple of some G that divides P
+                                              run as G independent groups of P/G ranks, one CTA per group
+                                              working from an on-chip copy of its part of the receive
+                                              buffers (one kernel instead of one per pass), as far as a
+                                              group's part stays within MIRROR_MAX_BYTES; 0 = every pass its
+                                              own kernel */
+    SPARBIT_TUNE_COUNT_ = 15
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

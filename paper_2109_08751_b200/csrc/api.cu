@@ -116,6 +116,7 @@ struct sparbit_plan_s {
         4,            // MIRROR_THREAD_VECTORS
         0,            // FLOW_COOPERATIVE
         0,            // FLOW_SKIP_WAITS
+        1,            // GROUPED_FRONT
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -124,6 +125,7 @@ struct sparbit_plan_s {
         GraphKey key;
         cudaGraphExec_t exec = nullptr;
         uint64_t stamp = 0;
+        uint64_t kernels = 0;  // kernel nodes of the graph
     };
     std::vector<GraphEntry> gcache;
     uint64_t gstamp = 0;
@@ -506,9 +508,37 @@ bool mirror_wins(const sparbit_plan_s* p, int vbytes, int first, int last) {
            p->sched.m <= p->tune[SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK];
 }
 
-int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
-    if (mirror_possible(p, first, last, (size_t)p->max_smem_optin) && mirror_wins(p, vbytes, first, last))
+int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32_t* groups);
+
+// The executor for a small collective, or -1 if it is none.  One CTA where everything is small
+// enough for it.  Beyond that the mirror executor on a cluster (about 3.5 us + 0.8 us per pass) or
+// the chain with its leading passes in the grouped mirror kernel (4.2-6.2 us for those + 2.05 us
+// per pass after them), whichever comes out shorter: the chain when at most three passes follow
+// the grouped ones (measured: P = 256, m = 8 B 10.4 us against 14.4; P = 128, m = 128 B 10.3
+// against 14.8; equal at P = 64 and 128 with m = 64 B).  P without a suitable power-of-two divisor
+// has no groups: the cluster it is (P = 253, m = 1 B 14.4 against 18.5 for the plain chain).
+int small_collective_exec(const sparbit_plan_s* p, int vbytes, int first, int last, size_t smem_limit) {
+    if (!mirror_possible(p, first, last, smem_limit) || !mirror_wins(p, vbytes, first, last)) return -1;
+    if (p->variable) return SPARBIT_EXEC_MIRROR;
+    const ExecSeq seq = make_seq(p, first, last);
+    uint64_t most = 0;
+    for (int i = 0; i < seq.count(); i++) {
+        const PhaseDesc& d = seq.item(i);
+        const uint64_t v = (uint64_t)p->sched.P * d.copies * (d.copy_bytes / (uint64_t)vbytes);
+        if (v > most) most = v;
+    }
+    if (mirror_smem_per_cta(p, 1) <= (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES] &&
+        most <= 8 * p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS])
         return SPARBIT_EXEC_MIRROR;
+    uint32_t groups = 1;
+    const int s = front_passes(p, seq, vbytes, &groups);
+    if (s >= 2 && seq.count() - s <= 3) return SPARBIT_EXEC_GRAPH;
+    return SPARBIT_EXEC_MIRROR;
+}
+
+int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    const int small = small_collective_exec(p, vbytes, first, last, (size_t)p->max_smem_optin);
+    if (small >= 0) return small;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
@@ -517,8 +547,8 @@ int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
 }
 
 int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
-    if (mirror_possible(p, -1, p->sched.last_phase(), 227u << 10) && mirror_wins(p, vbytes, -1, p->sched.last_phase()))
-        return SPARBIT_EXEC_MIRROR;
+    const int small = small_collective_exec(p, vbytes, -1, p->sched.last_phase(), 227u << 10);
+    if (small >= 0) return small;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
@@ -657,6 +687,91 @@ struct PhaseArgs {
     }
 };
 
+// How many leading passes of a call run in the grouped mirror kernel (0: none).  Sparbit's step
+// distances are descending powers of two; while they are multiples of a G that divides P the
+// ranks fall into G independent groups of R = P / G (see grouped_mirror_vec_kernel).  The largest
+// such run of passes whose group state, R*R*m bytes, one CTA handles well (MIRROR_MAX_BYTES, and
+// eight times MIRROR_CTA_VECTORS vectors in its largest pass); at least two passes, else nothing
+// is saved.
+int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32_t* groups) {
+    const Schedule& sc = p->sched;
+    if (!p->tune[SPARBIT_TUNE_GROUPED_FRONT] || p->variable || sc.algo != ALGO_SPARBIT || !seq.fused) return 0;
+    const int n = seq.count();  // item i is step i (item 0 with the own-block copy fused in)
+    int best = 0;
+    for (int s = 2; s <= n && s <= kMirrorMaxPasses; s++) {
+        const uint64_t G = (uint64_t)sc.steps[(size_t)s - 1].distance;
+        if (G < 1 || (G & (G - 1)) || sc.P % G) continue;
+        const uint64_t R = sc.P / G;
+        if ((unsigned __int128)R * R * sc.m > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) break;
+        uint64_t most = 0;
+        for (int i = 0; i < s; i++) {
+            const PhaseDesc& d = seq.item(i);
+            const uint64_t v = R * d.copies * (d.copy_bytes / (uint64_t)vbytes);
+            if (v > most) most = v;
+        }
+        if (most > 8 * p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS]) break;
+        if (G > 65535) continue;
+        best = s;
+        *groups = (uint32_t)G;
+    }
+    return best;
+}
+
+template <typename V>
+const void* grouped_mirror_fn() { return (const void*)grouped_mirror_vec_kernel<V>; }
+const void* pick_grouped_mirror(int vbytes) {
+    switch (vbytes) {
+        case 16: return grouped_mirror_fn<uint4>();
+        case 8: return grouped_mirror_fn<uint2>();
+        case 4: return grouped_mirror_fn<unsigned>();
+        case 2: return grouped_mirror_fn<unsigned short>();
+        default: return grouped_mirror_fn<unsigned char>();
+    }
+}
+
+int grant_max_smem(const sparbit_plan_s* p, const void* fn, int slot, bool big_cluster);
+int vec_slot(int vbytes);
+
+int launch_grouped_front(sparbit_plan_s* p, const Resolved& rs, const Geom& g, const ExecSeq& seq, int front,
+                         uint32_t groups, cudaStream_t st) {
+    MirrorArgs ma;
+    memset(&ma, 0, sizeof ma);
+    ma.n = front;
+    const uint64_t R = p->sched.P / groups;
+    uint64_t most = 1;
+    for (int i = 0; i < front; i++) {
+        ma.d[i] = seq.item(i);
+        const uint64_t vpc = ma.d[i].copy_bytes / (uint64_t)rs.vbytes;
+        const uint64_t v = R * ma.d[i].copies * vpc;
+        if (v > most) most = v;
+        ma.magic_vpc[i] = ((1ull << 40) + vpc - 1) / (vpc ? vpc : 1);
+        ma.magic_copies[i] = ((1ull << 40) + ma.d[i].copies - 1) / (ma.d[i].copies ? ma.d[i].copies : 1);
+    }
+    const void* fn = pick_grouped_mirror(rs.vbytes);
+    int rc = grant_max_smem(p, fn, 24 + vec_slot(rs.vbytes), false);
+    if (rc) return rc;
+    const uint64_t per_thread = p->tune[SPARBIT_TUNE_MIRROR_THREAD_VECTORS];
+    uint64_t threads = (most + per_thread - 1) / per_thread;
+    threads = (threads + 63) / 64 * 64;
+    if (threads > 1024) threads = 1024;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(groups);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = (size_t)(R * R * p->sched.m);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    Geom gg = g;
+    void* args[] = {&gg, &ma};
+    CU(cudaLaunchKernelExC(&cfg, fn, args));
+    p->kernel_launches++;
+    return SPARBIT_OK;
+}
+
 // One kernel per phase on `st`.  Consecutive phases are launched with programmatic stream
 // serialisation: a phase kernel lets its successor start launching at once
 // (griddepcontrol.launch_dependents) and itself waits for its predecessor to complete and flush
@@ -666,7 +781,16 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
                   int seq_end = -1) {
     const ExecSeq seq = make_seq(p, first, last);
     const int end = seq_end < 0 ? seq.count() : seq_end;  // only the first seq_end passes, if given
-    for (int i = 0; i < end; i++) {
+    int front = 0;
+    if (seq_end < 0 && rs.copy == SPARBIT_COPY_VECTOR) {
+        uint32_t groups = 1;
+        front = front_passes(p, seq, rs.vbytes, &groups);
+        if (front) {
+            int rc = launch_grouped_front(p, rs, g, seq, front, groups, st);
+            if (rc) return rc;
+        }
+    }
+    for (int i = front; i < end; i++) {
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
         cfg.stream = st;
@@ -740,6 +864,7 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
                                                 : launch_stream(p, rs, g, first, last, p->capture_stream);
         cudaGraph_t graph = nullptr;
         cudaError_t ce = cudaStreamEndCapture(p->capture_stream, &graph);
+        const uint64_t captured = p->kernel_launches - launches_before;
         p->kernel_launches = launches_before;  // captured, not launched
         if (rc) {
             if (graph) cudaGraphDestroy(graph);
@@ -777,11 +902,12 @@ int launch_graph(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first
         }
         cudaGraphDestroy(graph);
         hit->key = key;
+        hit->kernels = captured;
     }
     hit->stamp = ++p->gstamp;
     CU(cudaGraphLaunch(hit->exec, st));
     p->graph_launches++;
-    p->kernel_launches += rs.exec == SPARBIT_EXEC_MIRROR ? 1u : (uint64_t)make_seq(p, first, last).count();
+    p->kernel_launches += hit->kernels;
     return SPARBIT_OK;
 }
 
@@ -866,7 +992,7 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
 // maximum (asking for less per launch costs nothing), so that no plan can lower it under another.
 constexpr int kSmemDevices = 64;
 std::mutex g_smem_mutex;
-bool g_smem_granted[kSmemDevices][24];
+bool g_smem_granted[kSmemDevices][32];
 int vec_slot(int vbytes) { return vbytes == 16 ? 4 : vbytes == 8 ? 3 : vbytes == 4 ? 2 : vbytes == 2 ? 1 : 0; }
 int grant_max_smem(const sparbit_plan_s* p, const void* fn, int slot, bool big_cluster) {
     std::lock_guard<std::mutex> lock(g_smem_mutex);

@@ -735,6 +735,54 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
     }
 }
 
+// The first passes of Sparbit as INDEPENDENT small collectives.  While the step distance is still a
+// multiple of G (a power of two that divides P), a rank only ever exchanges blocks with ranks of its
+// own residue class mod G, and only blocks whose index is in that class too: the P ranks fall into
+// G groups of R = P / G ranks that do not talk to each other.  Each group's part of the receive
+// buffers - R ranks x R slots - is small even when the whole is not, so one CTA per group runs those
+// passes from an on-chip copy exactly as mirror_vec_kernel does for a whole collective (same copies,
+// same slots, written through to global memory); the passes after them, whose distance is below G,
+// run as the usual per-pass kernels and read what this kernel wrote.  grid = G CTAs.
+template <typename V>
+__global__ void __launch_bounds__(1024, 1) grouped_mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
+    // [R][R] slots of m bytes: local rank i is rank c + i * G, local slot k is slot c + k * G
+    extern __shared__ __align__(16) unsigned char mirror[];
+    chain_trigger();
+    chain_wait();
+    const uint32_t P = g.P;
+    const uint32_t c = blockIdx.x;
+    const uint32_t lgG = 31u - (uint32_t)__clz(gridDim.x);
+    const uint32_t R = P >> lgG;
+    const uint32_t vps = (uint32_t)(g.m / sizeof(V));  // vectors per slot
+    V* mir = reinterpret_cast<V*>(mirror);
+    const V* gsend = reinterpret_cast<const V*>(g.base[SPACE_SEND]);
+    V* grecv = reinterpret_cast<V*>(g.base[SPACE_RECV]);
+    for (int i = 0; i < ma.n; i++) {
+        if (i) __syncthreads();
+        const PhaseDesc& d = ma.d[i];
+        const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
+        const uint32_t total = R * d.copies * vpc;
+        const bool from_send = d.src_space == SPACE_SEND;
+        const unsigned long long mv = ma.magic_vpc[i], mc = ma.magic_copies[i];
+        for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
+            const uint32_t q = (uint32_t)((t * mv) >> 40);   // t / vpc
+            const uint32_t v = t - q * vpc;
+            const uint32_t li = (uint32_t)((q * mc) >> 40);  // q / copies: local rank of the sender
+            const uint32_t j = q - li * d.copies;
+            const uint32_t r = c + (li << lgG);
+            const CopyLoc loc = locate_copy(d, P, r, j);
+            const V x = from_send ? ld_cg<V>(gsend + (uint64_t)r * vps + v) : mir[(li * R + (loc.src_slot >> lgG)) * vps + v];
+            const uint32_t ls = loc.dst_slot >> lgG;
+            mir[((loc.dst_rank >> lgG) * R + ls) * vps + v] = x;
+            st_cg<V>(grecv + ((uint64_t)loc.dst_rank * P + loc.dst_slot) * vps + v, x);
+            if (d.dup_self) {
+                mir[(li * R + ls) * vps + v] = x;
+                st_cg<V>(grecv + ((uint64_t)r * P + loc.dst_slot) * vps + v, x);
+            }
+        }
+    }
+}
+
 // The same for blocks of DIFFERENT sizes (allgatherv), in one CTA: the passes' work comes as the task
 // lists the list kernels use (byte offsets inside the source and destination space, at most
 // kVarSegmentBytes each), a group of lanes per task; the on-chip copy is laid out like the receive space

@@ -197,6 +197,35 @@ def test_mirror_state_after_every_prefix(dev, algo, P):
             assert np.array_equal(work.cpu().numpy(), scratch), k
 
 
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_GRAPH, sp.EXEC_STREAM])
+@pytest.mark.parametrize("P,m", [(16, 64), (32, 272), (64, 64), (96, 100), (128, 16), (192, 24), (256, 64), (256, 8),
+                                 (24, 1000), (40, 6), (512, 16), (1000, 4), (48, 3)])
+def test_grouped_front_state_after_every_prefix(dev, exec_mode, P, m):
+    """Sparbit's leading passes as independent groups, one CTA each, then the chain: run passes
+    -1..k for every k into sentinel-filled buffers; the whole receive space must be the oracle's
+    state after step k, whether the call ends inside the grouped passes or behind them."""
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    ref = oracle.Plan(sp.ALGO_SPARBIT, P)
+    host_send = si.send_blocks(P, m, 79)
+    send = torch.from_numpy(host_send.reshape(-1)).to(dev)
+    recv = torch.empty((P * P * m,), dtype=torch.uint8, device=dev)
+    grouped = 0
+    for k in range(-1, ref.last_phase + 1):
+        recv.fill_(si.SENTINEL)
+        before = plan.launch_counts()[0]
+        plan.allgather_steps(send, recv, -1, k)
+        assert plan.status() == sp.OK
+        launches = plan.launch_counts()[0] - before
+        passes = max(1, k + 1)            # the own-block copy is fused into step 0
+        grouped = max(grouped, passes - launches)
+        want = si.sentinel_buffer(P * P * m)
+        ref.run(m, host_send.reshape(-1), want, None, first=-1, last=k)
+        assert np.array_equal(recv.cpu().numpy(), want), (P, m, k)
+    if P in (16, 32, 64, 128, 256, 512, 96, 192):
+        assert grouped >= 1, (P, m)        # some passes did share a kernel
+    plan.destroy()
+
+
 # ---------------------------------------------------------------- brute force over P
 ALL_IN_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 1}     # every pass in the flow kernel
 SPLIT_FLOW = {sp.TUNE_FLOW_MIN_PASS_SPANS: 40}     # passes of fewer than 40 spans as kernels in front of it
@@ -512,9 +541,15 @@ def test_runs_on_a_user_stream_and_counts_launches(dev, exec_mode):
         assert small.status() == sp.OK and small.launch_counts() == (2, 2)   # one kernel in a cached graph
         small.destroy()
     elif exec_mode == sp.EXEC_GRAPH:
-        assert (kernels, graphs) == (2 * phases, 2)
+        assert (kernels, graphs) == (2 * 2, 2)     # three passes as 2 groups of 8 ranks in one kernel, then the last pass
+        plain = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+        plain.set_tunable(sp.TUNE_GROUPED_FRONT, 0)
+        plain.allgather(send, recv, stream)
+        assert plain.status() == sp.OK and plain.launch_counts() == (phases, 1)   # every pass its own kernel
+        assert np.array_equal(recv.cpu().numpy(), want.reshape(-1))
+        plain.destroy()
     else:
-        assert (kernels, graphs) == (2 * phases, 0)
+        assert (kernels, graphs) == (2 * 2, 0)
     assert plan.exec_mode == exec_mode
 
 

@@ -136,10 +136,13 @@ def test_strerror_covers_every_code():
 def test_exec_mode_resolution():
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR            # 4 KiB of receive buffers: one CTA, on chip
     assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
-    assert sp.Plan(32, 128).exec_mode == sp.EXEC_MIRROR          # 128 KiB, small blocks: a cluster of CTAs
-    assert sp.Plan(128, 64).exec_mode == sp.EXEC_MIRROR          # 1 MiB: still
-    assert sp.Plan(128, 128).exec_mode == sp.EXEC_GRAPH          # 2 MiB: the chain is faster
-    assert sp.Plan(16, 4096).exec_mode == sp.EXEC_MIRROR         # 1 MiB of 4 KiB blocks: the last that gain
+    assert sp.Plan(45, 512).exec_mode == sp.EXEC_MIRROR          # 1 MiB, no power of two divides 45: a cluster of CTAs
+    assert sp.Plan(253, 1).exec_mode == sp.EXEC_MIRROR           # 63 KiB but 32 Ki one-byte vectors: a cluster too
+    assert sp.Plan(32, 128).exec_mode == sp.EXEC_GRAPH           # 128 KiB: the chain, its first four passes as 2 groups of 16 ranks
+    assert sp.Plan(128, 64).exec_mode == sp.EXEC_GRAPH           # 1 MiB: the chain, four passes as 8 groups of 16
+    assert sp.Plan(256, 64).exec_mode == sp.EXEC_GRAPH           # 4 MiB: the chain, five passes as 8 groups of 32
+    assert sp.Plan(128, 128).exec_mode == sp.EXEC_GRAPH          # 2 MiB
+    assert sp.Plan(13, 4096).exec_mode == sp.EXEC_MIRROR         # 676 KiB of 4 KiB blocks, odd P: a cluster
     assert sp.Plan(8, 8192).exec_mode == sp.EXEC_GRAPH           # 512 KiB of larger blocks: the chain
     assert sp.Plan(8, 8192, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
     assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR     # 144 KiB, and as much of working buffers
