@@ -689,20 +689,26 @@ struct PhaseArgs {
 
 // How many leading passes of a call run in the grouped mirror kernel (0: none).  Sparbit's step
 // distances are descending powers of two; while they are multiples of a G that divides P the
-// ranks fall into G independent groups of R = P / G (see grouped_mirror_vec_kernel).  The largest
+// ranks fall into G independent groups of R = P / G (see grouped_mirror_vec_kernel).  Recursive
+// doubling's are ascending: after s steps a rank has only talked inside its aligned run of 2^s.  The largest
 // such run of passes whose group state, R*R*m bytes, one CTA handles well (MIRROR_MAX_BYTES, and
 // eight times MIRROR_CTA_VECTORS vectors in its largest pass); at least two passes, else nothing
 // is saved.
 int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32_t* groups) {
     const Schedule& sc = p->sched;
-    if (!p->tune[SPARBIT_TUNE_GROUPED_FRONT] || p->variable || sc.algo != ALGO_SPARBIT || !seq.fused) return 0;
+    if (!p->tune[SPARBIT_TUNE_GROUPED_FRONT] || p->variable || !seq.fused) return 0;
+    if (sc.algo != ALGO_SPARBIT && sc.algo != ALGO_RD) return 0;
     const int n = seq.count();  // item i is step i (item 0 with the own-block copy fused in)
     int best = 0;
     for (int s = 2; s <= n && s <= kMirrorMaxPasses; s++) {
-        const uint64_t G = (uint64_t)sc.steps[(size_t)s - 1].distance;
-        if (G < 1 || (G & (G - 1)) || sc.P % G) continue;
+        // Sparbit: G = the distance of the last grouped step, a power of two that must divide P.
+        // Recursive doubling (P a power of two): runs of R = twice that distance.
+        const uint64_t dist = (uint64_t)sc.steps[(size_t)s - 1].distance;
+        if (dist < 1 || (dist & (dist - 1))) continue;
+        const uint64_t G = sc.algo == ALGO_SPARBIT ? dist : sc.P / (2 * dist);
+        if (G < 1 || sc.P % G || G > 65535) continue;
         const uint64_t R = sc.P / G;
-        if ((unsigned __int128)R * R * sc.m > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) break;
+        if ((unsigned __int128)R * R * sc.m > (unsigned __int128)p->tune[SPARBIT_TUNE_MIRROR_MAX_BYTES]) break;  // groups only grow
         uint64_t most = 0;
         for (int i = 0; i < s; i++) {
             const PhaseDesc& d = seq.item(i);
@@ -710,7 +716,6 @@ int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32
             if (v > most) most = v;
         }
         if (most > 8 * p->tune[SPARBIT_TUNE_MIRROR_CTA_VECTORS]) break;
-        if (G > 65535) continue;
         best = s;
         *groups = (uint32_t)G;
     }
@@ -737,6 +742,7 @@ int launch_grouped_front(sparbit_plan_s* p, const Resolved& rs, const Geom& g, c
     MirrorArgs ma;
     memset(&ma, 0, sizeof ma);
     ma.n = front;
+    ma.aligned = p->sched.algo == ALGO_RD ? 1 : 0;
     const uint64_t R = p->sched.P / groups;
     uint64_t most = 1;
     for (int i = 0; i < front; i++) {

@@ -685,7 +685,7 @@ struct MirrorArgs {
     int n;
     uint32_t work_at;  // Bruck: where, in vectors, the on-chip copy of the working buffers starts
     uint32_t extra_tx;  // cluster form, test hook: bytes expected on top of a pass's own (never arrive)
-    int pad_;
+    int aligned;        // grouped form: 0 = a group is a residue class mod G, 1 = a run of P/G consecutive ranks
     unsigned* status;   // cluster form: device status word (DEV_*)
     unsigned long long timeout_ns;
     // ceil(2^40 / x) for x = vectors per copy and x = copies per rank of each pass, so that t / x
@@ -735,17 +735,20 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
     }
 }
 
-// The first passes of Sparbit as INDEPENDENT small collectives.  While the step distance is still a
-// multiple of G (a power of two that divides P), a rank only ever exchanges blocks with ranks of its
-// own residue class mod G, and only blocks whose index is in that class too: the P ranks fall into
-// G groups of R = P / G ranks that do not talk to each other.  Each group's part of the receive
-// buffers - R ranks x R slots - is small even when the whole is not, so one CTA per group runs those
-// passes from an on-chip copy exactly as mirror_vec_kernel does for a whole collective (same copies,
-// same slots, written through to global memory); the passes after them, whose distance is below G,
-// run as the usual per-pass kernels and read what this kernel wrote.  grid = G CTAs.
+// The first passes of a collective as INDEPENDENT small collectives.  Sparbit: while the step distance
+// is still a multiple of G (a power of two that divides P), a rank only ever exchanges blocks with
+// ranks of its own residue class mod G, and only blocks whose index is in that class too: the P
+// ranks fall into G groups of R = P / G ranks that do not talk to each other.  Recursive doubling
+// starts at the other end: while the distance is below R = 2^s, partners (r xor 2^i) and slots stay
+// inside the aligned run of R consecutive ranks r belongs to.  Either way each group's part of the
+// receive buffers - R ranks x R slots - is small even when the whole is not, so one CTA per group
+// runs those passes from an on-chip copy exactly as mirror_vec_kernel does for a whole collective
+// (same copies, same slots, written through to global memory); the passes after them run as the
+// usual per-pass kernels and read what this kernel wrote.  grid = G CTAs.
 template <typename V>
 __global__ void __launch_bounds__(1024, 1) grouped_mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
-    // [R][R] slots of m bytes: local rank i is rank c + i * G, local slot k is slot c + k * G
+    // [R][R] slots of m bytes.  Residue classes: local rank i is rank c + i * G, local slot k is
+    // slot c + k * G.  Aligned runs: local rank i is rank c * R + i, local slot k is slot c * R + k.
     extern __shared__ __align__(16) unsigned char mirror[];
     chain_trigger();
     chain_wait();
@@ -753,10 +756,12 @@ __global__ void __launch_bounds__(1024, 1) grouped_mirror_vec_kernel(Geom g, con
     const uint32_t c = blockIdx.x;
     const uint32_t lgG = 31u - (uint32_t)__clz(gridDim.x);
     const uint32_t R = P >> lgG;
+    const bool aligned = ma.aligned != 0;
     const uint32_t vps = (uint32_t)(g.m / sizeof(V));  // vectors per slot
     V* mir = reinterpret_cast<V*>(mirror);
     const V* gsend = reinterpret_cast<const V*>(g.base[SPACE_SEND]);
     V* grecv = reinterpret_cast<V*>(g.base[SPACE_RECV]);
+    auto local = [&](uint32_t x) { return aligned ? x - c * R : x >> lgG; };  // of a rank or slot of this group
     for (int i = 0; i < ma.n; i++) {
         if (i) __syncthreads();
         const PhaseDesc& d = ma.d[i];
@@ -769,11 +774,11 @@ __global__ void __launch_bounds__(1024, 1) grouped_mirror_vec_kernel(Geom g, con
             const uint32_t v = t - q * vpc;
             const uint32_t li = (uint32_t)((q * mc) >> 40);  // q / copies: local rank of the sender
             const uint32_t j = q - li * d.copies;
-            const uint32_t r = c + (li << lgG);
+            const uint32_t r = aligned ? c * R + li : c + (li << lgG);
             const CopyLoc loc = locate_copy(d, P, r, j);
-            const V x = from_send ? ld_cg<V>(gsend + (uint64_t)r * vps + v) : mir[(li * R + (loc.src_slot >> lgG)) * vps + v];
-            const uint32_t ls = loc.dst_slot >> lgG;
-            mir[((loc.dst_rank >> lgG) * R + ls) * vps + v] = x;
+            const V x = from_send ? ld_cg<V>(gsend + (uint64_t)r * vps + v) : mir[(li * R + local(loc.src_slot)) * vps + v];
+            const uint32_t ls = local(loc.dst_slot);
+            mir[(local(loc.dst_rank) * R + ls) * vps + v] = x;
             st_cg<V>(grecv + ((uint64_t)loc.dst_rank * P + loc.dst_slot) * vps + v, x);
             if (d.dup_self) {
                 mir[(li * R + ls) * vps + v] = x;

@@ -198,14 +198,18 @@ def test_mirror_state_after_every_prefix(dev, algo, P):
 
 
 @pytest.mark.parametrize("exec_mode", [sp.EXEC_GRAPH, sp.EXEC_STREAM])
-@pytest.mark.parametrize("P,m", [(16, 64), (32, 272), (64, 64), (96, 100), (128, 16), (192, 24), (256, 64), (256, 8),
-                                 (24, 1000), (40, 6), (512, 16), (1000, 4), (48, 3)])
-def test_grouped_front_state_after_every_prefix(dev, exec_mode, P, m):
-    """Sparbit's leading passes as independent groups, one CTA each, then the chain: run passes
-    -1..k for every k into sentinel-filled buffers; the whole receive space must be the oracle's
-    state after step k, whether the call ends inside the grouped passes or behind them."""
-    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
-    ref = oracle.Plan(sp.ALGO_SPARBIT, P)
+@pytest.mark.parametrize("algo,P,m", [(sp.ALGO_SPARBIT, P, m) for P, m in
+                                      [(16, 64), (32, 272), (64, 64), (96, 100), (128, 16), (192, 24), (256, 64),
+                                       (256, 8), (24, 1000), (40, 6), (512, 16), (1000, 4), (48, 3)]] +
+                                     [(sp.ALGO_RECURSIVE_DOUBLING, P, m) for P, m in
+                                      [(16, 64), (32, 272), (64, 48), (128, 16), (256, 64), (256, 6), (512, 8)]])
+def test_grouped_front_state_after_every_prefix(dev, exec_mode, algo, P, m):
+    """The leading passes as independent groups, one CTA each, then the chain (Sparbit: residue
+    classes of ranks; recursive doubling: runs of consecutive ranks): run passes -1..k for every k
+    into sentinel-filled buffers; the whole receive space must be the oracle's state after step k,
+    whether the call ends inside the grouped passes or behind them."""
+    plan = sp.Plan(P, m, algo, exec_mode)
+    ref = oracle.Plan(algo, P)
     host_send = si.send_blocks(P, m, 79)
     send = torch.from_numpy(host_send.reshape(-1)).to(dev)
     recv = torch.empty((P * P * m,), dtype=torch.uint8, device=dev)
@@ -222,7 +226,7 @@ def test_grouped_front_state_after_every_prefix(dev, exec_mode, P, m):
         ref.run(m, host_send.reshape(-1), want, None, first=-1, last=k)
         assert np.array_equal(recv.cpu().numpy(), want), (P, m, k)
     if P in (16, 32, 64, 128, 256, 512, 96, 192):
-        assert grouped >= 1, (P, m)        # some passes did share a kernel
+        assert grouped >= 1, (algo, P, m)  # some passes did share a kernel
     plan.destroy()
 
 
