@@ -532,7 +532,7 @@ int small_collective_exec(const sparbit_plan_s* p, int vbytes, int first, int la
         return SPARBIT_EXEC_MIRROR;
     uint32_t groups = 1;
     const int s = front_passes(p, seq, vbytes, &groups);
-    if (s >= 2 && seq.count() - s <= 3) return SPARBIT_EXEC_GRAPH;
+    if (s >= 3 && seq.count() - s <= 3) return SPARBIT_EXEC_GRAPH;
     return SPARBIT_EXEC_MIRROR;
 }
 
@@ -692,7 +692,7 @@ struct PhaseArgs {
 // ranks fall into G independent groups of R = P / G (see grouped_mirror_vec_kernel).  Recursive
 // doubling's are ascending: after s steps a rank has only talked inside its aligned run of 2^s.  The largest
 // such run of passes whose group state, R*R*m bytes, one CTA handles well (MIRROR_MAX_BYTES, and
-// eight times MIRROR_CTA_VECTORS vectors in its largest pass); at least two passes, else nothing
+// eight times MIRROR_CTA_VECTORS vectors in its largest pass); at least three passes, else nothing
 // is saved.
 int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32_t* groups) {
     const Schedule& sc = p->sched;
@@ -719,7 +719,7 @@ int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32
         best = s;
         *groups = (uint32_t)G;
     }
-    return best;
+    return best >= 3 ? best : 0;  // two grouped passes cost what two chained passes cost
 }
 
 template <typename V>
