@@ -75,13 +75,17 @@ enum {
  * the first peer's): same state after phase 0, one pass less. */
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
-                                    buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB),
-                                    FLOW for collectives that move 0.45 to 6 GB, the graph chain
-                                    otherwise (thresholds: SPARBIT_TUNE_*) */
+                                    buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB,
+                                    where the chain with a grouped front is not at least as
+                                    fast), FLOW for collectives that move 0.45 to 6 GB, the graph
+                                    chain otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
-                                    re-parameterise the least recently used graph) */
+                                    re-parameterise the least recently used graph).  Sparbit's
+                                    (and recursive doubling's) leading passes share ONE kernel
+                                    where the ranks fall into independent groups small enough
+                                    for a CTA each (SPARBIT_TUNE_GROUPED_FRONT) */
     SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
     SPARBIT_EXEC_FLOW = 4,       /* one kernel (all CTAs resident) without grid barriers:
                                     Algorithm 1's Waitall is kept per rank (counters of what each
