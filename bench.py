@@ -267,6 +267,8 @@ def run_ours(args):
 
     plan = sp.Plan(P, m, algo, exec_mode)
     plan.set_copy_path(copy)
+    if args.no_grouped_front:
+        plan.set_tunable(sp.TUNE_GROUPED_FRONT, 0)
     seed = args.seed + rank
     # two input sets, alternated, so that no step finds its answer already in place
     sends = [torch.from_numpy(si.send_blocks(P, m, seed + k).reshape(-1)).to(dev) for k in range(2)]
@@ -554,6 +556,8 @@ def run_sweep(args):
                     continue  # fits no cluster
                 plan = sp.Plan(P, m, algos[name], e)
                 plan.set_copy_path(c)
+                if args.no_grouped_front:
+                    plan.set_tunable(sp.TUNE_GROUPED_FRONT, 0)
                 if name == "bruck":
                     plan.set_workspace(work, P * P * m)
                 # the paper's protocol (5 warm-ups, 50 timed runs), the way its benchmark times them:
@@ -847,6 +851,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "mirror", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
+    ap.add_argument("--no-grouped-front", action="store_true",
+                    help="every pass of the graph and stream executors as its own kernel (SPARBIT_TUNE_GROUPED_FRONT = 0)")
     ap.add_argument("--sweep-auto-only", action="store_true",
                     help="with --sweep: only the executor and engine the library picks by itself")
     ap.add_argument("--heatmap", nargs="?", const="coarse", default=None, choices=["coarse", "paper"],
