@@ -60,7 +60,7 @@ NCU_TRAFFIC = {
     "sparbit:P256:m64:graph:vector": (4.21e6, "profiles/phase_vec_kernel_P256_small_blocks.md"),
     "sparbit:P256:m8:graph:vector": (5.36e5, "profiles/phase_vec_kernel_P256_small_blocks.md"),
 }
-MIN_TIMED_MS = 250.0   # the timed rounds together last at least this long, whatever --steps is
+MIN_TIMED_MS = 500.0   # the timed rounds together last at least this long, whatever --steps is
 
 
 def effective_bytes(P: int, m: int) -> int:
