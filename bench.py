@@ -770,6 +770,82 @@ def run_mapping_study(args):
     return 0
 
 
+def run_multi_emulated(args):
+    """The multi-device executor (sparbit_allgather_multi_phases) with its G devices emulated on ONE
+    GPU: G pairs of allocations, one kernel per device and step, all on one stream, so that stream
+    order is the cross-device barrier and every "peer" store is a local store.  This times the
+    kernels and the G launches per step against the single-device executor on the same collective; it
+    says nothing about NVLink.  One JSON line per (G, mapping), plus the single-device line first."""
+    import torch
+    import paper_2109_08751_b200 as sp
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, _ = measured_peak()
+    P, m = args.P, args.m
+    stream = torch.cuda.Stream(device=dev)
+    host = [si.send_blocks(P, m, args.seed + k) for k in range(2)]
+    rdev = sp.binding.lib.sparbit_rank_device
+
+    def timed(run):
+        us = []
+        with torch.cuda.stream(stream):
+            for it in range(5):
+                run(it)
+            stream.synchronize()
+            for _ in range(10):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for it in range(20):
+                    run(it)
+                e1.record(stream)
+                stream.synchronize()
+                us.append(e0.elapsed_time(e1) / 20 * 1e3)
+        return us
+
+    def line(tag, us, ok):
+        avg = float(np.mean(us))
+        print(json.dumps({"P": P, "m": m, **tag, "us_min": round(min(us), 2), "us_avg": round(avg, 2),
+                          "us_max": round(max(us), 2), "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
+                          "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),
+                          "checked": ok}), flush=True)
+
+    plan = sp.Plan(P, m)
+    sends = [torch.from_numpy(h.reshape(-1)).to(dev) for h in host]
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    us = timed(lambda it: plan.allgather(sends[it & 1], recv, stream))
+    line({"devices": 1, "mapping": "-", "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}"},
+         us, bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1])))
+    del recv
+    for G in (1, 2, 4, 8):
+        for name, mp in (("sequential", sp.MAP_SEQUENTIAL), ("cyclic", sp.MAP_CYCLIC)):
+            ranks = [[r for r in range(P) if rdev(P, G, mp, r) == g] for g in range(G)]
+            dsend = [[torch.from_numpy(np.ascontiguousarray(h[ranks[g]]).reshape(-1)).to(dev) for g in range(G)]
+                     for h in host]
+            drecv = [torch.full((len(ranks[g]) * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+                     for g in range(G)]
+            bases = [t.data_ptr() for t in drecv]
+
+            def run(it):
+                # phases -1 and 0 as one pass, then step by step; every device's kernel of a step is
+                # enqueued before any kernel of the next step
+                for g in range(G):
+                    plan.allgather_multi_phases(G, mp, g, dsend[it & 1][g], bases, -1, 0, stream)
+                for ph in range(1, plan.last_phase + 1):
+                    for g in range(G):
+                        plan.allgather_multi_phases(G, mp, g, dsend[it & 1][g], bases, ph, ph, stream)
+
+            us = timed(run)
+            want = torch.from_numpy(host[1].reshape(-1)).to(dev)
+            ok = all(bool(torch.equal(drecv[g].view(len(ranks[g]), P * m)[-1], want)) for g in range(G))
+            line({"devices": G, "mapping": name, "ran": "multi-device kernels, emulated on one GPU",
+                  "launches_per_collective": G * (plan.last_phase + 1)}, us, ok)
+            del dsend, drecv
+            torch.cuda.empty_cache()
+    plan.destroy()
+    return 0
+
+
 def run_heatmap(args):
     """Which algorithm is fastest for each (P, m) on this executor, in the style of the paper's
     heat maps (Section IV): block sizes 1 B .. 1 MiB, P up to 256, powers of two and not, every
@@ -863,6 +939,9 @@ def main():
     ap.add_argument("--mapping-study", action="store_true",
                     help="blocks per Sparbit step that cross devices under the sequential and cyclic "
                          "rank-to-device mappings (host only), one JSON line per (P, G, mapping)")
+    ap.add_argument("--multi-emulated", action="store_true",
+                    help="the multi-device executor with G = 1, 2, 4, 8 devices emulated on one GPU "
+                         "(kernel and launch cost only; no NVLink involved)")
     ap.add_argument("--flow-wait-bound", action="store_true",
                     help="the flow executor with and without its waits (timing only): what any finer "
                          "readiness tracking could gain at most")
@@ -877,6 +956,8 @@ def main():
         return run_mapping_study(args)
     if args.allgatherv:
         return run_allgatherv(args)
+    if args.multi_emulated:
+        return run_multi_emulated(args)
     if args.flow_wait_bound:
         return run_flow_wait_bound(args)
     if args.placement_study:

@@ -56,8 +56,10 @@ enum {
     SPARBIT_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sparbit_last_cuda_error() */
     SPARBIT_ERR_TIMEOUT = 7,     /* the device-side grid barrier gave up waiting */
     SPARBIT_ERR_NOMEM = 8,       /* host allocation failed */
-    SPARBIT_ERR_LIMIT = 9        /* beyond a fixed limit of the entry point: the scratch of
+    SPARBIT_ERR_LIMIT = 9,       /* beyond a fixed limit of the entry point: the scratch of
                                     sparbit_allgather_noalloc, P of sparbit_plan_create_v / _validate */
+    SPARBIT_ERR_BARRIER = 10     /* the caller's cross-device barrier (sparbit_allgather_multi)
+                                    returned non-zero */
 };
 
 /* Algorithms (paper, Section II-A and Section III).  Only Sparbit is the product's hot path; the
@@ -272,8 +274,8 @@ int sparbit_plan_validate(const sparbit_plan_t* plan, int* bad_phase);
  * share a machine, so Sparbit's late steps (small distance, most of the data) stay inside it;
  * with the cyclic mapping they are the ones that leave it.  These calls state the same thing for
  * G devices: they split the messages of a phase into the copies a device performs inside its own
- * memory and the blocks it has to hand to each other device.  They only describe the split; this
- * library executes collectives on one device.
+ * memory and the blocks it has to hand to each other device.  They only describe the split; the
+ * sparbit_allgather_multi* calls further down execute it.
  */
 enum {
     SPARBIT_MAP_SEQUENTIAL = 0, /* device g holds ranks [floor(g*P/G), floor((g+1)*P/G)) */
@@ -298,6 +300,83 @@ int sparbit_plan_partition(const sparbit_plan_t* plan, int G, int mapping, int p
  */
 int sparbit_plan_partition_messages(const sparbit_plan_t* plan, int G, int mapping, int phase, int src_device,
                                     int dst_device, sparbit_msg* out, size_t cap, size_t* n);
+
+/*
+ * ---- One communicator on G devices (paper, Section III-C; locality argument of Sections II-B, III)
+ *
+ * The calls above describe the split; these execute it.  Device g holds, packed in increasing
+ * rank order, the send blocks ([n_g][m]) and the receive buffers ([n_g][P][m]) of the n_g ranks
+ * the mapping gives it.  A step of the schedule is one kernel per device: the device that holds
+ * the SENDING rank performs the copy - it reads the block from its own memory (the sender's
+ * receive buffer, as in the single-device executor) and stores it into the receiving rank's
+ * buffer, which is its own memory or, through a plain peer pointer, another device's.  A kernel
+ * never waits for another device.  Algorithm 1's Waitall between steps is a barrier ACROSS the
+ * devices, supplied by the caller.  Sparbit, ring, recursive doubling and neighbor exchange with
+ * fixed-size blocks; Bruck (working buffers, rotation) and variable sizes: ERR_UNSUPPORTED.
+ * The plan is only read: one plan may serve every device of a process, and each process of a
+ * multi-process job creates its own with the same (P, m, algorithm).
+ *
+ * recv_bases: HOST array of G DEVICE pointers, entry g = start of device g's receive buffers as
+ * THIS device can address it (its own allocation for g == device, a peer mapping otherwise; an
+ * entry may be NULL for a device that holds no rank).  The widest vector (16 B down to 1 B) that
+ * divides m and every pointer is used.  Peer access must be enabled by the caller
+ * (cudaDeviceEnablePeerAccess, or sparbit_ipc_open between processes).  All buffers stay owned
+ * by the caller.  1 <= G <= SPARBIT_MULTI_MAX_DEVICES.
+ */
+#define SPARBIT_MULTI_MAX_DEVICES 16
+
+/* Ranks held by `device`; -1 on a bad argument.  Sequential: floor((g+1)P/G) - floor(gP/G). */
+int sparbit_multi_rank_count(int P, int G, int mapping, int device);
+/* Position of `rank` among the ranks of the device that holds it (sparbit_rank_device); -1 on a
+ * bad argument. */
+int sparbit_multi_local_index(int P, int G, int mapping, int rank);
+
+/*
+ * Enqueues on `stream` (of the CURRENT device, which plays `device`) this device's share of the
+ * phases first_phase .. last_phase (-1 .. last phase; a call that runs -1 and 0 executes them as
+ * one pass where the schedule allows).  No barrier is issued: the caller must separate two steps
+ * by a cross-device barrier itself (run one step per call), or be the only "device" that
+ * matters - e.g. all G devices emulated on one GPU and one stream, where stream order is the
+ * barrier.  Errors: ERR_ARG, ERR_UNSUPPORTED, ERR_OVERFLOW, ERR_LIMIT (more than 66 passes in
+ * one call), ERR_CUDA.  Nothing is launched for a device without ranks.
+ */
+int sparbit_allgather_multi_phases(const sparbit_plan_t* plan, int G, int mapping, int device,
+                                   const void* send_local, void* const* recv_bases, void* stream, int first_phase,
+                                   int last_phase);
+
+/*
+ * The cross-device barrier of sparbit_allgather_multi.  It must arrange that work enqueued on
+ * `stream` AFTER it returns starts only when every device's work enqueued BEFORE its own call of
+ * the barrier is complete and visible (e.g. a one-element all-reduce of a communication library
+ * enqueued on `stream`; or cudaStreamSynchronize followed by a host barrier).  0 = success.
+ */
+typedef int (*sparbit_device_barrier_fn)(void* ctx, void* stream);
+
+/*
+ * The whole collective for this device: barrier (every device has entered, its receive buffers
+ * may be written), then pass by pass with a barrier after every communication step - after the
+ * last one too, so that the result is complete when work enqueued after this call runs.  Every
+ * device of the communicator must make the same call.  barrier may be NULL only for G == 1.
+ * Errors as above, and ERR_BARRIER when the barrier returns non-zero (passes already enqueued
+ * stay enqueued).
+ */
+int sparbit_allgather_multi(const sparbit_plan_t* plan, int G, int mapping, int device, const void* send_local,
+                            void* const* recv_bases, void* stream, sparbit_device_barrier_fn barrier,
+                            void* barrier_ctx);
+
+/*
+ * One process per device: how a process lets the others address its receive buffers.  The paper
+ * has no counterpart (MPI moves the bytes there).  sparbit_ipc_export writes the 64-byte handle
+ * of the device allocation that contains dev_ptr and dev_ptr's offset inside it; the allocation
+ * must come from cudaMalloc (not from a pool of mapped virtual memory).  sparbit_ipc_open, in
+ * another process, maps that allocation (enabling peer access to its device where needed) and
+ * returns the same location as *dev_ptr, plus *mapping_base for sparbit_ipc_close.  A process
+ * must not open its own handle; an allocation is opened at most once per process.
+ */
+#define SPARBIT_IPC_HANDLE_BYTES 64
+int sparbit_ipc_export(const void* dev_ptr, void* handle /* 64 bytes, host */, uint64_t* offset);
+int sparbit_ipc_open(const void* handle, uint64_t offset, void** dev_ptr, void** mapping_base);
+int sparbit_ipc_close(void* mapping_base);
 
 /*
  * The same kind of check for the bookkeeping of the FLOW executor, which replaces the Waitall of

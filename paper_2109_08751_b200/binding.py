@@ -13,8 +13,10 @@ import numpy as np
 _LIB_PATH = Path(__file__).resolve().parent / "libsparbit_b200.so"
 
 OK = 0
-ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT = \
-    range(1, 10)
+(ERR_ARG, ERR_OVERFLOW, ERR_ALIAS, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_LIMIT,
+ ERR_BARRIER) = range(1, 11)
+MULTI_MAX_DEVICES = 16
+IPC_HANDLE_BYTES = 64
 ALGO_SPARBIT, ALGO_RING, ALGO_RECURSIVE_DOUBLING, ALGO_BRUCK, ALGO_NEIGHBOR_EXCHANGE = range(5)
 EXEC_AUTO, EXEC_PERSISTENT, EXEC_GRAPH, EXEC_STREAM, EXEC_FLOW, EXEC_MIRROR = range(6)
 COPY_AUTO, COPY_VECTOR, COPY_BULK = range(3)
@@ -55,6 +57,13 @@ SYMBOLS = {
     "sparbit_rank_device": (_i, [_i, _i, _i, _i]),
     "sparbit_plan_partition": (_i, [_vp, _i, _i, _i, ctypes.POINTER(_u64)]),
     "sparbit_plan_partition_messages": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _sz, ctypes.POINTER(_sz)]),
+    "sparbit_multi_rank_count": (_i, [_i, _i, _i, _i]),
+    "sparbit_multi_local_index": (_i, [_i, _i, _i, _i]),
+    "sparbit_allgather_multi_phases": (_i, [_vp, _i, _i, _i, _vp, ctypes.POINTER(_vp), _vp, _i, _i]),
+    "sparbit_allgather_multi": (_i, [_vp, _i, _i, _i, _vp, ctypes.POINTER(_vp), _vp, _vp, _vp]),
+    "sparbit_ipc_export": (_i, [_vp, _vp, ctypes.POINTER(_u64)]),
+    "sparbit_ipc_open": (_i, [_vp, _u64, ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
+    "sparbit_ipc_close": (_i, [_vp]),
     "sparbit_plan_workspace_bytes": (_sz, [_vp]),
     "sparbit_plan_set_workspace": (_i, [_vp, _vp, _sz]),
     "sparbit_plan_set_copy_path": (_i, [_vp, _i]),
@@ -82,6 +91,10 @@ for _name, (_res, _args) in SYMBOLS.items():
     _fn = getattr(lib, _name)  # AttributeError here means the library does not match the header
     _fn.restype = _res
     _fn.argtypes = _args
+
+
+#: sparbit_device_barrier_fn
+BARRIER_FN = ctypes.CFUNCTYPE(_i, _vp, _vp)
 
 
 class SparbitError(RuntimeError):
@@ -196,6 +209,36 @@ class Plan:
                    "sparbit_plan_partition_messages")
         return out
 
+    # -- one communicator on G devices
+    def allgather_multi_phases(self, G: int, mapping: int, device: int, send_local, recv_bases, first: int,
+                               last: int, stream=None) -> None:
+        """This device's share of phases first..last (no cross-device barrier is issued)."""
+        bases = (_vp * G)(*[_ptr(b) for b in recv_bases])
+        _check(lib.sparbit_allgather_multi_phases(self._h, G, mapping, device, _ptr(send_local), bases,
+                                                  _stream_handle(stream), first, last),
+               "sparbit_allgather_multi_phases")
+
+    def allgather_multi(self, G: int, mapping: int, device: int, send_local, recv_bases, barrier,
+                        stream=None) -> None:
+        """The whole collective for this device; `barrier(stream_handle)` is the cross-device
+        barrier (returns None/0 on success), called K + 1 times by the library."""
+        bases = (_vp * G)(*[_ptr(b) for b in recv_bases])
+        failure = []
+
+        def _cb(_ctx, stream_handle):
+            try:
+                return int(barrier(stream_handle) or 0)
+            except BaseException as e:  # an exception must not unwind through the C frames
+                failure.append(e)
+                return 1
+
+        cb = BARRIER_FN(_cb) if barrier is not None else None
+        code = lib.sparbit_allgather_multi(self._h, G, mapping, device, _ptr(send_local), bases,
+                                           _stream_handle(stream), ctypes.cast(cb, _vp) if cb else None, None)
+        if failure:
+            raise failure[0]
+        _check(code, "sparbit_allgather_multi")
+
     def validate(self) -> None:
         """Host-side race and bounds check of the descriptors (raises with the offending phase)."""
         bad = ctypes.c_int()
@@ -286,6 +329,33 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+def multi_rank_count(P: int, G: int, mapping: int, device: int) -> int:
+    return lib.sparbit_multi_rank_count(P, G, mapping, device)
+
+
+def multi_local_index(P: int, G: int, mapping: int, rank: int) -> int:
+    return lib.sparbit_multi_local_index(P, G, mapping, rank)
+
+
+def ipc_export(dev_ptr) -> tuple[bytes, int]:
+    """(64-byte handle, offset) of the device allocation that contains dev_ptr."""
+    h = ctypes.create_string_buffer(IPC_HANDLE_BYTES)
+    off = _u64()
+    _check(lib.sparbit_ipc_export(_ptr(dev_ptr), h, ctypes.byref(off)), "sparbit_ipc_export")
+    return h.raw, int(off.value)
+
+
+def ipc_open(handle: bytes, offset: int) -> tuple[int, int]:
+    """(device address of the exported location, mapping base for ipc_close)."""
+    ptr, base = _vp(), _vp()
+    _check(lib.sparbit_ipc_open(handle, offset, ctypes.byref(ptr), ctypes.byref(base)), "sparbit_ipc_open")
+    return int(ptr.value), int(base.value)
+
+
+def ipc_close(mapping_base: int) -> None:
+    _check(lib.sparbit_ipc_close(mapping_base), "sparbit_ipc_close")
 
 
 def sparbit_plan(P: int, block_bytes: int) -> Plan:

@@ -12,8 +12,8 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libsparbit_b200.so"
-SOURCES = [CSRC / "api.cu", CSRC / "schedule.cpp"]
-HEADERS = [CSRC / "kernels.cuh", CSRC / "phase_desc.h", CSRC / "schedule.h",
+SOURCES = [CSRC / "api.cu", CSRC / "multi.cu", CSRC / "schedule.cpp"]
+HEADERS = [CSRC / "kernels.cuh", CSRC / "phase_desc.h", CSRC / "schedule.h", CSRC / "plan_access.h",
            HERE.parent / "include" / "sparbit.h"]
 
 NVCC_FLAGS = [

@@ -1338,6 +1338,13 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
 
 }  // namespace
 
+// What the multi-device entry points (multi.cu) need of a plan and of this file's error record.
+namespace spb {
+const Schedule* plan_schedule(const sparbit_plan_s* p) { return p ? &p->sched : nullptr; }
+bool plan_is_variable(const sparbit_plan_s* p) { return p && p->variable; }
+int record_cuda_error(int cuda_error, const char* what) { return cuda_fail((cudaError_t)cuda_error, what); }
+}  // namespace spb
+
 extern "C" {
 
 int sparbit_plan_create(int P, size_t block_bytes, int algo, int exec, sparbit_plan_t** out) {
@@ -1852,6 +1859,7 @@ const char* sparbit_strerror(int code) {
         case SPARBIT_ERR_TIMEOUT: return "device barrier timed out";
         case SPARBIT_ERR_NOMEM: return "out of host memory";
         case SPARBIT_ERR_LIMIT: return "beyond a fixed limit of this entry point (scratch size or rank count)";
+        case SPARBIT_ERR_BARRIER: return "the caller's cross-device barrier failed";
         default: return "unknown error";
     }
 }
