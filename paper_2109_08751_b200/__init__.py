@@ -16,7 +16,7 @@ def __getattr__(name):
     global _binding
     if name.startswith("__"):
         raise AttributeError(name)
-    if name in ("build", "binding"):  # submodules
+    if name in ("build", "binding", "multi"):  # submodules
         return importlib.import_module("." + name, __name__)
     if _binding is None:
         _binding = importlib.import_module(".binding", __name__)

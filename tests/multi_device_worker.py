@@ -67,6 +67,24 @@ def main():
             sp.ipc_close(opened.pop())
         dist.barrier()  # nobody frees an allocation that is still mapped elsewhere
         del recv, send
+    # the same through the package's torch.distributed wrapper, two collectives in a row
+    for P, m in ((21, 528), (32, 8192)):
+        ag = sp.multi.MultiDeviceAllgather(P, m, mapping=mapping, device=dev)
+        for seed in (1, 2):
+            host_send = si.send_blocks(P, m, seed=70 + seed)
+            send = torch.from_numpy(np.ascontiguousarray(host_send[ag.ranks]).reshape(-1)).to(dev)
+            ag.recv.fill_(si.SENTINEL)
+            torch.cuda.synchronize()
+            dist.barrier()  # nobody stores into a buffer that is still being filled
+            with torch.cuda.stream(stream):
+                got = ag.allgather(send)
+            stream.synchronize()
+            want, _ = oracle.allgather(sp.ALGO_SPARBIT, P, m, host_send)
+            got = got.cpu().numpy()[: ag.n_local * P * m].reshape(ag.n_local, P * m)
+            for li, r in enumerate(ag.ranks):
+                assert np.array_equal(got[li], want[r]), ("wrapper", P, m, "rank", r)
+        assert ag.barrier_calls == 2 * (ag.plan.num_steps + 1)
+        ag.close()
     dist.destroy_process_group()
     print("multi-device worker ok", me)
 
