@@ -817,7 +817,7 @@ def run_multi_emulated(args):
     line({"devices": 1, "mapping": "-", "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}"},
          us, bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1])))
     del recv
-    for G in (1, 2, 4, 8):
+    for G in args.multi_devices:
         for name, mp in (("sequential", sp.MAP_SEQUENTIAL), ("cyclic", sp.MAP_CYCLIC)):
             ranks = [[r for r in range(P) if rdev(P, G, mp, r) == g] for g in range(G)]
             dsend = [[torch.from_numpy(np.ascontiguousarray(h[ranks[g]]).reshape(-1)).to(dev) for g in range(G)]
@@ -942,6 +942,8 @@ def main():
     ap.add_argument("--multi-emulated", action="store_true",
                     help="the multi-device executor with G = 1, 2, 4, 8 devices emulated on one GPU "
                          "(kernel and launch cost only; no NVLink involved)")
+    ap.add_argument("--multi-devices", type=int, nargs="+", default=[1, 2, 4, 8],
+                    help="with --multi-emulated: the device counts to run")
     ap.add_argument("--flow-wait-bound", action="store_true",
                     help="the flow executor with and without its waits (timing only): what any finer "
                          "readiness tracking could gain at most")

@@ -181,6 +181,42 @@ def test_larger_collectives_several_tiles_and_a_ragged_tail(dev, algo, P, m, G, 
     em.check(want.reshape(-1))
 
 
+def random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        algo = int(rng.choice([sp.ALGO_SPARBIT] * 3 + [sp.ALGO_RING, sp.ALGO_RECURSIVE_DOUBLING,
+                                                       sp.ALGO_NEIGHBOR_EXCHANGE]))
+        P = int(rng.integers(1, 97))
+        if algo == sp.ALGO_RECURSIVE_DOUBLING:
+            P = 1 << int(rng.integers(0, 7))
+        if algo == sp.ALGO_NEIGHBOR_EXCHANGE:
+            P += P & 1
+        if algo == sp.ALGO_RING and P > 24:
+            P = int(rng.integers(1, 25))
+        m = int(rng.choice([1, 3, 8, 24, 64, 100, 272, 1040, 4096, 5000, 16400]))
+        G = int(rng.integers(1, 17))  # more devices than ranks happens: some devices hold nothing
+        out.append((algo, P, m, G, int(rng.integers(0, 2)), int(rng.choice([0, 0, 1, 2, 4, 8]))))
+    return out
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", random_cases(80, 20211), ids=lambda c: "-".join(map(str, c)))
+def test_random_cases_on_emulated_devices(dev, case):
+    algo, P, m, G, mapping, misalign = case
+    plan = sp.Plan(P, m, algo)
+    em = Emulated(dev, P, m, G, mapping, seed=P + m, misalign=misalign)
+    assert [len(r) for r in em.ranks] == [sp.multi_rank_count(P, G, mapping, g) for g in range(G)]
+    for g in range(G):
+        plan.allgather_multi_phases(G, mapping, g, em.send[g], em.bases, -1, min(0, plan.last_phase))
+    for ph in range(1, plan.last_phase + 1):
+        for g in range(G):
+            plan.allgather_multi_phases(G, mapping, g, em.send[g], em.bases, ph, ph)
+    torch.cuda.synchronize()
+    want, _ = oracle.allgather(algo, P, m, em.host_send)
+    em.check(want.reshape(-1))
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("mapping", MAPPINGS)
 @pytest.mark.parametrize("P,m,G", [(13, 272, 3), (32, 4096, 4), (8, 64, 8)])
