@@ -444,7 +444,9 @@ def run_ours(args):
             "pct_of_nominal_hbm": 100.0 * value / world / NOMINAL_HBM_GBS,
             "GBps_from_min_time": world * effective_bytes(P, m) / (min(per_ms) * 1e-3) / 1e9,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            # kernels of this library per round of --steps collectives; the timed region is `rounds` rounds
             "gpu_launches": int((k1 - k0) // rounds), "graph_launches": int((g1 - g0) // rounds),
+            "gpu_launches_timed_region": int(k1 - k0),
             "clocks": clocks, "checked": bool(checked),
         }
         print(json.dumps(line), flush=True)
