@@ -55,6 +55,15 @@ int main(void) {
         CHECK(sparbit_plan_get_tunable(plan, SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES, &v) == SPARBIT_OK && v == 8192);
         CHECK(sparbit_plan_set_tunable(plan, SPARBIT_TUNE_COUNT_, 1) == SPARBIT_ERR_ARG);
         CHECK(sparbit_rank_device(13, 2, SPARBIT_MAP_SEQUENTIAL, 6) == 1 && sparbit_rank_device(13, 2, SPARBIT_MAP_CYCLIC, 6) == 0);
+        /* 13 ranks on 2 devices: 6 + 7 under the sequential mapping, 7 + 6 under the cyclic one */
+        CHECK(sparbit_multi_rank_count(13, 2, SPARBIT_MAP_SEQUENTIAL, 0) == 6 && sparbit_multi_rank_count(13, 2, SPARBIT_MAP_CYCLIC, 0) == 7);
+        CHECK(sparbit_multi_local_index(13, 2, SPARBIT_MAP_SEQUENTIAL, 6) == 0 && sparbit_multi_local_index(13, 2, SPARBIT_MAP_CYCLIC, 6) == 3);
+        {
+            void* bases[2] = {(void*)(1 << 20), NULL};
+            /* the second device's buffers are missing; more devices than the table holds */
+            CHECK(sparbit_allgather_multi_phases(plan, 2, SPARBIT_MAP_SEQUENTIAL, 0, (const void*)4096, bases, NULL, -1, 0) == SPARBIT_ERR_ARG);
+            CHECK(sparbit_allgather_multi(plan, SPARBIT_MULTI_MAX_DEVICES + 1, SPARBIT_MAP_SEQUENTIAL, 0, (const void*)4096, bases, NULL, NULL, NULL) == SPARBIT_ERR_ARG);
+        }
     }
     /* argument errors are found before anything touches a device */
     CHECK(sparbit_allgather(plan, NULL, NULL, NULL) == SPARBIT_ERR_ARG);
