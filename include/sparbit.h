@@ -79,7 +79,10 @@ enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
                                     buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB,
                                     where the chain with a grouped front is not at least as
-                                    fast), FLOW for collectives that move 0.45 to 6 GB, the graph
+                                    fast), FLOW for collectives that move 0.45 to 6 GB (unless
+                                    COPY_AUTO gives them the bulk engine and m is not a multiple
+                                    of 128 B: the vector engine, which FLOW runs on, is 10-30 %
+                                    slower on blocks that straddle 128-byte lines), the graph
                                     chain otherwise (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch

@@ -536,12 +536,26 @@ int small_collective_exec(const sparbit_plan_s* p, int vbytes, int first, int la
     return SPARBIT_EXEC_MIRROR;
 }
 
+// COPY_AUTO gives this plan the bulk engine and its blocks do not start on 128-byte lines.  The
+// vector engine pays 10-30 % for such blocks (every warp row straddles lines; P = 128, m = 65520 B:
+// 406 us in the chain, 363 in the flow kernel, against 331 at m = 65536 B), the bulk engine 2 %
+// (345 us): the flow executor, which runs on the vector engine only, is then not worth leaving
+// the bulk engine for.
+bool bulk_off_line(const sparbit_plan_s* p, int vbytes) {
+    if (p->variable || p->copy_req != SPARBIT_COPY_AUTO || vbytes != 16) return false;
+    const uint64_t m = p->sched.m;
+    const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
+    return (m & 127u) != 0 && m >= p->tune[SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES] &&
+           moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_BULK_MIN_MOVED_BYTES];
+}
+
 int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
     const int small = small_collective_exec(p, vbytes, first, last, (size_t)p->max_smem_optin);
     if (small >= 0) return small;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
-        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && flow_possible(p, vbytes, first, last))
+        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && !bulk_off_line(p, vbytes) &&
+        flow_possible(p, vbytes, first, last))
         return SPARBIT_EXEC_FLOW;
     return SPARBIT_EXEC_GRAPH;
 }
@@ -551,7 +565,7 @@ int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
     if (small >= 0) return small;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
-        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] &&
+        moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && !bulk_off_line(p, vbytes) &&
         flow_possible(p, vbytes, -1, p->sched.last_phase(), true))
         return SPARBIT_EXEC_FLOW;
     return SPARBIT_EXEC_GRAPH;

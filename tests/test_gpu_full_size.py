@@ -24,7 +24,7 @@ def dev():
     return torch.device("cuda:0")
 
 
-def full_compare(dev, P, m, algo, exec_mode, copy, seed, iters=2):
+def full_compare(dev, P, m, algo, exec_mode, copy, seed, iters=2, ran_on=None):
     plan = sp.Plan(P, m, algo, exec_mode)
     plan.set_copy_path(copy)
     ref = oracle.Plan(algo, P)
@@ -43,6 +43,8 @@ def full_compare(dev, P, m, algo, exec_mode, copy, seed, iters=2):
             work.fill_(si.SENTINEL)
         plan.allgather(send, recv)
         assert plan.status() == sp.OK
+        if ran_on is not None:
+            assert (plan.exec_mode, plan.copy_path) == ran_on
         want.fill(si.SENTINEL)
         if scratch is not None:
             scratch.fill(si.SENTINEL)
@@ -68,6 +70,12 @@ def test_config3_p128_m64k_flow(dev):
 
 def test_config3_auto_is_what_the_benchmark_runs(dev):
     full_compare(dev, 128, 64 * 1024, sp.ALGO_SPARBIT, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 3, iters=1)
+
+
+def test_blocks_off_128_byte_lines_auto_keeps_the_bulk_engine(dev):
+    # 1.07 GB moved, m a multiple of 16 but not of 128: AUTO leaves the flow executor aside
+    full_compare(dev, 128, 32752, sp.ALGO_SPARBIT, sp.EXEC_AUTO, sp.COPY_AUTO, si.BASE_SEED + 3, iters=1,
+                 ran_on=(sp.EXEC_GRAPH, sp.COPY_BULK))
 
 
 # config 4: many small blocks, non-power-of-two; graph chain vs persistent

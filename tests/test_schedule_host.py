@@ -152,6 +152,9 @@ def test_exec_mode_resolution():
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
     assert sp.Plan(256, 4096).exec_mode == sp.EXEC_FLOW           # 0.53 GB moved
     assert sp.Plan(128, 8192).exec_mode == sp.EXEC_GRAPH          # 0.27 GB moved
+    assert sp.Plan(128, 65520).exec_mode == sp.EXEC_GRAPH         # blocks off 128-byte lines stay on the bulk engine
+    assert sp.Plan(128, 65520, ).exec_mode != sp.Plan(128, 65536).exec_mode
+    assert sp.Plan(1000, 1008).exec_mode == sp.EXEC_FLOW          # ... where COPY_AUTO would pick it (m >= 8 KiB)
     assert sp.Plan(40000, 1).exec_mode == sp.EXEC_GRAPH           # blocks shorter than a warp row
     assert sp.Plan(256, 65536, exec_mode=sp.EXEC_PERSISTENT).exec_mode == sp.EXEC_PERSISTENT
 
