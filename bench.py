@@ -520,7 +520,11 @@ def run_sweep(args):
              "bruck": sp.ALGO_BRUCK, "ne": sp.ALGO_NEIGHBOR_EXCHANGE}
     execs = {"persistent": sp.EXEC_PERSISTENT, "graph": sp.EXEC_GRAPH, "stream": sp.EXEC_STREAM,
              "flow": sp.EXEC_FLOW, "mirror": sp.EXEC_MIRROR}
-    if args.sweep == "engines":
+    if args.sweep == "offline":  # block sizes that are not a multiple of 128 B beside neighbours that are
+        points += [(P, m, ["sparbit"]) for P, m in (
+            (256, 2032), (256, 2048), (256, 4080), (256, 4096), (256, 16368), (256, 16384),
+            (128, 65520), (128, 65536), (1000, 1008), (1000, 1024))]
+    if args.sweep in ("engines", "offline"):
         execs = {"graph": sp.EXEC_GRAPH, "flow": sp.EXEC_FLOW}
     if args.sweep == "mirror":  # where the mirror executor (one CTA, then a cluster) wins and where it stops winning
         points += [(P, m, ["sparbit"]) for P, m in (
@@ -927,7 +931,7 @@ def main():
                          "(0 = one round, for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "mirror", "all"], default=None,
+    ap.add_argument("--sweep", choices=["small", "config3", "config4", "config5", "engines", "mirror", "offline", "all"], default=None,
                     help="print latency/bandwidth curves (one JSON line per point) instead of the bench line")
     ap.add_argument("--no-grouped-front", action="store_true",
                     help="every pass of the graph and stream executors as its own kernel (SPARBIT_TUNE_GROUPED_FRONT = 0)")

@@ -455,7 +455,13 @@ enum {
                                               buffers (one kernel instead of one per pass), as far as a
                                               group's part stays within MIRROR_MAX_BYTES; 0 = every pass its
                                               own kernel */
-    SPARBIT_TUNE_COUNT_ = 15
+    SPARBIT_TUNE_FLOW_WIDE_MAX_MOVED_BYTES = 15, /* EXEC_FLOW: a collective that moves less than this (9*10^8)
+                                              in blocks of at least 256 vectors (4 KiB) runs the flow kernel
+                                              with four vectors per lane (warp spans of 2 KiB) instead of
+                                              two: much of it is served by L2, which takes more loads in
+                                              flight than DRAM rewards (P = 256, m = 4 KiB: 85.0 us against
+                                              90.3); 0 = never */
+    SPARBIT_TUNE_COUNT_ = 16
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

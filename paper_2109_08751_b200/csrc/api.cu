@@ -88,7 +88,7 @@ struct sparbit_plan_s {
     unsigned* d_ctl = nullptr;  // [0] barrier counter, [1] status word
     unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
     unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
-    int flow_vbytes = 0;             // vector width those launches ran with
+    int flow_vbytes = 0;             // vector width and vectors per lane (width * 16 + unroll) of those launches
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -117,6 +117,7 @@ struct sparbit_plan_s {
         0,            // FLOW_COOPERATIVE
         0,            // FLOW_SKIP_WAITS
         1,            // GROUPED_FRONT
+        900000000u,   // FLOW_WIDE_MAX_MOVED_BYTES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -337,15 +338,19 @@ const void* pick_cluster_mirror_vec(int vbytes) {
         default: return cluster_mirror_vec_fn<unsigned char>();
     }
 }
+constexpr int kFlowWideUnroll = 4;  // vectors per lane of the flow kernel's wide form
 template <typename V>
-const void* flow_vec_fn() { return (const void*)flow_vec_kernel<V, kVecUnroll>; }
-const void* pick_flow_vec(int vbytes) {
+const void* flow_vec_fn(int unroll) {
+    return unroll == kFlowWideUnroll ? (const void*)flow_vec_kernel<V, kFlowWideUnroll>
+                                     : (const void*)flow_vec_kernel<V, kVecUnroll>;
+}
+const void* pick_flow_vec(int vbytes, int unroll) {
     switch (vbytes) {
-        case 16: return flow_vec_fn<uint4>();
-        case 8: return flow_vec_fn<uint2>();
-        case 4: return flow_vec_fn<unsigned>();
-        case 2: return flow_vec_fn<unsigned short>();
-        default: return flow_vec_fn<unsigned char>();
+        case 16: return flow_vec_fn<uint4>(unroll);
+        case 8: return flow_vec_fn<uint2>(unroll);
+        case 4: return flow_vec_fn<unsigned>(unroll);
+        case 2: return flow_vec_fn<unsigned short>(unroll);
+        default: return flow_vec_fn<unsigned char>(unroll);
     }
 }
 
@@ -435,14 +440,32 @@ bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_l
 // 2 % faster than any split (one launch instead of several, and the small passes overlap their
 // neighbours), so the default is 1.  Returns the position of the first flow pass, or the sequence
 // length if there is none.
+// Vectors per lane and warp span in the flow kernel.  A collective that moves less than
+// FLOW_WIDE_MAX_MOVED_BYTES in blocks of at least two wide spans (4 KiB in 16-byte vectors) runs
+// with four instead of two: half of such a collective lives in L2, which answers faster than the
+// 32 KiB of loads in flight per SM that suit DRAM can keep busy (P = 256, m = 4 KiB: 85.0 us
+// against 90.3; P = 128, m = 16 KiB: 84.3 against 88.0; P = 256, m = 6 KiB: 125.6 against 129.7).
+// From about 1 GB moved the narrow form wins (P = 256, m = 8 KiB: 168.6 us against 174.4; P = 128,
+// m = 64 KiB: 330.7 against 346.7), and smaller blocks leave a wide span half empty.
+int flow_unroll(const sparbit_plan_s* p, int vbytes) {
+    if (p->variable) return kVecUnroll;
+    const uint64_t m = p->sched.m;
+    const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
+    if (moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_WIDE_MAX_MOVED_BYTES] &&
+        m / (uint64_t)vbytes >= 2ull * 32 * kFlowWideUnroll)
+        return kFlowWideUnroll;
+    return kVecUnroll;
+}
+
 int flow_first_pass(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint64_t max_warps) {
+    const uint64_t span = 32ull * flow_unroll(p, vbytes);
     const int n = seq.count();
     int f = n;
     for (int i = n - 1; i >= 0 && n - i <= kFlowMaxPasses; i--) {
         const PhaseDesc& d = seq.item(i);
         const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
         if (vpc < 32) break;
-        const uint64_t spc = (vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll);
+        const uint64_t spc = (vpc + span - 1) / span;
         const uint64_t spans = (uint64_t)p->sched.P * d.copies * spc;
         if (spans >> 31) break;
         const uint64_t least = p->tune[SPARBIT_TUNE_FLOW_MIN_PASS_SPANS] ? p->tune[SPARBIT_TUNE_FLOW_MIN_PASS_SPANS] : max_warps;
@@ -1185,7 +1208,8 @@ uint64_t flow_pass_table(const sparbit_plan_s* p, const ExecSeq& seq, int f, int
         const PhaseDesc& d = seq.item(f + i);
         FlowPass& fp = fa.pass[i];
         const uint64_t vpc = d.copy_bytes / (uint64_t)vbytes;
-        fp.spc = (uint32_t)((vpc + 32ull * kVecUnroll - 1) / (32ull * kVecUnroll));
+        const uint64_t span = 32ull * flow_unroll(p, vbytes);
+        fp.spc = (uint32_t)((vpc + span - 1) / span);
         const uint64_t spans = (uint64_t)d.copies * fp.spc;  // per source rank
         // Unit size: a small pass is cut into single spans, so that as many warps as possible share
         // it and a hop (copy, release, the next pass's poll) stays short; a pass that keeps every
@@ -1228,7 +1252,8 @@ FlowStream g_flow_last[kFlowDevices];
 int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first, int last, cudaStream_t st) {
     const uint32_t P = p->sched.P;
     const ExecSeq seq = make_seq(p, first, last);
-    const void* fn = pick_flow_vec(rs.vbytes);
+    const int unroll = flow_unroll(p, rs.vbytes);
+    const void* fn = pick_flow_vec(rs.vbytes, unroll);
     int per_sm = 0;
     CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kVecBlock, 0));
     if (per_sm < 1) return cuda_fail(cudaErrorLaunchOutOfResources, "flow kernel does not fit on an SM");
@@ -1245,12 +1270,12 @@ int launch_flow(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int first,
         p->flow_epoch = 0;
         p->flow_vbytes = 0;
     }
-    if (p->flow_vbytes != rs.vbytes || p->flow_epoch == 0) {
-        // counters count units, and a unit's size follows the vector width: start over
+    if (p->flow_vbytes != rs.vbytes * 16 + unroll || p->flow_epoch == 0) {
+        // counters count units, and a unit's size follows the vector width and the span: start over
         // (with leading per-pass kernels in front this memset sits between kernels: rare, and correct)
         CU(cudaMemsetAsync(p->d_flow_cnt, 0, (size_t)P * kFlowMaxPasses * sizeof(unsigned), st));
         p->flow_epoch = 0;
-        p->flow_vbytes = rs.vbytes;
+        p->flow_vbytes = rs.vbytes * 16 + unroll;
     }
     p->flow_epoch++;
     FlowArgs fa;

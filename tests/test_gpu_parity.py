@@ -450,7 +450,9 @@ def test_two_flow_collectives_at_once(dev):
 def test_flow_all_algorithms_changing_data(dev, algo):
     """Every algorithm on the flow executor, several calls in a row on one plan (the counters
     carry over from call to call) with new data and a fresh sentinel fill each time."""
-    for P, m in ((16, 2048), (12, 1024), (64, 512), (13, 4096), (1, 512), (2, 8192)):
+    narrow = dict(ALL_IN_FLOW)
+    narrow[sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES] = 0   # two vectors per lane whatever the block size
+    for P, m in ((16, 2048), (12, 1024), (64, 512), (13, 4096), (1, 512), (2, 8192), (5, 4144), (24, 12304)):
         if algo == sp.ALGO_RECURSIVE_DOUBLING and not is_pow2(P):
             continue
         if algo == sp.ALGO_NEIGHBOR_EXCHANGE and P % 2:
@@ -459,6 +461,8 @@ def test_flow_all_algorithms_changing_data(dev, algo):
             continue   # more passes than the flow executor's counter line holds: runs as a graph
         run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 77 + P, iters=3, tune=ALL_IN_FLOW, ran=sp.EXEC_FLOW)
         run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 78 + P, iters=2, tune=SPLIT_FLOW)
+        if m >= 4096:   # by default these run with four vectors per lane
+            run_case(dev, P, m, algo, sp.EXEC_FLOW, sp.COPY_AUTO, 79 + P, iters=2, tune=narrow, ran=sp.EXEC_FLOW)
 
 
 @pytest.mark.parametrize("algo", ALGOS)

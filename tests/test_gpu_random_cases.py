@@ -51,7 +51,9 @@ def test_random_cases(dev, chunk):
         tune = None
         if exec_mode == sp.EXEC_FLOW and rng.integers(2):
             tune = {sp.TUNE_FLOW_MIN_PASS_SPANS: int(rng.choice([0, 1, 40])),
-                    sp.TUNE_FLOW_COOPERATIVE: int(rng.integers(2))}
+                    sp.TUNE_FLOW_COOPERATIVE: int(rng.integers(2)),
+                    # two vectors per lane, or four wherever blocks are long enough for it
+                    sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES: 0 if done % 2 else 10 ** 12}
         if exec_mode == sp.EXEC_MIRROR and rng.integers(2):
             tune = {sp.TUNE_MIRROR_CTA_VECTORS: int(rng.choice([16, 64, 256, 4096])),
                     sp.TUNE_MIRROR_THREAD_VECTORS: int(rng.choice([1, 2, 4, 8])),

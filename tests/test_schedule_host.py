@@ -218,21 +218,28 @@ def test_flow_units_and_counters_are_consistent(algo):
             plan = sp.Plan(P, m, algo)
             plan.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)   # a pass needs one span per resident warp
             passes = plan.last_phase + 2 - (1 if algo != sp.ALGO_BRUCK and P > 1 else 0)   # fused first pass
-            firsts = []
-            for warps in (1, 64, 4736):
-                code = plan.validate_flow(vb, warps)
-                assert code in (sp.OK, sp.ERR_UNSUPPORTED)
-                if warps == 1:
-                    assert code == sp.OK and plan.first_flow_pass == max(0, passes - 32), (algo, P, m)
-                firsts.append(plan.first_flow_pass if code == sp.OK else passes)
-                ran += code == sp.OK
-            assert firsts == sorted(firsts), (algo, P, m, firsts)
+            # spans of four vectors per lane (blocks of 256 vectors and more, up to the given bytes
+            # moved) and of two
+            for wide_below in (10 ** 12, 0):
+                plan.set_tunable(sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES, wide_below)
+                firsts = []
+                for warps in (1, 64, 4736):
+                    code = plan.validate_flow(vb, warps)
+                    assert code in (sp.OK, sp.ERR_UNSUPPORTED)
+                    if warps == 1:
+                        assert code == sp.OK and plan.first_flow_pass == max(0, passes - 32), (algo, P, m)
+                    firsts.append(plan.first_flow_pass if code == sp.OK else passes)
+                    ran += code == sp.OK
+                assert firsts == sorted(firsts), (algo, P, m, firsts)
             plan.destroy()
-    assert ran > 60
+    assert ran > 120
     assert sp.Plan(8, 64).validate_flow(16, 1) == sp.ERR_UNSUPPORTED   # blocks shorter than a warp row
     big = sp.Plan(256, 4096)
     assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 0   # by default every pass
     big.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)
+    assert big.get_tunable(sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES) == 9 * 10 ** 8   # 0.53 GB moved: spans of 2 KiB
+    assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 4   # 8192 of them in pass 4
+    big.set_tunable(sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES, 0)                      # spans of 1 KiB
     assert big.validate_flow(16, 4736) == sp.OK and big.first_flow_pass == 3   # 8192 spans in pass 3
 
 
