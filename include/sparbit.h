@@ -461,7 +461,11 @@ enum {
                                               two: much of it is served by L2, which takes more loads in
                                               flight than DRAM rewards (P = 256, m = 4 KiB: 85.0 us against
                                               90.3); 0 = never */
-    SPARBIT_TUNE_COUNT_ = 16
+    SPARBIT_TUNE_VEC_DENSE_MAX_RECV_BYTES = 16, /* GRAPH and STREAM executors, vector engine: while the receive
+                                              buffers total at most this (256 MiB, about twice the L2) a full
+                                              per-pass kernel runs three CTAs per SM instead of two (1-5 %:
+                                              P = 256, m = 2 KiB 45.4 us against 46.7); 0 = never */
+    SPARBIT_TUNE_COUNT_ = 17
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

@@ -118,6 +118,7 @@ struct sparbit_plan_s {
         0,            // FLOW_SKIP_WAITS
         1,            // GROUPED_FRONT
         900000000u,   // FLOW_WIDE_MAX_MOVED_BYTES
+        256u << 20,   // VEC_DENSE_MAX_RECV_BYTES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -686,13 +687,19 @@ int plan_phase_launch(sparbit_plan_s* p, const Resolved& rs, const PhaseDesc& d,
         if (tasks >> 32) return SPARBIT_ERR_OVERFLOW;
         const uint64_t wpb = kVecBlock / 32;
         uint64_t ctas = (tasks + wpb - 1) / wpb;
-        const uint64_t cap = (uint64_t)p->sm_count * 2;  // 1024 threads x 2 vectors in flight per SM
+        // 1024 threads x 2 vectors in flight per SM suit DRAM.  Receive buffers of up to about twice the
+        // L2 are served by L2 for a good part, which rewards a third CTA per SM (what the kernel's 40
+        // registers allow): P = 256, m = 2 KiB 45.4 us against 46.7; P = 512, m = 512 B 61.4 against
+        // 64.9; P = 512, m = 1 KiB 89.9 against 91.2; a fourth (fewer registers) gave nothing.
+        const bool dense = (unsigned __int128)P * P * p->sched.m <=
+                           (unsigned __int128)p->tune[SPARBIT_TUNE_VEC_DENSE_MAX_RECV_BYTES];
+        const uint64_t cap = (uint64_t)p->sm_count * (dense ? 3 : 2);
         if (ctas > cap) ctas = cap;
         if (ctas < 1) ctas = 1;
         pl.fn = pick_phase_vec(rs.vbytes);
         pl.grid = dim3((unsigned)ctas);
         pl.block = dim3(kVecBlock);
-        pl.smem = ctas == cap ? kVecOccupancySmem : 0;
+        pl.smem = ctas == cap && !dense ? kVecOccupancySmem : 0;
     }
     return SPARBIT_OK;
 }

@@ -165,6 +165,7 @@ def test_engine_thresholds_are_plan_fields():
     assert plan.get_tunable(sp.TUNE_BULK_MIN_MOVED_BYTES) == 10 ** 9
     plan.set_tunable(sp.TUNE_BULK_MIN_BLOCK_BYTES, 4096)
     assert plan.get_tunable(sp.TUNE_BULK_MIN_BLOCK_BYTES) == 4096
+    assert plan.get_tunable(sp.TUNE_VEC_DENSE_MAX_RECV_BYTES) == 256 << 20
     with pytest.raises(sp.binding.SparbitError):
         plan.set_tunable(99, 1)
 
