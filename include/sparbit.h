@@ -79,7 +79,7 @@ enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
                                     buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB,
                                     where the chain with a grouped front is not at least as
-                                    fast), FLOW for collectives that move 0.45 to 6 GB (unless
+                                    fast), FLOW for collectives that move 0.4 to 6 GB (unless
                                     COPY_AUTO gives them the bulk engine and m is not a multiple
                                     of 128 B: the vector engine, which FLOW runs on, is 10-30 %
                                     slower on blocks that straddle 128-byte lines), the graph
@@ -418,7 +418,7 @@ enum {
     SPARBIT_TUNE_FLOW_UNITS_PER_WARP = 2,  /* EXEC_FLOW: a pass is cut into units of 1..4 warp spans
                                               so that every warp gets at least about this many (1) */
     SPARBIT_TUNE_FLOW_MAX_UNIT_SPANS = 3,  /* EXEC_FLOW: largest unit, in warp spans of 1 KiB (8) */
-    SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (4.5*10^8) */
+    SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES = 4, /* EXEC_AUTO: FLOW when 2*P*(P-1)*m is at least this (4*10^8) */
     SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES = 5, /* ... and below this (6*10^9); GRAPH otherwise */
     SPARBIT_TUNE_MIRROR_MAX_BYTES = 6,     /* EXEC_AUTO: MIRROR when P*P*m is at most this (64 KiB) */
     SPARBIT_TUNE_FLOW_MIN_PASS_SPANS = 7,  /* EXEC_FLOW: the flow kernel takes the passes at the end of
@@ -456,7 +456,7 @@ enum {
                                               group's part stays within MIRROR_MAX_BYTES; 0 = every pass its
                                               own kernel */
     SPARBIT_TUNE_FLOW_WIDE_MAX_MOVED_BYTES = 15, /* EXEC_FLOW: a collective that moves less than this (9*10^8)
-                                              in blocks of at least 256 vectors (4 KiB) runs the flow kernel
+                                              in blocks of at least 128 vectors (2 KiB) runs the flow kernel
                                               with four vectors per lane (warp spans of 2 KiB) instead of
                                               two: much of it is served by L2, which takes more loads in
                                               flight than DRAM rewards (P = 256, m = 4 KiB: 85.0 us against

@@ -106,7 +106,7 @@ struct sparbit_plan_s {
         1000000000u,  // BULK_MIN_MOVED_BYTES
         1,            // FLOW_UNITS_PER_WARP
         8,            // FLOW_MAX_UNIT_SPANS
-        450000000u,   // FLOW_MIN_MOVED_BYTES
+        400000000u,   // FLOW_MIN_MOVED_BYTES
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
         1,            // FLOW_MIN_PASS_SPANS (every pass; 0: passes of at least one span per resident warp)
@@ -442,18 +442,19 @@ bool mirror_possible(const sparbit_plan_s* p, int first, int last, size_t smem_l
 // neighbours), so the default is 1.  Returns the position of the first flow pass, or the sequence
 // length if there is none.
 // Vectors per lane and warp span in the flow kernel.  A collective that moves less than
-// FLOW_WIDE_MAX_MOVED_BYTES in blocks of at least two wide spans (4 KiB in 16-byte vectors) runs
+// FLOW_WIDE_MAX_MOVED_BYTES in blocks of at least one wide span (2 KiB in 16-byte vectors) runs
 // with four instead of two: half of such a collective lives in L2, which answers faster than the
 // 32 KiB of loads in flight per SM that suit DRAM can keep busy (P = 256, m = 4 KiB: 85.0 us
-// against 90.3; P = 128, m = 16 KiB: 84.3 against 88.0; P = 256, m = 6 KiB: 125.6 against 129.7).
-// From about 1 GB moved the narrow form wins (P = 256, m = 8 KiB: 168.6 us against 174.4; P = 128,
-// m = 64 KiB: 330.7 against 346.7), and smaller blocks leave a wide span half empty.
+// against 90.3; P = 362, m = 2 KiB: 85.5 against 91.4; P = 128, m = 16 KiB: 84.3 against 88.0;
+// P = 256, m = 6 KiB: 125.6 against 129.7).  From about 1 GB moved the narrow form wins (P = 256,
+// m = 8 KiB: 168.6 us against 174.4; P = 128, m = 64 KiB: 330.7 against 346.7), and blocks shorter
+// than one wide span would leave it half empty.
 int flow_unroll(const sparbit_plan_s* p, int vbytes) {
     if (p->variable) return kVecUnroll;
     const uint64_t m = p->sched.m;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * m;
     if (moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_WIDE_MAX_MOVED_BYTES] &&
-        m / (uint64_t)vbytes >= 2ull * 32 * kFlowWideUnroll)
+        m / (uint64_t)vbytes >= 32ull * kFlowWideUnroll)
         return kFlowWideUnroll;
     return kVecUnroll;
 }
@@ -503,11 +504,12 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
 //    - are most of it), so there the host's cost decides: one graph launch (2.6 us) instead of one
 //    launch per pass (4 us each).  The graph chain it is.
-//  - From about 0.45 GB moved (80 us and more) the flow executor is 1-4 % ahead of the chain: the
-//    start-up and drain of every pass overlap with its neighbours (P = 256, m = 4 KiB: 90.9 us
-//    against 92.5; P = 1000, m = 1 KiB: 324.7 against 336.5; P = 509, m = 4 KiB: 331.1 against
-//    347.1; P = 128, m = 64 KiB: 332.4 against 338.7 on the bulk engine).  At 0.27 GB it is
-//    behind (P = 128, m = 8 KiB: 48.7 against 47.1).
+//  - From about 0.4 GB moved (65 us and more) the flow executor is 1-7 % ahead of the chain: the
+//    start-up and drain of every pass overlap with its neighbours (P = 256, m = 4 KiB: 85.0 us
+//    against 92.1; P = 160, m = 8 KiB: 69.6 against 71.1; P = 1000, m = 1 KiB: 324.7 against 336.5;
+//    P = 509, m = 4 KiB: 331.1 against 347.1; P = 128, m = 64 KiB: 332.4 against 338.7 on the bulk
+//    engine).  At 0.33 GB it is behind (P = 200, m = 4 KiB: 58.5 against 56.8; P = 64, m = 40 KiB:
+//    57.4 against 53.9).
 //  - From about 6 GB moved the chain on the bulk engine wins again by 1-2 %: the pass boundaries
 //    no longer matter and the bulk engine moves a byte a little cheaper than the vector engine,
 //    which is the only one the flow executor has.

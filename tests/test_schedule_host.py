@@ -219,7 +219,7 @@ def test_flow_units_and_counters_are_consistent(algo):
             plan = sp.Plan(P, m, algo)
             plan.set_tunable(sp.TUNE_FLOW_MIN_PASS_SPANS, 0)   # a pass needs one span per resident warp
             passes = plan.last_phase + 2 - (1 if algo != sp.ALGO_BRUCK and P > 1 else 0)   # fused first pass
-            # spans of four vectors per lane (blocks of 256 vectors and more, up to the given bytes
+            # spans of four vectors per lane (blocks of 128 vectors and more, up to the given bytes
             # moved) and of two
             for wide_below in (10 ** 12, 0):
                 plan.set_tunable(sp.TUNE_FLOW_WIDE_MAX_MOVED_BYTES, wide_below)
