@@ -210,3 +210,22 @@ def test_config5_largest_point_p256_m256k_sampled(dev):
     for r in range(P):
         assert torch.equal(view[r], send), r
     plan.destroy()
+
+
+@pytest.mark.parametrize("P,m", [(4097, 3), (20011, 4), (65536, 1), (2, 1 << 30)])
+@pytest.mark.parametrize("exec_mode", [sp.EXEC_AUTO, sp.EXEC_PERSISTENT])
+def test_extreme_shapes_against_the_plain_definition(dev, P, m, exec_mode):
+    """Communicators far larger than any the paper measures (tens of thousands of ranks with
+    blocks of a few bytes; a prime P) and blocks of 1 GiB: too many messages for the oracle's lists,
+    so the whole state is checked on the device against what holds at any size - every receive
+    buffer is the concatenation of the send blocks - after a sentinel fill."""
+    plan = sp.Plan(P, m, sp.ALGO_SPARBIT, exec_mode)
+    send = torch.from_numpy(si.send_blocks(P, m, si.BASE_SEED + 8).reshape(-1)).to(dev)
+    recv = torch.full((P * P * m,), si.SENTINEL, dtype=torch.uint8, device=dev)
+    plan.allgather(send, recv)
+    assert plan.status() == sp.OK
+    view = recv.view(P, P * m)
+    step = max(1, (256 << 20) // (P * m))
+    for r0 in range(0, P, step):
+        assert bool((view[r0:r0 + step] == send).all()), (P, m, r0)
+    plan.destroy()
