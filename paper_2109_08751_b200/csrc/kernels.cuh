@@ -266,7 +266,10 @@ __device__ __forceinline__ VarTask ld_task(const VarTask* p) {
 template <typename V>
 __device__ __forceinline__ void vec_list_phase(const Geom& g, const PhaseDesc& d, const VarTask* __restrict__ list,
                                                uint64_t count, uint32_t warp_id, uint32_t n_warps, uint32_t lane) {
-    constexpr int U = kVecUnroll;
+    // four vectors per lane: blocks of arbitrary sizes rarely start on 128-byte lines, which makes
+    // every load slower, and more of them in flight make up for part of it (uniformly random sizes
+    // around 4 KiB at P = 256: 113.7 us against 128.4 with two; around 1 KiB at P = 1000: 452 against 486)
+    constexpr int U = 4;
     constexpr uint32_t span = 32u * U;  // vectors per warp iteration
     const char* sbase = space_base(g, d.src_space);
     char* dbase = space_base(g, d.dst_space);
