@@ -55,7 +55,7 @@ NCU_TRAFFIC = {
     "sparbit:P1000:m1024:graph:vector": (9.79e8, "profiles/phase_vec_and_flow_kernel_P1000_m1k.md"),
     # config 5, small blocks: last pass of phase_vec_kernel (captured alone, caches cold)
     "sparbit:P256:m4096:flow:vector": (3.72e8, "profiles/flow_vec_kernel_P256_m4k.md"),
-    "sparbit:P256:m4096:graph:vector": (2.24e8, "profiles/phase_vec_kernel_P256_small_blocks.md"),
+    "sparbit:P256:m4096:graph:vector": (2.21e8, "profiles/phase_vec_kernel_P256_small_blocks.md"),
     "sparbit:P256:m512:graph:vector": (1.68e7, "profiles/phase_vec_kernel_P256_small_blocks.md"),
     "sparbit:P256:m64:graph:vector": (4.21e6, "profiles/phase_vec_kernel_P256_small_blocks.md"),
     "sparbit:P256:m8:graph:vector": (5.36e5, "profiles/phase_vec_kernel_P256_small_blocks.md"),
