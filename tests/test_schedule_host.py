@@ -35,6 +35,23 @@ def as_set(msgs):
     return {tuple(int(x) for x in m) for m in msgs}
 
 
+def test_binding_constants_match_the_header():
+    """Every SPARBIT_* enumerator of the header has the same value under the binding's name for
+    it (SPARBIT_ERR_ARG -> ERR_ARG ...): the binding spells the numbers out a second time."""
+    import re
+    header = (ROOT / "include" / "sparbit.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    seen = 0
+    for body in re.findall(r"enum\s*\{(.*?)\}", header, flags=re.S):
+        for name, value in re.findall(r"SPARBIT_([A-Z0-9_]+)\s*=\s*(-?\d+)", body):
+            if name.endswith("_"):
+                continue   # counts, not part of the binding
+            assert hasattr(sp, name), name
+            assert getattr(sp, name) == int(value), name
+            seen += 1
+    assert seen >= 45
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_descriptors_expand_to_oracle_message_sets(algo):
     """Per phase, the library's messages equal the oracle's as a set (order inside a phase is free)."""
