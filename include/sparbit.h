@@ -82,8 +82,9 @@ enum {
                                     fast), FLOW for collectives that move 0.4 to 6 GB (unless
                                     COPY_AUTO gives them the bulk engine and m is not a multiple
                                     of 128 B: the vector engine, which FLOW runs on, is 10-30 %
-                                    slower on blocks that straddle 128-byte lines), the graph
-                                    chain otherwise (thresholds: SPARBIT_TUNE_*) */
+                                    slower on blocks that straddle 128-byte lines), the chain of
+                                    per-pass kernels otherwise - as a graph, or kernel by kernel
+                                    (STREAM) while it is short (thresholds: SPARBIT_TUNE_*) */
     SPARBIT_EXEC_PERSISTENT = 1, /* one cooperative kernel, bounded-wait grid barrier per pass */
     SPARBIT_EXEC_GRAPH = 2,      /* one kernel per pass, chained by programmatic dependent launch
                                     in a CUDA graph cached per buffer set (4 sets; further sets
@@ -91,7 +92,9 @@ enum {
                                     (and recursive doubling's) leading passes share ONE kernel
                                     where the ranks fall into independent groups small enough
                                     for a CTA each (SPARBIT_TUNE_GROUPED_FRONT) */
-    SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream */
+    SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream; what AUTO
+                                    resolves to where it says "the graph chain" below and the
+                                    chain is short (SPARBIT_TUNE_STREAM_MAX_LAUNCHES) */
     SPARBIT_EXEC_FLOW = 4,       /* one kernel (all CTAs resident) without grid barriers:
                                     Algorithm 1's Waitall is kept per rank (counters of what each
                                     rank has received), so a pass starts where its senders are
@@ -465,7 +468,13 @@ enum {
                                               buffers total at most this (256 MiB, about twice the L2) a full
                                               per-pass kernel runs three CTAs per SM instead of two (1-5 %:
                                               P = 256, m = 2 KiB 45.4 us against 46.7); 0 = never */
-    SPARBIT_TUNE_COUNT_ = 17
+    SPARBIT_TUNE_STREAM_MAX_LAUNCHES = 17, /* EXEC_AUTO: a chain of per-pass kernels on the vector engine that
+                                              needs at most this many launches (6; the grouped front counts
+                                              as one) is launched kernel by kernel (STREAM) instead of as a
+                                              graph: back-to-back graph launches start 1-2 us apart from one
+                                              another where plain launches overlap (P = 256, m = 8 B: 10.0 us
+                                              against 12.3); 0 = always GRAPH */
+    SPARBIT_TUNE_COUNT_ = 18
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);
 int sparbit_plan_get_tunable(const sparbit_plan_t* plan, int key, uint64_t* value);

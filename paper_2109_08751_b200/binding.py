@@ -26,7 +26,8 @@ MAP_SEQUENTIAL, MAP_CYCLIC = range(2)
  TUNE_FLOW_MIN_MOVED_BYTES, TUNE_FLOW_MAX_MOVED_BYTES, TUNE_MIRROR_MAX_BYTES,
  TUNE_FLOW_MIN_PASS_SPANS, TUNE_MIRROR_MAX_VECTORS, TUNE_MIRROR_CLUSTER_MAX_BLOCK,
  TUNE_MIRROR_CTA_VECTORS, TUNE_MIRROR_THREAD_VECTORS, TUNE_FLOW_COOPERATIVE, TUNE_FLOW_SKIP_WAITS,
- TUNE_GROUPED_FRONT, TUNE_FLOW_WIDE_MAX_MOVED_BYTES, TUNE_VEC_DENSE_MAX_RECV_BYTES) = range(17)
+ TUNE_GROUPED_FRONT, TUNE_FLOW_WIDE_MAX_MOVED_BYTES, TUNE_VEC_DENSE_MAX_RECV_BYTES,
+ TUNE_STREAM_MAX_LAUNCHES) = range(18)
 
 ALGO_NAMES = {ALGO_SPARBIT: "sparbit", ALGO_RING: "ring", ALGO_RECURSIVE_DOUBLING: "recursive_doubling",
               ALGO_BRUCK: "bruck", ALGO_NEIGHBOR_EXCHANGE: "neighbor_exchange"}

@@ -119,6 +119,7 @@ struct sparbit_plan_s {
         1,            // GROUPED_FRONT
         900000000u,   // FLOW_WIDE_MAX_MOVED_BYTES
         256u << 20,   // VEC_DENSE_MAX_RECV_BYTES
+        6,            // STREAM_MAX_LAUNCHES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -502,8 +503,11 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 //  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
 //    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
-//    - are most of it), so there the host's cost decides: one graph launch (2.6 us) instead of one
-//    launch per pass (4 us each).  The graph chain it is.
+//    - are most of it), so there the launches decide.  One graph launch costs the host the same
+//    whatever the graph holds, which a long chain needs; but back-to-back graph launches start a
+//    microsecond or two apart where plain launches with programmatic stream serialisation overlap,
+//    so a chain of at most STREAM_MAX_LAUNCHES kernels is launched kernel by kernel (chain_exec),
+//    and so are the one-kernel executors.
 //  - From about 0.4 GB moved (65 us and more) the flow executor is 1-7 % ahead of the chain: the
 //    start-up and drain of every pass overlap with its neighbours (P = 256, m = 4 KiB: 85.0 us
 //    against 92.1; P = 160, m = 8 KiB: 69.6 against 71.1; P = 1000, m = 1 KiB: 324.7 against 336.5;
@@ -586,15 +590,47 @@ int auto_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
     return SPARBIT_EXEC_GRAPH;
 }
 
+// Kernels a call launches on the chain (graph or stream executor, vector engine): one per pass,
+// the grouped front counting as one.
+int chain_launches(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    const ExecSeq seq = make_seq(p, first, last);
+    uint32_t groups = 1;
+    const int f = front_passes(p, seq, vbytes, &groups);
+    return f ? 1 + seq.count() - f : seq.count();
+}
+
+// GRAPH or STREAM for a chain on the vector engine.  A graph launch costs the host the same whatever
+// the graph holds, but back-to-back graph launches start on a coarser grid than plain launches
+// with programmatic stream serialisation do, about 1-2 us per collective: a chain of up to
+// STREAM_MAX_LAUNCHES kernels is launched kernel by kernel (P = 256, m = 8 B, three launches: 10.0 us
+// against 12.3; P = 64, m = 64 B, two: 6.8 against 8.2), longer ones as a graph, where the host's
+// cost per launch would show.
+int chain_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
+    return (uint64_t)chain_launches(p, vbytes, first, last) <= p->tune[SPARBIT_TUNE_STREAM_MAX_LAUNCHES]
+               ? SPARBIT_EXEC_STREAM
+               : SPARBIT_EXEC_GRAPH;
+}
+
+bool auto_copy_is_bulk(const sparbit_plan_s* p, int vbytes) {
+    if (p->copy_req != SPARBIT_COPY_AUTO) return p->copy_req == SPARBIT_COPY_BULK && vbytes == 16;
+    if (vbytes != 16) return false;
+    const uint64_t block = p->variable ? p->voff.back() / p->sched.P : p->sched.m;
+    const unsigned __int128 moved = p->variable ? (unsigned __int128)2 * (p->sched.P - 1) * p->voff.back()
+                                                : (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
+    return block >= p->tune[SPARBIT_TUNE_BULK_MIN_BLOCK_BYTES] &&
+           moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_BULK_MIN_MOVED_BYTES];
+}
+
 int auto_exec_before_launch(const sparbit_plan_s* p, int vbytes) {
     const int small = small_collective_exec(p, vbytes, -1, p->sched.last_phase(), 227u << 10);
+    if (small == SPARBIT_EXEC_GRAPH) return chain_exec(p, vbytes, -1, p->sched.last_phase());
     if (small >= 0) return small;
     const unsigned __int128 moved = (unsigned __int128)2 * p->sched.P * (p->sched.P - 1) * p->sched.m;
     if (moved >= (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MIN_MOVED_BYTES] &&
         moved < (unsigned __int128)p->tune[SPARBIT_TUNE_FLOW_MAX_MOVED_BYTES] && !bulk_off_line(p, vbytes) &&
         flow_possible(p, vbytes, -1, p->sched.last_phase(), true))
         return SPARBIT_EXEC_FLOW;
-    return SPARBIT_EXEC_GRAPH;
+    return auto_copy_is_bulk(p, vbytes) ? SPARBIT_EXEC_GRAPH : chain_exec(p, vbytes, -1, p->sched.last_phase());
 }
 
 Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv, int first, int last) {
@@ -627,7 +663,10 @@ Resolved resolve(const sparbit_plan_s* p, const void* send, const void* recv, in
     if (copy == SPARBIT_COPY_BULK && !bulk_possible) copy = SPARBIT_COPY_VECTOR;
     r.copy = copy;
     int exec = p->exec_req;
-    if (exec == SPARBIT_EXEC_AUTO) exec = auto_exec(p, r.vbytes, first, last);
+    if (exec == SPARBIT_EXEC_AUTO) {
+        exec = auto_exec(p, r.vbytes, first, last);
+        if (exec == SPARBIT_EXEC_GRAPH && r.copy == SPARBIT_COPY_VECTOR) exec = chain_exec(p, r.vbytes, first, last);
+    }
     if (exec == SPARBIT_EXEC_PERSISTENT && !p->coop) exec = SPARBIT_EXEC_GRAPH;
     if (exec == SPARBIT_EXEC_MIRROR && !mirror_possible(p, first, last, (size_t)p->max_smem_optin))
         exec = SPARBIT_EXEC_GRAPH;
@@ -1372,7 +1411,7 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
         case SPARBIT_EXEC_PERSISTENT: rc = launch_persistent(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_GRAPH: rc = launch_graph(p, rs, g, first, last, st); break;
         case SPARBIT_EXEC_FLOW: rc = launch_flow(p, rs, g, first, last, st); break;
-        case SPARBIT_EXEC_MIRROR: rc = launch_graph(p, rs, g, first, last, st); break;  // a graph of one kernel
+        case SPARBIT_EXEC_MIRROR: rc = launch_mirror(p, rs, g, first, last, st); break;
         default: rc = launch_stream(p, rs, g, first, last, st); break;
     }
     if (rc == SPARBIT_OK) {

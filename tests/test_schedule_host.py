@@ -155,12 +155,13 @@ def test_exec_mode_resolution():
     assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
     assert sp.Plan(45, 512).exec_mode == sp.EXEC_MIRROR          # 1 MiB, no power of two divides 45: a cluster of CTAs
     assert sp.Plan(253, 1).exec_mode == sp.EXEC_MIRROR           # 63 KiB but 32 Ki one-byte vectors: a cluster too
-    assert sp.Plan(32, 128).exec_mode == sp.EXEC_GRAPH           # 128 KiB: the chain, its first four passes as 2 groups of 16 ranks
-    assert sp.Plan(128, 64).exec_mode == sp.EXEC_GRAPH           # 1 MiB: the chain, four passes as 8 groups of 16
-    assert sp.Plan(256, 64).exec_mode == sp.EXEC_GRAPH           # 4 MiB: the chain, five passes as 8 groups of 32
-    assert sp.Plan(128, 128).exec_mode == sp.EXEC_GRAPH          # 2 MiB
+    assert sp.Plan(32, 128).exec_mode == sp.EXEC_STREAM          # 128 KiB: the chain, its first four passes as 2 groups of 16 ranks;
+                                                                 # two launches: kernel by kernel, not as a graph
+    assert sp.Plan(128, 64).exec_mode == sp.EXEC_STREAM          # 1 MiB: the chain, four passes as 8 groups of 16, then three
+    assert sp.Plan(256, 64).exec_mode == sp.EXEC_STREAM          # 4 MiB: the chain, five passes as 8 groups of 32, then three
+    assert sp.Plan(128, 128).exec_mode == sp.EXEC_STREAM         # 2 MiB
     assert sp.Plan(13, 4096).exec_mode == sp.EXEC_MIRROR         # 676 KiB of 4 KiB blocks, odd P: a cluster
-    assert sp.Plan(8, 8192).exec_mode == sp.EXEC_GRAPH           # 512 KiB of larger blocks: the chain
+    assert sp.Plan(8, 8192).exec_mode == sp.EXEC_STREAM          # 512 KiB of larger blocks: the chain, three launches
     assert sp.Plan(8, 8192, exec_mode=sp.EXEC_MIRROR).exec_mode == sp.EXEC_MIRROR   # but it fits, on request
     assert sp.Plan(6, 4096, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR     # 144 KiB, and as much of working buffers
     assert sp.Plan(8, 64, sp.ALGO_BRUCK).exec_mode == sp.EXEC_MIRROR
@@ -168,11 +169,14 @@ def test_exec_mode_resolution():
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
     assert sp.Plan(256, 4096).exec_mode == sp.EXEC_FLOW           # 0.53 GB moved
-    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_GRAPH          # 0.27 GB moved
+    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_GRAPH          # 0.27 GB moved, seven launches: a graph
     assert sp.Plan(128, 65520).exec_mode == sp.EXEC_GRAPH         # blocks off 128-byte lines stay on the bulk engine
     assert sp.Plan(128, 65520, ).exec_mode != sp.Plan(128, 65536).exec_mode
     assert sp.Plan(1000, 1008).exec_mode == sp.EXEC_FLOW          # ... where COPY_AUTO would pick it (m >= 8 KiB)
-    assert sp.Plan(40000, 1).exec_mode == sp.EXEC_GRAPH           # blocks shorter than a warp row
+    assert sp.Plan(40000, 1).exec_mode == sp.EXEC_GRAPH           # blocks shorter than a warp row, 16 launches
+    short = sp.Plan(128, 64)
+    short.set_tunable(sp.TUNE_STREAM_MAX_LAUNCHES, 0)             # never kernel by kernel
+    assert short.exec_mode == sp.EXEC_GRAPH
     assert sp.Plan(256, 65536, exec_mode=sp.EXEC_PERSISTENT).exec_mode == sp.EXEC_PERSISTENT
 
 
@@ -195,7 +199,7 @@ def test_environment_overrides_only_the_automatic_choice(monkeypatch):
     monkeypatch.setenv("SPARBIT_EXEC", "flow")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_FLOW
     assert sp.Plan.create_v([16, 32]).exec_mode == sp.EXEC_MIRROR                 # flow is not offered there: AUTO's own pick
-    assert sp.Plan.create_v([70000, 80000]).exec_mode == sp.EXEC_GRAPH
+    assert sp.Plan.create_v([70000, 80000]).exec_mode == sp.EXEC_STREAM              # one launch: a plain one
     monkeypatch.setenv("SPARBIT_EXEC", "nonsense")
     assert sp.Plan(8, 64).exec_mode == sp.EXEC_MIRROR
 
