@@ -431,7 +431,7 @@ enum {
                                               warp, 4736 on B200); smaller leading passes run as chained
                                               per-pass kernels in front of it */
     SPARBIT_TUNE_MIRROR_MAX_VECTORS = 8,   /* EXEC_AUTO: MIRROR only when the largest pass moves at most this
-                                              many vectors (40960: 1 MiB of receive buffers in 16-byte
+                                              many vectors (65536: 2 MiB of receive buffers in 16-byte
                                               vectors) ... */
     SPARBIT_TUNE_MIRROR_CLUSTER_MAX_BLOCK = 9, /* ... and, where P*P*m exceeds MIRROR_MAX_BYTES, m is at most
                                               this (4 KiB) */
@@ -469,7 +469,7 @@ enum {
                                               per-pass kernel runs three CTAs per SM instead of two (1-5 %:
                                               P = 256, m = 2 KiB 45.4 us against 46.7); 0 = never */
     SPARBIT_TUNE_STREAM_MAX_LAUNCHES = 17, /* EXEC_AUTO: a chain of per-pass kernels on the vector engine that
-                                              needs at most this many launches (6; the grouped front counts
+                                              needs at most this many launches (8; the grouped front counts
                                               as one) is launched kernel by kernel (STREAM) instead of as a
                                               graph: back-to-back graph launches start 1-2 us apart from one
                                               another where plain launches overlap (P = 256, m = 8 B: 10.0 us

@@ -110,7 +110,7 @@ struct sparbit_plan_s {
         6000000000ull,  // FLOW_MAX_MOVED_BYTES
         64u << 10,    // MIRROR_MAX_BYTES
         1,            // FLOW_MIN_PASS_SPANS (every pass; 0: passes of at least one span per resident warp)
-        40960,        // MIRROR_MAX_VECTORS
+        65536,        // MIRROR_MAX_VECTORS
         4096,         // MIRROR_CLUSTER_MAX_BLOCK
         256,          // MIRROR_CTA_VECTORS
         4,            // MIRROR_THREAD_VECTORS
@@ -119,7 +119,7 @@ struct sparbit_plan_s {
         1,            // GROUPED_FRONT
         900000000u,   // FLOW_WIDE_MAX_MOVED_BYTES
         256u << 20,   // VEC_DENSE_MAX_RECV_BYTES
-        6,            // STREAM_MAX_LAUNCHES
+        8,            // STREAM_MAX_LAUNCHES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -544,9 +544,12 @@ int front_passes(const sparbit_plan_s* p, const ExecSeq& seq, int vbytes, uint32
 // enough for it.  Beyond that the mirror executor on a cluster (about 3.5 us + 0.8 us per pass) or
 // the chain with its leading passes in the grouped mirror kernel (4.2-6.2 us for those + 2.05 us
 // per pass after them), whichever comes out shorter: the chain when at most three passes follow
-// the grouped ones (measured: P = 256, m = 8 B 10.4 us against 14.4; P = 128, m = 128 B 10.3
-// against 14.8; equal at P = 64 and 128 with m = 64 B).  P without a suitable power-of-two divisor
-// has no groups: the cluster it is (P = 253, m = 1 B 14.4 against 18.5 for the plain chain).
+// the grouped ones and the largest pass has more than 16 Ki vectors (measured, GPU time per
+// collective: P = 256, m = 8 B 9.8 us against 11.7; P = 128, m = 128 B 10.0 against 13.3; P = 64,
+// m = 512 B 8.6 against 12.6; but P = 64, m = 64 B 6.7 against 6.1 on the cluster, P = 32, m = 512 B
+// 6.7 against 6.1, P = 16, m = 1 KiB 5.6 against 5.0).  P without a suitable power-of-two divisor
+// has no groups: the cluster it is (P = 253, m = 1 B 13.6 against 18.5 for the plain chain;
+// P = 181, m = 64 B 14.2 against 18.5).
 int small_collective_exec(const sparbit_plan_s* p, int vbytes, int first, int last, size_t smem_limit) {
     if (!mirror_possible(p, first, last, smem_limit) || !mirror_wins(p, vbytes, first, last)) return -1;
     if (p->variable) return SPARBIT_EXEC_MIRROR;
@@ -562,7 +565,7 @@ int small_collective_exec(const sparbit_plan_s* p, int vbytes, int first, int la
         return SPARBIT_EXEC_MIRROR;
     uint32_t groups = 1;
     const int s = front_passes(p, seq, vbytes, &groups);
-    if (s >= 3 && seq.count() - s <= 3) return SPARBIT_EXEC_GRAPH;
+    if (s >= 3 && seq.count() - s <= 3 && most > 16384) return SPARBIT_EXEC_GRAPH;
     return SPARBIT_EXEC_MIRROR;
 }
 
@@ -603,8 +606,9 @@ int chain_launches(const sparbit_plan_s* p, int vbytes, int first, int last) {
 // the graph holds, but back-to-back graph launches start on a coarser grid than plain launches
 // with programmatic stream serialisation do, about 1-2 us per collective: a chain of up to
 // STREAM_MAX_LAUNCHES kernels is launched kernel by kernel (P = 256, m = 8 B, three launches: 10.0 us
-// against 12.3; P = 64, m = 64 B, two: 6.8 against 8.2), longer ones as a graph, where the host's
-// cost per launch would show.
+// against 12.3; P = 64, m = 64 B, two: 6.8 against 8.2; P = 256, m = 64 B without the grouped front,
+// eight: 17.5 against 18.5), longer ones as a graph, where the host's cost per launch would show
+// (ten launches at P = 1000, m = 1 KiB: 334 us either way).
 int chain_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
     return (uint64_t)chain_launches(p, vbytes, first, last) <= p->tune[SPARBIT_TUNE_STREAM_MAX_LAUNCHES]
                ? SPARBIT_EXEC_STREAM

@@ -155,8 +155,10 @@ def test_exec_mode_resolution():
     assert sp.Plan(32, 64).exec_mode == sp.EXEC_MIRROR           # 64 KiB
     assert sp.Plan(45, 512).exec_mode == sp.EXEC_MIRROR          # 1 MiB, no power of two divides 45: a cluster of CTAs
     assert sp.Plan(253, 1).exec_mode == sp.EXEC_MIRROR           # 63 KiB but 32 Ki one-byte vectors: a cluster too
-    assert sp.Plan(32, 128).exec_mode == sp.EXEC_STREAM          # 128 KiB: the chain, its first four passes as 2 groups of 16 ranks;
-                                                                 # two launches: kernel by kernel, not as a graph
+    assert sp.Plan(32, 128).exec_mode == sp.EXEC_MIRROR          # 128 KiB, 4 Ki vectors in the largest pass: a cluster beats the
+                                                                 # chain even with the chain's first four passes in one kernel
+    assert sp.Plan(64, 512).exec_mode == sp.EXEC_STREAM          # 2 MiB, 64 Ki vectors: the chain, three passes as 8 groups of 8
+                                                                 # ranks, then three: kernel by kernel, not as a graph
     assert sp.Plan(128, 64).exec_mode == sp.EXEC_STREAM          # 1 MiB: the chain, four passes as 8 groups of 16, then three
     assert sp.Plan(256, 64).exec_mode == sp.EXEC_STREAM          # 4 MiB: the chain, five passes as 8 groups of 32, then three
     assert sp.Plan(128, 128).exec_mode == sp.EXEC_STREAM         # 2 MiB
@@ -169,7 +171,9 @@ def test_exec_mode_resolution():
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
     assert sp.Plan(256, 4096).exec_mode == sp.EXEC_FLOW           # 0.53 GB moved
-    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_GRAPH          # 0.27 GB moved, seven launches: a graph
+    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_STREAM         # 0.27 GB moved, seven launches: kernel by kernel
+    assert sp.Plan(512, 2048).exec_mode == sp.EXEC_FLOW           # 1.07 GB moved
+    assert sp.Plan(300, 1024).exec_mode == sp.EXEC_GRAPH          # 0.18 GB moved, nine launches: a graph
     assert sp.Plan(128, 65520).exec_mode == sp.EXEC_GRAPH         # blocks off 128-byte lines stay on the bulk engine
     assert sp.Plan(128, 65520, ).exec_mode != sp.Plan(128, 65536).exec_mode
     assert sp.Plan(1000, 1008).exec_mode == sp.EXEC_FLOW          # ... where COPY_AUTO would pick it (m >= 8 KiB)
