@@ -472,8 +472,8 @@ enum {
                                               needs at most this many launches (8; the grouped front counts
                                               as one) is launched kernel by kernel (STREAM) instead of as a
                                               graph: back-to-back graph launches start 1-2 us apart from one
-                                              another where plain launches overlap (P = 256, m = 8 B: 10.0 us
-                                              against 12.3); 0 = always GRAPH */
+                                              another where plain launches overlap (P = 256, m = 8 B: 9.8 us
+                                              against 11.8); 0 = always GRAPH */
     SPARBIT_TUNE_COUNT_ = 18
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);

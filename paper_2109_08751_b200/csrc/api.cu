@@ -491,15 +491,15 @@ bool flow_possible(const sparbit_plan_s* p, int vbytes, int first, int last, boo
 
 // Executor for SPARBIT_EXEC_AUTO, from measurements on B200.
 //  - Up to 64 KiB of receive buffers in all, the mirror executor: one CTA, passes separated by its
-//    own barrier and fed from shared memory (P = 8, m = 64 B: 4.1 us against 6.2 for the chain;
-//    P = 32, m = 64 B: 6.2 against 10.3).  Above that one CTA's bandwidth eats the gain, and a
-//    cluster of CTAs with the copies in distributed shared memory takes over, up to 40 Ki vectors
-//    in the largest pass (1 MiB of receive buffers in 16-byte vectors; blocks of a few bytes make
-//    as many vectors of a few bytes: P = 253, m = 1 B runs on a cluster too, 14.4 against 20.2 for
-//    the chain and 36.8 in one CTA) with blocks of at most 4 KiB (P = 64, m = 64 B: 8.2 against 14.4; P = 128,
-//    m = 64 B: 10.3 against 16.4; P = 256, m = 8 B: 14.4 against 20.5; P = 16, m = 4 KiB: 8.2
-//    against 9.2): a pass is one push through the SM-to-SM network and an mbarrier, about 0.8 us.
-//    Beyond 1 MiB sixteen SMs' bandwidth eats the gain (P = 64, m = 512 B: 14.4 against 12.3).
+//    own barrier and fed from shared memory (GPU time per collective, back to back: P = 8, m = 64 B
+//    2.5 us against 4.7 for the chain; P = 32, m = 64 B: 5.5 against 9.1).  Above that one CTA's
+//    bandwidth eats the gain, and a cluster of CTAs with the copies in distributed shared memory
+//    takes over, up to 64 Ki vectors in the largest pass (2 MiB of receive buffers in 16-byte
+//    vectors; blocks of a few bytes make as many vectors of a few bytes: P = 253, m = 1 B runs on a
+//    cluster too, 13.6 against 18.5 for the chain and 36.8 in one CTA) with blocks of at most 4 KiB
+//    (P = 64, m = 64 B: 6.1 against 11.5; P = 181, m = 64 B: 14.2 against 18.5; P = 16, m = 4 KiB: 7.2
+//    either way): a pass is one push through the SM-to-SM network and an mbarrier, about 0.8 us.
+//    Beyond that sixteen SMs' bandwidth eats the gain (P = 100, m = 200 B: 16.4 either way).
 //  - A pass costs 1.6-2.3 us of GPU time in the latency regime whichever way it is separated from
 //    the next one (kernel boundary with programmatic dependent launch, a CTA's own barrier, a grid
 //    barrier, per-rank counters: two memory round trips - the loads, then the acknowledged stores
