@@ -316,14 +316,16 @@ const void* pick_persistent_vec(int vbytes, bool list = false) {
     }
 }
 template <typename V>
-const void* mirror_vec_fn() { return (const void*)mirror_vec_kernel<V>; }
-const void* pick_mirror_vec(int vbytes) {
+const void* mirror_vec_fn(bool work) {
+    return work ? (const void*)mirror_vec_kernel<V, true> : (const void*)mirror_vec_kernel<V, false>;
+}
+const void* pick_mirror_vec(int vbytes, bool work) {
     switch (vbytes) {
-        case 16: return mirror_vec_fn<uint4>();
-        case 8: return mirror_vec_fn<uint2>();
-        case 4: return mirror_vec_fn<unsigned>();
-        case 2: return mirror_vec_fn<unsigned short>();
-        default: return mirror_vec_fn<unsigned char>();
+        case 16: return mirror_vec_fn<uint4>(work);
+        case 8: return mirror_vec_fn<uint2>(work);
+        case 4: return mirror_vec_fn<unsigned>(work);
+        case 2: return mirror_vec_fn<unsigned short>(work);
+        default: return mirror_vec_fn<unsigned char>(work);
     }
 }
 template <typename V>
@@ -1087,7 +1089,7 @@ int launch_persistent(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int 
 // maximum (asking for less per launch costs nothing), so that no plan can lower it under another.
 constexpr int kSmemDevices = 64;
 std::mutex g_smem_mutex;
-bool g_smem_granted[kSmemDevices][32];
+bool g_smem_granted[kSmemDevices][40];
 int vec_slot(int vbytes) { return vbytes == 16 ? 4 : vbytes == 8 ? 3 : vbytes == 4 ? 2 : vbytes == 2 ? 1 : 0; }
 int grant_max_smem(const sparbit_plan_s* p, const void* fn, int slot, bool big_cluster) {
     std::lock_guard<std::mutex> lock(g_smem_mutex);
@@ -1195,7 +1197,8 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
     Geom gg = g;
     void* args[] = {&gg, &ma};
     for (;;) {
-        const void* fn = C == 1 ? pick_mirror_vec(rs.vbytes) : pick_cluster_mirror_vec(rs.vbytes);
+        const bool work = p->sched.algo == ALGO_BRUCK;  // the only schedule with working buffers
+        const void* fn = C == 1 ? pick_mirror_vec(rs.vbytes, work) : pick_cluster_mirror_vec(rs.vbytes);
         const size_t ranks = (P + C - 1) / C;
         size_t smem = ranks * P * p->sched.m;
         ma.work_at = 0;
@@ -1209,7 +1212,7 @@ int launch_mirror(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
         threads = (threads + 63) / 64 * 64;
         if (threads > 1024) threads = 1024;
         {
-            const int grc = grant_max_smem(p, fn, (C == 1 ? 0 : 8) + vec_slot(rs.vbytes), C > 1);
+            const int grc = grant_max_smem(p, fn, (C == 1 ? (work ? 32 : 0) : 8) + vec_slot(rs.vbytes), C > 1);
             if (grc) return grc;
         }
         memset(&cfg, 0, sizeof cfg);

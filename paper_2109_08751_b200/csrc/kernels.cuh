@@ -698,7 +698,9 @@ struct MirrorArgs {
     unsigned long long magic_copies[kMirrorMaxPasses];
 };
 
-template <typename V>
+// kWork: the collective has working buffers (Bruck); without them every pass writes the receive
+// space and the space look-ups fold away.
+template <typename V, bool kWork>
 __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __grid_constant__ MirrorArgs ma) {
     // [P][P] slots of m bytes, laid out as the RECV space; for Bruck a second such array for its
     // working buffers behind it
@@ -714,9 +716,9 @@ __global__ void __launch_bounds__(1024, 1) mirror_vec_kernel(Geom g, const __gri
         const uint32_t vpc = (uint32_t)(d.copy_bytes / sizeof(V));
         const uint32_t total = P * d.copies * vpc;  // fits: the whole receive space is below 256 KiB
         const bool from_send = d.src_space == SPACE_SEND;
-        const V* msrc = mir + (d.src_space == SPACE_WORK ? ma.work_at : 0u);
-        V* mdst = mir + (d.dst_space == SPACE_WORK ? ma.work_at : 0u);
-        V* gdst = reinterpret_cast<V*>(space_base(g, d.dst_space));
+        const V* msrc = mir + (kWork && d.src_space == SPACE_WORK ? ma.work_at : 0u);
+        V* mdst = mir + (kWork && d.dst_space == SPACE_WORK ? ma.work_at : 0u);
+        V* gdst = reinterpret_cast<V*>(kWork ? space_base(g, d.dst_space) : g.base[SPACE_RECV]);
         const unsigned long long mv = ma.magic_vpc[i], mc = ma.magic_copies[i];
         for (uint32_t t = threadIdx.x; t < total; t += blockDim.x) {
             const uint32_t q = (uint32_t)((t * mv) >> 40);  // t / vpc
