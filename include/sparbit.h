@@ -93,8 +93,8 @@ enum {
                                     where the ranks fall into independent groups small enough
                                     for a CTA each (SPARBIT_TUNE_GROUPED_FRONT) */
     SPARBIT_EXEC_STREAM = 3,     /* the same kernels launched one by one on the stream; what AUTO
-                                    resolves to where it says "the graph chain" below and the
-                                    chain is short (SPARBIT_TUNE_STREAM_MAX_LAUNCHES) */
+                                    resolves to for a chain of few kernels
+                                    (SPARBIT_TUNE_STREAM_MAX_LAUNCHES) */
     SPARBIT_EXEC_FLOW = 4,       /* one kernel (all CTAs resident) without grid barriers:
                                     Algorithm 1's Waitall is kept per rank (counters of what each
                                     rank has received), so a pass starts where its senders are
