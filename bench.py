@@ -157,8 +157,9 @@ def head_start(us_per_collective):
     the whole batch, and what lies between the two stamps is GPU time.  None = not measured yet:
     treated as short."""
     import torch
-    if us_per_collective is None or us_per_collective < HEAD_START_BELOW_US:
-        torch.cuda._sleep(HEAD_START_CYCLES)
+    spin = getattr(torch.cuda, "_sleep", None)   # torch's spinning kernel; without it the batch is timed as it comes
+    if spin is not None and (us_per_collective is None or us_per_collective < HEAD_START_BELOW_US):
+        spin(HEAD_START_CYCLES)
 
 
 def whole_job_value(world: int, P: int, m: int, ms_per_step: float) -> float:
