@@ -606,14 +606,30 @@ def run_sweep(args):
                         e1.record(stream)
                         stream.synchronize()
                         us.append(e0.elapsed_time(e1) / 50 * 1e3)
+                    k_after = plan.launch_counts()[0]
+                    # the same loop as the host feeds it (no delay in front: short collectives are then
+                    # bound by the launches of this Python loop, 3-4 us per call and more per plain
+                    # kernel launch; reported beside the GPU time, not instead of it)
+                    fed = None
+                    if float(np.mean(us)) < HEAD_START_BELOW_US:
+                        fed = []
+                        for _ in range(3):
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record(stream)
+                            for it in range(50):
+                                plan.allgather(sends[it & 1], recv, stream)
+                            e1.record(stream)
+                            stream.synchronize()
+                            fed.append(e0.elapsed_time(e1) / 50 * 1e3)
                 assert plan.status() == sp.OK
                 ok = bool(torch.equal(recv.view(P, P * m)[P - 1], sends[1]))
                 avg = float(np.mean(us))
                 print(json.dumps({
                     "algo": name, "exec": ename, "copy": cname, "P": P, "m": m,
                     "ran": f"{sp.EXEC_NAMES[plan.exec_mode]}/{sp.COPY_NAMES[plan.copy_path]}",
-                    "launches_per_collective": (plan.launch_counts()[0] - k_before) / 500,
+                    "launches_per_collective": (k_after - k_before) / 500,
                     "us_min": round(min(us), 2), "us_avg": round(avg, 2), "us_max": round(max(us), 2),
+                    "us_host_fed": round(min(fed), 2) if fed else None,
                     "GBps_avg": round(effective_bytes(P, m) / avg / 1e3, 1),
                     "GBps_min_time": round(effective_bytes(P, m) / min(us) / 1e3, 1),
                     "pct_measured_peak": round(100 * effective_bytes(P, m) / avg / 1e3 / peak, 1),

@@ -469,11 +469,14 @@ enum {
                                               per-pass kernel runs three CTAs per SM instead of two (1-5 %:
                                               P = 256, m = 2 KiB 45.4 us against 46.7); 0 = never */
     SPARBIT_TUNE_STREAM_MAX_LAUNCHES = 17, /* EXEC_AUTO: a chain of per-pass kernels on the vector engine that
-                                              needs at most this many launches (8; the grouped front counts
+                                              needs at most this many launches (6; the grouped front counts
                                               as one) is launched kernel by kernel (STREAM) instead of as a
                                               graph: back-to-back graph launches start 1-2 us apart from one
                                               another where plain launches overlap (P = 256, m = 8 B: 9.8 us
-                                              against 11.8); 0 = always GRAPH */
+                                              of GPU time against 11.8), but each plain launch costs the host
+                                              2-3 us where a whole graph costs it 1.8 us, so longer chains
+                                              would leave a caller in a tight loop bound by its own
+                                              launches; 0 = always GRAPH */
     SPARBIT_TUNE_COUNT_ = 18
 };
 int sparbit_plan_set_tunable(sparbit_plan_t* plan, int key, uint64_t value);

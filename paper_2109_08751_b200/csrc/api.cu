@@ -89,6 +89,15 @@ struct sparbit_plan_s {
     unsigned* d_flow_cnt = nullptr;  // flow executor: [P][kFlowMaxPasses] unit counters
     unsigned flow_epoch = 0;         // flow launches since the counters were last cleared
     int flow_vbytes = 0;             // vector width and vectors per lane (width * 16 + unroll) of those launches
+    // what resolve() gave for (vector width, phase range) under the current settings: the automatic
+    // choices walk the schedule several times, too much for every call of a 2 us collective
+    struct {
+        bool valid = false;
+        int vbytes = 0, first = 0, last = 0;
+        uint64_t version = 0;
+        int exec = 0, copy = 0;
+    } resolved;
+    uint64_t settings_version = 0;  // bumped by every setter the automatic choices depend on
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -119,7 +128,7 @@ struct sparbit_plan_s {
         1,            // GROUPED_FRONT
         900000000u,   // FLOW_WIDE_MAX_MOVED_BYTES
         256u << 20,   // VEC_DENSE_MAX_RECV_BYTES
-        8,            // STREAM_MAX_LAUNCHES
+        6,            // STREAM_MAX_LAUNCHES
     };
 
     // cached graphs: one instantiated chain per (buffers, phase range, engine), a few of them so
@@ -604,13 +613,17 @@ int chain_launches(const sparbit_plan_s* p, int vbytes, int first, int last) {
     return f ? 1 + seq.count() - f : seq.count();
 }
 
-// GRAPH or STREAM for a chain on the vector engine.  A graph launch costs the host the same whatever
-// the graph holds, but back-to-back graph launches start on a coarser grid than plain launches
-// with programmatic stream serialisation do, about 1-2 us per collective: a chain of up to
-// STREAM_MAX_LAUNCHES kernels is launched kernel by kernel (P = 256, m = 8 B, three launches: 10.0 us
-// against 12.3; P = 64, m = 64 B, two: 6.8 against 8.2; P = 256, m = 64 B without the grouped front,
-// eight: 17.5 against 18.5), longer ones as a graph, where the host's cost per launch would show
-// (ten launches at P = 1000, m = 1 KiB: 334 us either way).
+// GRAPH or STREAM for a chain on the vector engine.  Back-to-back graph launches start on a grid
+// of about 2 us; plain launches with programmatic stream serialisation overlap, which is worth 1-2 us
+// of GPU time per collective (P = 256, m = 8 B, three launches: 9.8 us against 11.8; P = 64, m = 64 B,
+// two: 6.7 against 8.2; P = 64, m = 4 KiB, six: 13.4 against 14.4).  But a graph launch costs the
+// host 1.8 us whatever the graph holds and a plain launch of these kernels 2-3 us each (5 us into a
+// queue that is already deep), so a caller that issues collectives back to back becomes bound by
+// its own launches once they add up to more than the collective takes on the GPU.  Measured with
+// the host feeding the loop, six launches still come out ahead of the graph (13.4 us against 14.4
+// at P = 64, m = 4 KiB; five: 10.3 either way at P = 32, m = 4 KiB); eight would cost the host
+// about 20 us where P = 256, m = 64 B without its grouped front takes the GPU 17.5.  Hence kernel by
+// kernel up to STREAM_MAX_LAUNCHES (6), as a graph beyond.
 int chain_exec(const sparbit_plan_s* p, int vbytes, int first, int last) {
     return (uint64_t)chain_launches(p, vbytes, first, last) <= p->tune[SPARBIT_TUNE_STREAM_MAX_LAUNCHES]
                ? SPARBIT_EXEC_STREAM
@@ -1391,7 +1404,25 @@ int run_phases(sparbit_plan_s* p, const void* send, void* recv, void* stream, in
         return SPARBIT_ERR_ALIAS;
     int rc = ensure_device(p);
     if (rc) return rc;
-    const Resolved rs = resolve(p, send, recv, first, last);
+    Resolved rs;
+    {
+        const int vb = pick_vector_bytes(p, send, recv);
+        auto& c = p->resolved;
+        if (c.valid && c.vbytes == vb && c.first == first && c.last == last && c.version == p->settings_version) {
+            rs.vbytes = vb;
+            rs.exec = c.exec;
+            rs.copy = c.copy;
+        } else {
+            rs = resolve(p, send, recv, first, last);
+            c.valid = true;
+            c.vbytes = rs.vbytes;
+            c.first = first;
+            c.last = last;
+            c.version = p->settings_version;
+            c.exec = rs.exec;
+            c.copy = rs.copy;
+        }
+    }
     const Geom g = make_geom(p, send, recv);
     cudaStream_t st = (cudaStream_t)stream;
     // On a stream that is being captured the work must be replayable as it stands.  The persistent
@@ -1699,6 +1730,7 @@ int sparbit_plan_set_workspace(sparbit_plan_t* p, void* dev, size_t bytes) {
     if (bytes < sparbit_plan_workspace_bytes(p)) return SPARBIT_ERR_WORKSPACE;
     if (!dev && sparbit_plan_workspace_bytes(p) > 0) return SPARBIT_ERR_WORKSPACE;
     p->work = dev;
+    p->settings_version++;
     p->work_bytes = bytes;
     return SPARBIT_OK;
 }
@@ -1706,6 +1738,7 @@ int sparbit_plan_set_workspace(sparbit_plan_t* p, void* dev, size_t bytes) {
 int sparbit_plan_set_copy_path(sparbit_plan_t* p, int copy_path) {
     if (!p || copy_path < SPARBIT_COPY_AUTO || copy_path > SPARBIT_COPY_BULK) return SPARBIT_ERR_ARG;
     p->copy_req = copy_path;
+    p->settings_version++;
     return SPARBIT_OK;
 }
 
@@ -1720,6 +1753,7 @@ int sparbit_plan_set_tunable(sparbit_plan_t* p, int key, uint64_t value) {
         drop_graph(p);
     }
     p->tune[key] = value;
+    p->settings_version++;
     return SPARBIT_OK;
 }
 

@@ -171,7 +171,7 @@ def test_exec_mode_resolution():
     assert sp.Plan(128, 65536).exec_mode == sp.EXEC_FLOW          # 2.1 GB moved
     assert sp.Plan(1000, 1024).exec_mode == sp.EXEC_FLOW          # 2.0 GB moved
     assert sp.Plan(256, 4096).exec_mode == sp.EXEC_FLOW           # 0.53 GB moved
-    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_STREAM         # 0.27 GB moved, seven launches: kernel by kernel
+    assert sp.Plan(128, 8192).exec_mode == sp.EXEC_GRAPH          # 0.27 GB moved, seven launches: a graph
     assert sp.Plan(512, 2048).exec_mode == sp.EXEC_FLOW           # 1.07 GB moved
     assert sp.Plan(300, 1024).exec_mode == sp.EXEC_GRAPH          # 0.18 GB moved, nine launches: a graph
     assert sp.Plan(128, 65520).exec_mode == sp.EXEC_GRAPH         # blocks off 128-byte lines stay on the bulk engine
