@@ -98,6 +98,14 @@ struct sparbit_plan_s {
         int exec = 0, copy = 0;
     } resolved;
     uint64_t settings_version = 0;  // bumped by every setter the automatic choices depend on
+    // the grouped front of the stream executor for (vector width, phase range), under the same version
+    struct {
+        bool valid = false;
+        int vbytes = 0, first = 0, last = 0;
+        uint64_t version = 0;
+        int front = 0;
+        uint32_t groups = 1;
+    } front_cache;
     unsigned bar_base = 0;
     int extra_arrivals = 0;
     unsigned long long timeout_ns = kDefaultTimeoutNs;
@@ -893,7 +901,21 @@ int launch_stream(sparbit_plan_s* p, const Resolved& rs, const Geom& g, int firs
     int front = 0;
     if (seq_end < 0 && rs.copy == SPARBIT_COPY_VECTOR) {
         uint32_t groups = 1;
-        front = front_passes(p, seq, rs.vbytes, &groups);
+        auto& fc = p->front_cache;
+        if (fc.valid && fc.vbytes == rs.vbytes && fc.first == first && fc.last == last &&
+            fc.version == p->settings_version) {
+            front = fc.front;
+            groups = fc.groups;
+        } else {
+            front = front_passes(p, seq, rs.vbytes, &groups);
+            fc.valid = true;
+            fc.vbytes = rs.vbytes;
+            fc.first = first;
+            fc.last = last;
+            fc.version = p->settings_version;
+            fc.front = front;
+            fc.groups = groups;
+        }
         if (front) {
             int rc = launch_grouped_front(p, rs, g, seq, front, groups, st);
             if (rc) return rc;
