@@ -77,7 +77,7 @@ enum {
  * the first peer's): same state after phase 0, one pass less. */
 enum {
     SPARBIT_EXEC_AUTO = 0,       /* the measured best on B200: MIRROR up to 64 KiB of receive
-                                    buffers in all (up to 1 MiB for blocks of 16 B to 4 KiB,
+                                    buffers in all (up to 2 MiB for blocks of 16 B to 4 KiB,
                                     where the chain with a grouped front is not at least as
                                     fast), FLOW for collectives that move 0.4 to 6 GB (unless
                                     COPY_AUTO gives them the bulk engine and m is not a multiple
